@@ -1,0 +1,168 @@
+/*
+ * efqat.h -- C ABI of the B200 (sm_100a) library for the EfQAT training step of a
+ * fake-quantized linear / convolution layer (EfQAT, arxiv 2411.11038).
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller unless a parameter is
+ *     documented as "host".  The library never frees or keeps caller memory.
+ *   - Calls enqueue work on `stream` and return without synchronising.  Scratch memory
+ *     comes from the caller-provided workspace `ws` (size it with the *_workspace_bytes
+ *     queries); nothing is allocated on the hot path.
+ *   - Return value: 0 (EFQAT_OK) or a negative efqat_status found on the host before any
+ *     launch.  Conditions only the device can see (a non-positive or non-finite scale, an
+ *     index out of range, a bounded wait that ran out) are recorded in a context-owned
+ *     status word read with efqat_device_status() after the caller synchronised.
+ *   - Layouts: row-major.  Linear: X[M,K], W[N,K], Y/dY[M,N] (PyTorch Linear convention,
+ *     paper Section 3.1 footnote).  Convolution: X NHWC [B,H,W,Cin], W [N,R,S,Cin],
+ *     Y/dY [B,Ho,Wo,N]; its GEMM view is M = B*Ho*Wo, K = R*S*Cin.
+ *   - Alignment: every base pointer 16-byte aligned; N % 8 == 0 and K % 8 == 0 (Cin % 8 == 0
+ *     for convolutions).  Violations return EFQAT_ERR_ALIGN; there is no slow path.
+ *   - Activations (X, dY, Y, dX) are fp32 or bf16 (efqat_dtype); weights, scales, zero
+ *     point, bias and all gradients of parameters are fp32.
+ */
+#ifndef EFQAT_H_
+#define EFQAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct efqat_ctx efqat_ctx;          /* opaque: device, SM count, status word */
+typedef struct CUstream_st* efqat_stream_t;  /* same type as cudaStream_t / CUstream */
+
+typedef enum {
+  EFQAT_OK = 0,
+  EFQAT_ERR_NULL = -1,       /* a required pointer is NULL */
+  EFQAT_ERR_SHAPE = -2,      /* a dimension is < 1 or inconsistent */
+  EFQAT_ERR_ALIGN = -3,      /* pointer or pitch alignment contract violated */
+  EFQAT_ERR_DTYPE = -4,      /* unknown efqat_dtype */
+  EFQAT_ERR_BITS = -5,       /* bit-width outside [2,8] */
+  EFQAT_ERR_MODE = -6,       /* unknown efqat_mode */
+  EFQAT_ERR_WORKSPACE = -7,  /* workspace too small or NULL */
+  EFQAT_ERR_K_RANGE = -8,    /* k_sel / budget outside its range */
+  EFQAT_ERR_UNIMPL = -9,     /* combination not built (e.g. conv stride != 1) */
+  EFQAT_ERR_CUDA = -10,      /* a CUDA runtime / driver call failed */
+  /* device-side conditions, reported by efqat_device_status (positive) */
+  EFQAT_DEV_BAD_SCALE = 1,   /* a scale was <= 0 or not finite */
+  EFQAT_DEV_BAD_INDEX = 2,   /* idx entry outside [0,N) or not strictly ascending */
+  EFQAT_DEV_WAIT_TIMEOUT = 3 /* a bounded in-kernel wait expired */
+} efqat_status;
+
+/* Table 2 of the paper: freezing granularity x selection scope. */
+typedef enum { EFQAT_CWPL = 0, EFQAT_CWPN = 1, EFQAT_LWPN = 2 } efqat_mode;
+typedef enum { EFQAT_F32 = 0, EFQAT_BF16 = 1 } efqat_dtype;
+
+/* Bit-widths b of Eq. 1 / Eq. 3.  Weights are always symmetric per output channel
+ * (Eq. 3-4); activations are per tensor, asymmetric (Eq. 1-2) unless x_symmetric != 0,
+ * in which case Z = 0 and the code range is [-(2^(b-1)-1), 2^(b-1)-1]. */
+typedef struct {
+  int w_bits;
+  int x_bits;
+  int x_symmetric;
+} efqat_qspec;
+
+/* One quantized layer.  Linear: is_conv = 0 and only M, N, K, act_dtype are read.
+ * Convolution: is_conv = 1, stride 1, pad < R; M and K must equal B*Ho*Wo and R*S*Cin. */
+typedef struct {
+  int64_t M, N, K;
+  int is_conv;
+  int B, H, W, Cin, R, S, stride, pad;
+  int act_dtype; /* efqat_dtype of X, dY, Y, dX */
+} efqat_layer_desc;
+
+/* Optional fused optimizer for the unfrozen rows (Algorithm 1, optimizer step; SGD with
+ * momentum as in the paper's Section 4): v <- momentum*v + (g + weight_decay*w);
+ * w <- w - lr*v on rows idx[] of W_inout / mom_inout (both fp32 [N,K]); other rows are
+ * never touched. */
+typedef struct {
+  float lr, momentum, weight_decay;
+  float* W_inout;
+  float* mom_inout;
+} efqat_sgd;
+
+/* ---- context ------------------------------------------------------------------- */
+/* Creates a context bound to CUDA device `device` (allocates a few hundred bytes of
+ * device memory for the status word; the only allocation the library ever makes). */
+int efqat_create(efqat_ctx** out, int device);
+int efqat_destroy(efqat_ctx* ctx);
+/* Static, human-readable name of a status code (host or device side). */
+const char* efqat_status_string(int status);
+/* Reads and clears the device status word.  Synchronises the device; call it after the
+ * stream work of interest was enqueued.  *code = 0 or an EFQAT_DEV_* value. */
+int efqat_device_status(efqat_ctx* ctx, int* code);
+
+/* ---- host-only helpers ---------------------------------------------------------- */
+/* floor(ratio * n): number of unfrozen channels for ratio r (Eq. 7). */
+int64_t efqat_ratio_to_k(double ratio, int64_t n);
+/* Checks a layer description + quantizer spec exactly as the compute calls do. */
+int efqat_validate_layer(const efqat_layer_desc* layer, const efqat_qspec* q);
+/* Workspace bytes for efqat_fq_linear_fwd / _bwd on `layer` with at most k_sel_max
+ * selected channels (pass N to cover full-QAT). */
+int efqat_workspace_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, int64_t k_sel_max, size_t* out);
+/* Workspace bytes for efqat_select_channels over L layers with total_channels rows. */
+int efqat_select_workspace_bytes(int L, int64_t total_channels, size_t* out);
+
+/* ---- a1: importance + Top-K selection (Eq. 6, Table 2, Algorithm 1 "extract the unfrozen
+ * channels") ---------------------------------------------------------------------- */
+/* layers[l].N / .K give the shape of weights[l] (fp32 [N_l, K_l], device); `layers`,
+ * `weights` (array of device pointers) and `k` are HOST arrays of length L.
+ *   CWPL: k[l] channels are kept in layer l (0 <= k[l] <= N_l).
+ *   CWPN: k[0] = channel budget over the whole network; one ranking of all channels by
+ *         importance, ties to the smaller (layer, channel).
+ *   LWPN: k[0] = number of layers kept; layers ranked by mean |w| over the whole layer;
+ *         a kept layer has every channel selected.
+ * Ranking: larger mean |w| first, ties to the smaller index.
+ * Outputs (device): idx int32, concatenated per layer, ascending inside a layer (capacity:
+ * sum of k for CWPL, k[0] for CWPN, total_channels for LWPN); offsets int32 [L+1] with
+ * layer l owning idx[offsets[l] .. offsets[l+1]); importance_or_null fp32 keys
+ * (concatenated channels for CWPL/CWPN, one per layer for LWPN). */
+int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_desc* layers,
+                          const float* const* weights, const int64_t* k, int32_t* idx, int32_t* offsets,
+                          float* importance_or_null, void* ws, size_t ws_bytes, efqat_stream_t stream);
+
+/* ---- a2 + a3: fake-quantize X and W, forward GEMM (Eq. 1, Eq. 3, Section 3.1) -------- */
+/* Y[m,n] = s_x * s_w[n] * sum_k (q_x[m,k] - Z) * q_w[n,k] + bias[n].
+ * s_w [N], s_x [1], z_x [1] (ignored when x_symmetric), bias [N] or NULL; Y in act_dtype. */
+int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
+                        const float* W, const float* s_w, const float* s_x, const float* z_x,
+                        const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream);
+
+/* ---- a4 + a5 + a6 (+ a7): backward (Eq. 5, Algorithm 1, straight-through estimator) --- */
+/* Always: dX = (dY W^) * [x not clipped]  (act_dtype, shape of X), dS_x [1], dZ_x [1],
+ * db_or_null [N] = column sums of dY.
+ * Unfrozen channels only: idx [k_sel] ascending device int32 (may be NULL when k_sel == 0
+ * or k_sel == N); dW_sel fp32 [k_sel, K] with row i <-> channel idx[i];
+ * dS_w_sel fp32 [k_sel].  k_sel == N is the ordinary QAT backward; k_sel == 0 does no
+ * weight-gradient work at all.  dW_sel carries the weight quantizer's clip mask.
+ * opt_or_null != NULL applies the fused SGD-momentum update to rows idx of opt->W_inout. */
+int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
+                        const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
+                        const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,
+                        float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null, void* ws,
+                        size_t ws_bytes, efqat_stream_t stream);
+
+/* ---- helpers: quantizer export and MinMax initialisation ---------------------------- */
+/* Eq. 1: codes int32 [count] (asymmetric: 0..2^b-1; symmetric: signed), clip uint8 [count]
+ * (0 in range, 1 clipped low, 2 clipped high), either may be NULL.  x in `dtype`. */
+int efqat_fake_quant_act(efqat_ctx* ctx, const efqat_qspec* q, int dtype, const void* x, int64_t count,
+                         const float* s_x, const float* z_x, int32_t* codes_or_null, uint8_t* clip_or_null,
+                         efqat_stream_t stream);
+/* Eq. 3: W fp32 [N,K] with per-row scales s_w [N]; codes int32 [N,K], clip uint8 [N,K]. */
+int efqat_fake_quant_weight(efqat_ctx* ctx, const efqat_qspec* q, const float* W, int64_t N, int64_t K,
+                            const float* s_w, int32_t* codes_or_null, uint8_t* clip_or_null,
+                            efqat_stream_t stream);
+/* Eq. 2 (activations, per tensor; symmetric variant when q->x_symmetric) -> s_x[1], z_x[1].
+ * ws: at least 8192 bytes. */
+int efqat_init_act_qparams(efqat_ctx* ctx, const efqat_qspec* q, int dtype, const void* x, int64_t count,
+                           float* s_x, float* z_x, void* ws, size_t ws_bytes, efqat_stream_t stream);
+/* Eq. 4 (weights, per output channel) -> s_w[N]. */
+int efqat_init_weight_scales(efqat_ctx* ctx, const efqat_qspec* q, const float* W, int64_t N, int64_t K,
+                             float* s_w, efqat_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EFQAT_H_ */

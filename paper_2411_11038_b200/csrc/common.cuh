@@ -1,0 +1,98 @@
+// Shared definitions of the CUDA path: the derived quantizer parameters and the
+// per-element quantizer arithmetic (Eq. 1 and Eq. 3 of the paper).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "../../include/efqat.h"
+
+namespace efqat {
+
+// Derived per-tensor activation quantizer parameters, written once per call by
+// prep_act_kernel and read by every kernel that quantizes activations.
+struct ActQ {
+  float s;        // scale
+  float rinv;     // fl32(1/s): the multiplier that decides the integer code
+  float rinv_lo;  // 1/s - rinv in fp32: correction term for the scale gradient
+  float zr;       // rounded, clamped zero point (0 for the symmetric variant)
+  float lo, hi;   // code range [lo, hi]
+  float pad0, pad1;
+};
+
+struct QElem {
+  float c0;   // clamp(c, lo, hi) - zr : the centred integer entering the contractions
+  float t;    // d(dequantised value)/d(scale) under the straight-through estimator
+  int flag;   // 0 in range, 1 clipped low, 2 clipped high
+  int code;   // clamp(c, lo, hi)
+};
+
+__device__ __forceinline__ void record_status(int* status, int code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+// Eq. 1 on one element.  The code is decided by u = fl32(x * fl32(1/s)), rounded to
+// nearest-even; the scale gradient uses x/s to roughly fp64 accuracy through the
+// two-term reciprocal (rne(u) - x*rinv is exact in one fma because rne(u) is within
+// half a unit of the product).
+__device__ __forceinline__ QElem quant_act(float x, const ActQ& p) {
+  QElem e;
+  const float u = __fmul_rn(x, p.rinv);
+  const float r = rintf(u);
+  const float c = r + p.zr;
+  const float q = fminf(fmaxf(c, p.lo), p.hi);
+  e.flag = (c < p.lo) ? 1 : ((c > p.hi) ? 2 : 0);
+  e.c0 = q - p.zr;
+  e.code = static_cast<int>(q);
+  // in range: t = rne(u) - x/s ; clipped: t = c0
+  const float resid = fmaf(-x, p.rinv_lo, fmaf(-x, p.rinv, r));
+  e.t = e.flag ? e.c0 : resid;
+  return e;
+}
+
+struct RowQ {
+  float s, rinv, rinv_lo, qmax;
+};
+
+__device__ __forceinline__ RowQ make_rowq(float s, int w_bits) {
+  RowQ r;
+  r.s = s;
+  const double inv = 1.0 / static_cast<double>(s);
+  r.rinv = static_cast<float>(inv);
+  r.rinv_lo = static_cast<float>(inv - static_cast<double>(r.rinv));
+  r.qmax = static_cast<float>((1 << (w_bits - 1)) - 1);
+  return r;
+}
+
+// Eq. 3 on one element (symmetric, zero point 0, clamp to [-qmax, qmax]).
+__device__ __forceinline__ QElem quant_weight(float w, const RowQ& p) {
+  QElem e;
+  const float u = __fmul_rn(w, p.rinv);
+  const float c = rintf(u);
+  const float q = fminf(fmaxf(c, -p.qmax), p.qmax);
+  e.flag = (c < -p.qmax) ? 1 : ((c > p.qmax) ? 2 : 0);
+  e.c0 = q;
+  e.code = static_cast<int>(q);
+  const float resid = fmaf(-w, p.rinv_lo, fmaf(-w, p.rinv, c));
+  e.t = e.flag ? q : resid;
+  return e;
+}
+
+__device__ __forceinline__ bool scale_ok(float s) { return s > 0.f && isfinite(s); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__host__ __device__ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+__host__ __device__ inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+
+}  // namespace efqat

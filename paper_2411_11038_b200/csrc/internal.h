@@ -1,0 +1,83 @@
+// Host-side launchers shared between the translation units of the library.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace efqat {
+
+typedef __nv_bfloat16 bf16;
+
+// ---- elementwise.cu -----------------------------------------------------------------
+void launch_prep_act(const float* s_x, const float* z_x, int x_bits, int x_sym, ActQ* out, int* status,
+                     cudaStream_t st);
+void launch_quant_act_operand(const void* X, int dtype, int64_t count, const ActQ* q, bf16* out, cudaStream_t st);
+void launch_quant_act_export(const void* X, int dtype, int64_t count, const ActQ* q, int32_t* codes,
+                             uint8_t* clip, cudaStream_t st);
+// mode 0: integer codes q_w as bf16; mode 1: dequantised bf16(fl32(s_w*q_w)).
+void launch_quant_weight_operand(const float* W, int64_t N, int64_t K, const float* s_w, int w_bits, int mode,
+                                 bf16* out, int* status, cudaStream_t st);
+void launch_quant_weight_export(const float* W, int64_t N, int64_t K, const float* s_w, int w_bits,
+                                int32_t* codes, uint8_t* clip, int* status, cudaStream_t st);
+void launch_to_bf16(const float* in, int64_t count, bf16* out, cudaStream_t st);
+void launch_gather_cols(const void* dY, int dtype, int64_t M, int64_t N, const int32_t* idx, int64_t k_sel,
+                        int64_t pitch, bf16* out, int* status, cudaStream_t st);
+// ws: COLSUM_SLABS * N floats
+static const int COLSUM_SLABS = 64;
+void launch_colsum(const void* dY, int dtype, int64_t M, int64_t N, float* ws, float* db, cudaStream_t st);
+void launch_dx_finalize(const float* partials, int n, float* dS_x, float* dZ_x, cudaStream_t st);
+void launch_dw_finalize(const float* P, int splits, int64_t split_stride, int64_t k_sel, int64_t N, int64_t K,
+                        const float* W, const float* s_w, const int32_t* idx_or_null, const ActQ* xq, int w_bits,
+                        float* dW_sel, float* dS_w_sel, const efqat_sgd* opt, int* status, cudaStream_t st);
+void launch_minmax_act(const void* x, int dtype, int64_t count, int x_bits, int x_sym, float* s_x, float* z_x,
+                       float* ws, cudaStream_t st);
+void launch_absmax_rows(const float* W, int64_t N, int64_t K, int w_bits, float* s_w, cudaStream_t st);
+
+// ---- select.cu ----------------------------------------------------------------------
+size_t select_workspace_bytes(int L, int64_t total_channels);
+int run_select(int mode, int L, const efqat_layer_desc* layers, const float* const* weights, const int64_t* k,
+               int32_t* idx, int32_t* offsets, float* importance, void* ws, size_t ws_bytes, int* status,
+               cudaStream_t st);
+
+// ---- gemm.cu ------------------------------------------------------------------------
+enum GemmEpi { EPI_FWD = 0, EPI_DX = 1, EPI_PART = 2 };
+
+struct GemmArgs {
+  // D[Mr, Nc] = A * B over contraction length Kc.
+  // a_mn = 0: A is stored [Mr, Kc] row-major; a_mn = 1: A is stored [Kc, Mr] row-major.
+  // b_mn = 0: B is stored [Nc, Kc] row-major; b_mn = 1: B is stored [Kc, Nc] row-major.
+  const bf16* A;
+  const bf16* B;
+  int64_t Mr, Nc, Kc;
+  int64_t lda, ldb;  // row pitch in elements of the stored matrices
+  int a_mn, b_mn;
+  int epi;
+  int out_bf16;      // EPI_FWD / EPI_DX: output dtype
+  void* out;         // EPI_FWD: Y [Mr,Nc]; EPI_DX: dX [Mr,Nc]; EPI_PART: fp32 partials
+  int64_t ldo;
+  // EPI_FWD
+  const float* col_scale;  // s_w[Nc]
+  const float* col_bias;   // bias[Nc] or null
+  // EPI_FWD / EPI_DX
+  const ActQ* xq;
+  // EPI_DX
+  const void* X;     // raw activations [Mr,Nc] in x_dtype
+  int x_dtype;
+  float* partials;   // [gemm_dx_num_partials][2]
+  // EPI_PART: out[split*split_stride + col*ldo + row], col < part_cols only
+  int splits;
+  int64_t split_stride;
+  int64_t part_cols;
+  int* status;
+};
+// Number of (dS_x, dZ_x) partial pairs EPI_DX writes for this problem.
+int gemm_dx_num_partials(int64_t Mr, int64_t Nc);
+// Split count along the contraction for EPI_PART.
+int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count);
+int gemm_init();  // resolves the tensor-map encoder; returns an efqat_status
+int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st);
+
+}  // namespace efqat

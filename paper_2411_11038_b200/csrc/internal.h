@@ -78,6 +78,7 @@ int gemm_dx_num_partials(int64_t Mr, int64_t Nc);
 // Split count along the contraction for EPI_PART.
 int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count);
 int gemm_init();  // resolves the tensor-map encoder; returns an efqat_status
-int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st);
+// tiles_out (optional): number of output tiles = number of partial pairs EPI_DX wrote.
+int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out = nullptr);
 
 }  // namespace efqat

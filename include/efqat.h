@@ -162,6 +162,15 @@ int efqat_init_act_qparams(efqat_ctx* ctx, const efqat_qspec* q, int dtype, cons
 int efqat_init_weight_scales(efqat_ctx* ctx, const efqat_qspec* q, const float* W, int64_t N, int64_t K,
                              float* s_w, efqat_stream_t stream);
 
+/* ---- helper: the tensor-core contraction shared by a3, a4 and a6 (Eq. 5 shapes) -------- */
+/* out[n*M + m] = sum_k A(m,k) * B(n,k) in fp32, bf16 operands (device), i.e. the product is
+ * written transposed, [N,M] row-major, one slab per split: out has splits*N*M floats and
+ * the caller adds the slabs.  a_mn = 0: A stored [M,K] row-major; a_mn = 1: A stored [K,M].
+ * b_mn = 0: B stored [N,K]; b_mn = 1: B stored [K,N].  M, N, K multiples of 8;
+ * 1 <= splits <= ceil(K/64).  Exposed so the four operand layouts can be tested alone. */
+int efqat_gemm_bf16(efqat_ctx* ctx, const void* A, const void* B, int64_t M, int64_t N, int64_t K, int a_mn,
+                    int b_mn, int splits, float* out, efqat_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

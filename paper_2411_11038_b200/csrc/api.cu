@@ -1,0 +1,419 @@
+// C ABI of the library: argument validation, workspace carving and the launch sequence
+// of each entry point.  Every step of the path runs in this library's kernels; there is
+// no host fallback.
+#include <new>
+
+#include "internal.h"
+
+using namespace efqat;
+
+struct efqat_ctx {
+  int device;
+  int sm_count;
+  int* d_status;
+};
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_bits(const efqat_qspec* q) {
+  if (!q) return EFQAT_ERR_NULL;
+  if (q->w_bits < 2 || q->w_bits > 8 || q->x_bits < 2 || q->x_bits > 8) return EFQAT_ERR_BITS;
+  return EFQAT_OK;
+}
+
+int check_layer(const efqat_layer_desc* l, const efqat_qspec* q) {
+  if (!l) return EFQAT_ERR_NULL;
+  int rc = check_bits(q);
+  if (rc != EFQAT_OK) return rc;
+  if (l->act_dtype != EFQAT_F32 && l->act_dtype != EFQAT_BF16) return EFQAT_ERR_DTYPE;
+  if (l->M < 1 || l->N < 1 || l->K < 1) return EFQAT_ERR_SHAPE;
+  if (l->M > INT32_MAX || l->N > INT32_MAX || l->K > INT32_MAX) return EFQAT_ERR_SHAPE;
+  if ((l->N & 7) || (l->K & 7)) return EFQAT_ERR_ALIGN;
+  if (l->is_conv) {
+    if (l->B < 1 || l->H < 1 || l->W < 1 || l->Cin < 1 || l->R < 1 || l->S < 1) return EFQAT_ERR_SHAPE;
+    if (l->stride != 1) return EFQAT_ERR_UNIMPL;
+    if (l->pad < 0 || l->pad >= l->R || l->pad >= l->S) return EFQAT_ERR_SHAPE;
+    if (l->Cin & 7) return EFQAT_ERR_ALIGN;
+    const int64_t Ho = l->H + 2 * l->pad - l->R + 1, Wo = l->W + 2 * l->pad - l->S + 1;
+    if (Ho < 1 || Wo < 1) return EFQAT_ERR_SHAPE;
+    if (l->M != static_cast<int64_t>(l->B) * Ho * Wo) return EFQAT_ERR_SHAPE;
+    if (l->K != static_cast<int64_t>(l->R) * l->S * l->Cin) return EFQAT_ERR_SHAPE;
+    if (l->R != 1 || l->S != 1 || l->pad != 0) return EFQAT_ERR_UNIMPL;   // 1x1 convolutions only so far
+  }
+  return EFQAT_OK;
+}
+
+// Workspace sections of the forward / backward calls.
+struct LayerWs {
+  ActQ* actq;
+  bf16* Xc;        // [M,K] centred activation codes
+  bf16* Wq;        // [N,K] weight codes (forward) or dequantised weights (backward)
+  bf16* dYb;       // [M,N] bf16 copy of an fp32 dY
+  bf16* dYsel;     // [M,pitch] gathered selected columns of dY
+  float* P;        // [splits][k_sel][K] partial weight-gradient products
+  float* dxpart;   // [tiles][2]
+  float* colsum;   // [COLSUM_SLABS][N]
+  int64_t pitch;
+  int splits;
+  size_t bytes;
+};
+
+int64_t sel_pitch(int64_t k_sel) { return round_up(k_sel, 64); }
+
+LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, int64_t p_elems_override) {
+  LayerWs w = {};
+  char* base = ws ? reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~uintptr_t(255)) : nullptr;
+  size_t off = 0;
+  auto take = [&](int64_t bytes) {
+    char* r = base ? base + off : nullptr;
+    off += static_cast<size_t>(round_up(bytes, 256));
+    return r;
+  };
+  const int64_t M = l->M, N = l->N, K = l->K;
+  w.actq = reinterpret_cast<ActQ*>(take(sizeof(ActQ)));
+  w.Xc = reinterpret_cast<bf16*>(take(M * K * 2));
+  w.Wq = reinterpret_cast<bf16*>(take(N * K * 2));
+  w.dYb = reinterpret_cast<bf16*>(take(l->act_dtype == EFQAT_F32 ? M * N * 2 : 0));
+  const bool gathered = k_sel > 0 && k_sel < N;
+  w.pitch = gathered ? sel_pitch(k_sel) : N;
+  w.dYsel = reinterpret_cast<bf16*>(take(gathered ? M * w.pitch * 2 : 0));
+  w.splits = k_sel > 0 ? gemm_choose_splits(K, gathered ? round_up(k_sel, 16) : N, M, sm_count) : 1;
+  const int64_t p_elems = p_elems_override >= 0 ? p_elems_override : static_cast<int64_t>(w.splits) * k_sel * K;
+  w.P = reinterpret_cast<float*>(take(p_elems * 4));
+  w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(gemm_dx_num_partials(M, K)) * 8));
+  w.colsum = reinterpret_cast<float*>(take(static_cast<int64_t>(COLSUM_SLABS) * N * 4));
+  w.bytes = off + 256;
+  return w;
+}
+
+int guard_device(const efqat_ctx* ctx) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device) return EFQAT_ERR_CUDA;
+  return EFQAT_OK;
+}
+
+int last_error() { return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int efqat_create(efqat_ctx** out, int device) {
+  if (!out) return EFQAT_ERR_NULL;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return EFQAT_ERR_CUDA;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  if (cudaSetDevice(device) != cudaSuccess) return EFQAT_ERR_CUDA;
+  efqat_ctx* c = new (std::nothrow) efqat_ctx();
+  if (!c) return EFQAT_ERR_CUDA;
+  c->device = device;
+  int rc = EFQAT_OK;
+  if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+      cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMemset(c->d_status, 0, 256) != cudaSuccess)
+    rc = EFQAT_ERR_CUDA;
+  if (rc == EFQAT_OK) rc = gemm_init();
+  cudaSetDevice(prev);
+  if (rc != EFQAT_OK) {
+    delete c;
+    return rc;
+  }
+  *out = c;
+  return EFQAT_OK;
+}
+
+int efqat_destroy(efqat_ctx* ctx) {
+  if (!ctx) return EFQAT_ERR_NULL;
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+  return EFQAT_OK;
+}
+
+const char* efqat_status_string(int s) {
+  switch (s) {
+    case EFQAT_OK: return "ok";
+    case EFQAT_ERR_NULL: return "required pointer is NULL";
+    case EFQAT_ERR_SHAPE: return "invalid or inconsistent shape";
+    case EFQAT_ERR_ALIGN: return "alignment contract violated";
+    case EFQAT_ERR_DTYPE: return "unknown dtype";
+    case EFQAT_ERR_BITS: return "bit-width outside [2,8]";
+    case EFQAT_ERR_MODE: return "unknown selection mode";
+    case EFQAT_ERR_WORKSPACE: return "workspace missing or too small";
+    case EFQAT_ERR_K_RANGE: return "selection count out of range";
+    case EFQAT_ERR_UNIMPL: return "combination not implemented";
+    case EFQAT_ERR_CUDA: return "CUDA call failed";
+    case EFQAT_DEV_BAD_SCALE: return "device: scale not positive and finite";
+    case EFQAT_DEV_BAD_INDEX: return "device: channel index out of range or not ascending";
+    case EFQAT_DEV_WAIT_TIMEOUT: return "device: bounded wait expired";
+    default: return "unknown status";
+  }
+}
+
+int efqat_device_status(efqat_ctx* ctx, int* code) {
+  if (!ctx || !code) return EFQAT_ERR_NULL;
+  if (cudaDeviceSynchronize() != cudaSuccess) return EFQAT_ERR_CUDA;
+  if (cudaMemcpy(code, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EFQAT_ERR_CUDA;
+  if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) return EFQAT_ERR_CUDA;
+  return EFQAT_OK;
+}
+
+int64_t efqat_ratio_to_k(double ratio, int64_t n) {
+  if (!(ratio > 0.0) || n <= 0) return 0;
+  if (ratio >= 1.0) return n;
+  return static_cast<int64_t>(floor(ratio * static_cast<double>(n)));
+}
+
+int efqat_validate_layer(const efqat_layer_desc* layer, const efqat_qspec* q) { return check_layer(layer, q); }
+
+int efqat_workspace_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, int64_t k_sel_max, size_t* out) {
+  if (!out) return EFQAT_ERR_NULL;
+  int rc = check_layer(layer, q);
+  if (rc != EFQAT_OK) return rc;
+  if (k_sel_max < 0 || k_sel_max > layer->N) return EFQAT_ERR_K_RANGE;
+  // the partial-product buffer is the only section that is not monotone in k_sel
+  // (fewer channels -> more splits of the contraction); take its maximum.  148 SMs
+  // is assumed when no context is at hand; a larger part would only lower the split count.
+  const int sm = 148;
+  int64_t p_max = 0;
+  for (int64_t k = 1; k <= k_sel_max; ++k) {
+    const int64_t nc = (k < layer->N) ? round_up(k, 16) : layer->N;
+    const int64_t e = static_cast<int64_t>(gemm_choose_splits(layer->K, nc, layer->M, sm)) * k * layer->K;
+    if (e > p_max) p_max = e;
+  }
+  // dYsel is largest for the largest gathered k
+  const int64_t k_g = (k_sel_max == layer->N && layer->N > 1) ? layer->N - 1 : k_sel_max;
+  *out = carve(nullptr, layer, k_g, sm, p_max).bytes;
+  return EFQAT_OK;
+}
+
+int efqat_select_workspace_bytes(int L, int64_t total_channels, size_t* out) {
+  if (!out) return EFQAT_ERR_NULL;
+  if (L < 1 || total_channels < 1) return EFQAT_ERR_SHAPE;
+  *out = select_workspace_bytes(L, total_channels) + 256;
+  return EFQAT_OK;
+}
+
+int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_desc* layers,
+                          const float* const* weights, const int64_t* k, int32_t* idx, int32_t* offsets,
+                          float* importance_or_null, void* ws, size_t ws_bytes, efqat_stream_t stream) {
+  if (!ctx || !layers || !weights || !k || !offsets) return EFQAT_ERR_NULL;
+  if (L < 1) return EFQAT_ERR_SHAPE;
+  if (mode != EFQAT_CWPL && mode != EFQAT_CWPN && mode != EFQAT_LWPN) return EFQAT_ERR_MODE;
+  if (!ws) return EFQAT_ERR_WORKSPACE;
+  int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  void* base = reinterpret_cast<void*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~uintptr_t(255));
+  const size_t slack = static_cast<size_t>(reinterpret_cast<char*>(base) - reinterpret_cast<char*>(ws));
+  if (ws_bytes < slack) return EFQAT_ERR_WORKSPACE;
+  if (!idx) {
+    // idx may only be NULL when nothing can be selected
+    int64_t want = 0;
+    for (int l = 0; l < (mode == EFQAT_CWPL ? L : 1); ++l) want += k[l];
+    if (want > 0) return EFQAT_ERR_NULL;
+  }
+  return run_select(mode, L, layers, weights, k, idx, offsets, importance_or_null, base, ws_bytes - slack,
+                    ctx->d_status, stream);
+}
+
+int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
+                        const float* W, const float* s_w, const float* s_x, const float* z_x,
+                        const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream) {
+  if (!ctx || !X || !W || !s_w || !s_x || !Y) return EFQAT_ERR_NULL;
+  int rc = check_layer(layer, q);
+  if (rc != EFQAT_OK) return rc;
+  if (!q->x_symmetric && !z_x) return EFQAT_ERR_NULL;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y)) return EFQAT_ERR_ALIGN;
+  if (!ws) return EFQAT_ERR_WORKSPACE;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  const LayerWs w = carve(ws, layer, 0, ctx->sm_count, 0);
+  if (ws_bytes < w.bytes) return EFQAT_ERR_WORKSPACE;
+  const int64_t M = layer->M, N = layer->N, K = layer->K;
+  cudaStream_t st = stream;
+
+  launch_prep_act(s_x, z_x, q->x_bits, q->x_symmetric, w.actq, ctx->d_status, st);
+  launch_quant_act_operand(X, layer->act_dtype, M * K, w.actq, w.Xc, st);
+  launch_quant_weight_operand(W, N, K, s_w, q->w_bits, 0, w.Wq, ctx->d_status, st);
+  GemmArgs g = {};
+  g.A = w.Xc; g.B = w.Wq;
+  g.Mr = M; g.Nc = N; g.Kc = K;
+  g.lda = K; g.ldb = K;
+  g.a_mn = 0; g.b_mn = 0;
+  g.epi = EPI_FWD;
+  g.out_bf16 = layer->act_dtype == EFQAT_BF16;
+  g.out = Y; g.ldo = N;
+  g.col_scale = s_w; g.col_bias = bias_or_null;
+  g.xq = w.actq;
+  g.status = ctx->d_status;
+  rc = run_gemm(g, ctx->sm_count, st);
+  if (rc != EFQAT_OK) return rc;
+  return last_error();
+}
+
+int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
+                        const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
+                        const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,
+                        float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null, void* ws,
+                        size_t ws_bytes, efqat_stream_t stream) {
+  if (!ctx || !dY || !X || !W || !s_w || !s_x || !dX || !dS_x || !dZ_x) return EFQAT_ERR_NULL;
+  int rc = check_layer(layer, q);
+  if (rc != EFQAT_OK) return rc;
+  if (!q->x_symmetric && !z_x) return EFQAT_ERR_NULL;
+  const int64_t M = layer->M, N = layer->N, K = layer->K;
+  if (k_sel < 0 || k_sel > N) return EFQAT_ERR_K_RANGE;
+  if (k_sel > 0 && (!dW_sel || !dS_w_sel)) return EFQAT_ERR_NULL;
+  if (k_sel > 0 && k_sel < N && !idx) return EFQAT_ERR_NULL;
+  if (opt_or_null && k_sel > 0 && (!opt_or_null->W_inout || !opt_or_null->mom_inout)) return EFQAT_ERR_NULL;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(dX) || (dW_sel && !aligned16(dW_sel)))
+    return EFQAT_ERR_ALIGN;
+  if (!ws) return EFQAT_ERR_WORKSPACE;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  const LayerWs w = carve(ws, layer, k_sel, ctx->sm_count, -1);
+  if (ws_bytes < w.bytes) return EFQAT_ERR_WORKSPACE;
+  cudaStream_t st = stream;
+  const int act_bf16 = layer->act_dtype == EFQAT_BF16;
+
+  // a2: quantizer parameters, dequantised weight operand, bf16 view of dY
+  launch_prep_act(s_x, z_x, q->x_bits, q->x_symmetric, w.actq, ctx->d_status, st);
+  launch_quant_weight_operand(W, N, K, s_w, q->w_bits, 1, w.Wq, ctx->d_status, st);
+  const bf16* dYb = static_cast<const bf16*>(dY);
+  if (!act_bf16) {
+    launch_to_bf16(static_cast<const float*>(dY), M * N, w.dYb, st);
+    dYb = w.dYb;
+  }
+  // a4 + a5: dX = (dY W^) masked, with the dS_x / dZ_x partial sums in the epilogue
+  {
+    GemmArgs g = {};
+    g.A = dYb; g.B = w.Wq;
+    g.Mr = M; g.Nc = K; g.Kc = N;
+    g.lda = N; g.ldb = K;
+    g.a_mn = 0; g.b_mn = 1;
+    g.epi = EPI_DX;
+    g.out_bf16 = act_bf16;
+    g.out = dX; g.ldo = K;
+    g.xq = w.actq;
+    g.X = X; g.x_dtype = layer->act_dtype;
+    g.partials = w.dxpart;
+    g.status = ctx->d_status;
+    int tiles = 0;
+    rc = run_gemm(g, ctx->sm_count, st, &tiles);
+    if (rc != EFQAT_OK) return rc;
+    launch_dx_finalize(w.dxpart, tiles, dS_x, dZ_x, st);
+  }
+  if (db_or_null) launch_colsum(dY, layer->act_dtype, M, N, w.colsum, db_or_null, st);
+  // a6 (+ a7): weight gradient of the unfrozen channels only
+  if (k_sel > 0) {
+    launch_quant_act_operand(X, layer->act_dtype, M * K, w.actq, w.Xc, st);
+    const bool gathered = k_sel < N;
+    const bf16* Bop = dYb;
+    int64_t ldb = N, nc = N;
+    if (gathered) {
+      launch_gather_cols(dY, layer->act_dtype, M, N, idx, k_sel, w.pitch, w.dYsel, ctx->d_status, st);
+      Bop = w.dYsel;
+      ldb = w.pitch;
+      nc = round_up(k_sel, 16);
+    }
+    GemmArgs g = {};
+    g.A = w.Xc; g.B = Bop;           // D[k, i] = sum_m Xc[m,k] * dYsel[m,i]
+    g.Mr = K; g.Nc = nc; g.Kc = M;
+    g.lda = K; g.ldb = ldb;
+    g.a_mn = 1; g.b_mn = 1;
+    g.epi = EPI_PART;
+    g.out = w.P; g.ldo = K;
+    g.splits = w.splits;
+    g.split_stride = k_sel * K;
+    g.part_cols = k_sel;
+    g.status = ctx->d_status;
+    rc = run_gemm(g, ctx->sm_count, st);
+    if (rc != EFQAT_OK) return rc;
+    launch_dw_finalize(w.P, w.splits, k_sel * K, k_sel, N, K, W, s_w, gathered ? idx : nullptr, w.actq,
+                       q->w_bits, dW_sel, dS_w_sel, opt_or_null, ctx->d_status, st);
+  }
+  return last_error();
+}
+
+int efqat_gemm_bf16(efqat_ctx* ctx, const void* A, const void* B, int64_t M, int64_t N, int64_t K, int a_mn,
+                    int b_mn, int splits, float* out, efqat_stream_t stream) {
+  if (!ctx || !A || !B || !out) return EFQAT_ERR_NULL;
+  if (M < 1 || N < 1 || K < 1 || splits < 1) return EFQAT_ERR_SHAPE;
+  if ((M & 7) || (N & 7) || (K & 7)) return EFQAT_ERR_ALIGN;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(out)) return EFQAT_ERR_ALIGN;
+  int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  GemmArgs g = {};
+  g.A = static_cast<const bf16*>(A); g.B = static_cast<const bf16*>(B);
+  g.Mr = M; g.Nc = N; g.Kc = K;
+  g.lda = a_mn ? M : K; g.ldb = b_mn ? N : K;
+  g.a_mn = a_mn ? 1 : 0; g.b_mn = b_mn ? 1 : 0;
+  g.epi = EPI_PART;
+  g.out = out; g.ldo = M;
+  g.splits = splits;
+  g.split_stride = M * N;
+  g.part_cols = N;
+  g.status = ctx->d_status;
+  rc = run_gemm(g, ctx->sm_count, stream);
+  if (rc != EFQAT_OK) return rc;
+  return last_error();
+}
+
+int efqat_fake_quant_act(efqat_ctx* ctx, const efqat_qspec* q, int dtype, const void* x, int64_t count,
+                         const float* s_x, const float* z_x, int32_t* codes_or_null, uint8_t* clip_or_null,
+                         efqat_stream_t stream) {
+  if (!ctx || !x || !s_x) return EFQAT_ERR_NULL;
+  int rc = check_bits(q);
+  if (rc != EFQAT_OK) return rc;
+  if (!q->x_symmetric && !z_x) return EFQAT_ERR_NULL;
+  if (dtype != EFQAT_F32 && dtype != EFQAT_BF16) return EFQAT_ERR_DTYPE;
+  if (count < 0) return EFQAT_ERR_SHAPE;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  ActQ* scratch = reinterpret_cast<ActQ*>(reinterpret_cast<char*>(ctx->d_status) + 128);
+  launch_prep_act(s_x, z_x, q->x_bits, q->x_symmetric, scratch, ctx->d_status, stream);
+  launch_quant_act_export(x, dtype, count, scratch, codes_or_null, clip_or_null, stream);
+  return last_error();
+}
+
+int efqat_fake_quant_weight(efqat_ctx* ctx, const efqat_qspec* q, const float* W, int64_t N, int64_t K,
+                            const float* s_w, int32_t* codes_or_null, uint8_t* clip_or_null,
+                            efqat_stream_t stream) {
+  if (!ctx || !W || !s_w) return EFQAT_ERR_NULL;
+  int rc = check_bits(q);
+  if (rc != EFQAT_OK) return rc;
+  if (N < 0 || K < 1) return EFQAT_ERR_SHAPE;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  launch_quant_weight_export(W, N, K, s_w, q->w_bits, codes_or_null, clip_or_null, ctx->d_status, stream);
+  return last_error();
+}
+
+int efqat_init_act_qparams(efqat_ctx* ctx, const efqat_qspec* q, int dtype, const void* x, int64_t count,
+                           float* s_x, float* z_x, void* ws, size_t ws_bytes, efqat_stream_t stream) {
+  if (!ctx || !x || !s_x || !z_x) return EFQAT_ERR_NULL;
+  int rc = check_bits(q);
+  if (rc != EFQAT_OK) return rc;
+  if (dtype != EFQAT_F32 && dtype != EFQAT_BF16) return EFQAT_ERR_DTYPE;
+  if (count < 1) return EFQAT_ERR_SHAPE;
+  if (!ws || ws_bytes < 8192) return EFQAT_ERR_WORKSPACE;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  launch_minmax_act(x, dtype, count, q->x_bits, q->x_symmetric, s_x, z_x, static_cast<float*>(ws), stream);
+  return last_error();
+}
+
+int efqat_init_weight_scales(efqat_ctx* ctx, const efqat_qspec* q, const float* W, int64_t N, int64_t K,
+                             float* s_w, efqat_stream_t stream) {
+  if (!ctx || !W || !s_w) return EFQAT_ERR_NULL;
+  int rc = check_bits(q);
+  if (rc != EFQAT_OK) return rc;
+  if (N < 1 || K < 1) return EFQAT_ERR_SHAPE;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  launch_absmax_rows(W, N, K, q->w_bits, s_w, stream);
+  return last_error();
+}
+
+}  // extern "C"

@@ -1,0 +1,383 @@
+"""ctypes binding of libefqat.so: argument marshalling only.
+
+Function names mirror include/efqat.h.  Tensors are torch CUDA tensors used purely as
+device memory; every computation happens inside the library's kernels.  Importing this
+module does not load the library; the first call does, and fails loudly if the shared
+object has not been built (python -m paper_2411_11038_b200.build).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libefqat.so")
+
+CWPL, CWPN, LWPN = 0, 1, 2
+F32, BF16 = 0, 1
+
+EXPORTS = [
+    "efqat_create", "efqat_destroy", "efqat_status_string", "efqat_device_status",
+    "efqat_ratio_to_k", "efqat_validate_layer", "efqat_workspace_bytes",
+    "efqat_select_workspace_bytes", "efqat_select_channels", "efqat_fq_linear_fwd",
+    "efqat_fq_linear_bwd", "efqat_fake_quant_act", "efqat_fake_quant_weight",
+    "efqat_init_act_qparams", "efqat_init_weight_scales", "efqat_gemm_bf16",
+]
+
+
+class QSpec(C.Structure):
+    _fields_ = [("w_bits", C.c_int), ("x_bits", C.c_int), ("x_symmetric", C.c_int)]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64), ("is_conv", C.c_int),
+                ("B", C.c_int), ("H", C.c_int), ("W", C.c_int), ("Cin", C.c_int), ("R", C.c_int),
+                ("S", C.c_int), ("stride", C.c_int), ("pad", C.c_int), ("act_dtype", C.c_int)]
+
+
+class Sgd(C.Structure):
+    _fields_ = [("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
+                ("W_inout", C.c_void_p), ("mom_inout", C.c_void_p)]
+
+
+class EfqatError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: efqat status {code} ({status_string(code)})")
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Loads libefqat.so once.  No fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2411_11038_b200.build`")
+    lib = C.CDLL(LIB_PATH)
+    vp, i64, i32, sz = C.c_void_p, C.c_int64, C.c_int, C.c_size_t
+    lib.efqat_create.argtypes = [C.POINTER(vp), i32]
+    lib.efqat_destroy.argtypes = [vp]
+    lib.efqat_status_string.argtypes = [i32]
+    lib.efqat_status_string.restype = C.c_char_p
+    lib.efqat_device_status.argtypes = [vp, C.POINTER(i32)]
+    lib.efqat_ratio_to_k.argtypes = [C.c_double, i64]
+    lib.efqat_ratio_to_k.restype = i64
+    lib.efqat_validate_layer.argtypes = [C.POINTER(LayerDesc), C.POINTER(QSpec)]
+    lib.efqat_workspace_bytes.argtypes = [C.POINTER(LayerDesc), C.POINTER(QSpec), i64, C.POINTER(sz)]
+    lib.efqat_select_workspace_bytes.argtypes = [i32, i64, C.POINTER(sz)]
+    lib.efqat_select_channels.argtypes = [vp, i32, i32, C.POINTER(LayerDesc), C.POINTER(vp), C.POINTER(i64),
+                                          vp, vp, vp, vp, sz, vp]
+    lib.efqat_fq_linear_fwd.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(QSpec), vp, vp, vp, vp, vp, vp, vp,
+                                        vp, sz, vp]
+    lib.efqat_fq_linear_bwd.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(QSpec), vp, vp, vp, vp, vp, vp,
+                                        vp, i64, vp, vp, vp, vp, vp, vp, C.POINTER(Sgd), vp, sz, vp]
+    lib.efqat_fake_quant_act.argtypes = [vp, C.POINTER(QSpec), i32, vp, i64, vp, vp, vp, vp, vp]
+    lib.efqat_fake_quant_weight.argtypes = [vp, C.POINTER(QSpec), vp, i64, i64, vp, vp, vp, vp]
+    lib.efqat_init_act_qparams.argtypes = [vp, C.POINTER(QSpec), i32, vp, i64, vp, vp, vp, sz, vp]
+    lib.efqat_init_weight_scales.argtypes = [vp, C.POINTER(QSpec), vp, i64, i64, vp, vp]
+    lib.efqat_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp]
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if name not in ("efqat_status_string", "efqat_ratio_to_k"):
+            fn.restype = i32
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().efqat_status_string(int(code)).decode()
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise EfqatError(rc, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"activations must be fp32 or bf16, got {t.dtype}")
+
+
+def _dev(t: torch.Tensor) -> torch.Tensor:
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t
+
+
+class Context:
+    """efqat_create / efqat_destroy."""
+
+    def __init__(self, device: int = 0):
+        lib = load()
+        h = C.c_void_p()
+        torch.cuda.set_device(device)
+        _check(lib.efqat_create(C.byref(h), int(device)), "efqat_create")
+        self.handle = h
+        self.device = device
+
+    def device_status(self) -> int:
+        code = C.c_int(0)
+        _check(load().efqat_device_status(self.handle, C.byref(code)), "efqat_device_status")
+        return code.value
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().efqat_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+@dataclass
+class ConvGeom:
+    B: int
+    H: int
+    W: int
+    Cin: int
+    R: int
+    S: int
+    stride: int = 1
+    pad: int = 0
+
+
+def layer_desc(M: int, N: int, K: int, act_dtype: int, conv: Optional[ConvGeom] = None) -> LayerDesc:
+    d = LayerDesc(M=M, N=N, K=K, is_conv=0, B=1, H=1, W=1, Cin=K, R=1, S=1, stride=1, pad=0,
+                  act_dtype=act_dtype)
+    if conv is not None:
+        d.is_conv = 1
+        d.B, d.H, d.W, d.Cin, d.R, d.S, d.stride, d.pad = (conv.B, conv.H, conv.W, conv.Cin, conv.R, conv.S,
+                                                         conv.stride, conv.pad)
+    return d
+
+
+def ratio_to_k(ratio: float, n: int) -> int:
+    return int(load().efqat_ratio_to_k(float(ratio), int(n)))
+
+
+def validate_layer(desc: LayerDesc, spec: QSpec) -> int:
+    return int(load().efqat_validate_layer(C.byref(desc), C.byref(spec)))
+
+
+def workspace_bytes(desc: LayerDesc, spec: QSpec, k_sel_max: int) -> int:
+    out = C.c_size_t(0)
+    _check(load().efqat_workspace_bytes(C.byref(desc), C.byref(spec), int(k_sel_max), C.byref(out)),
+           "efqat_workspace_bytes")
+    return out.value
+
+
+def select_workspace_bytes(L: int, total_channels: int) -> int:
+    out = C.c_size_t(0)
+    _check(load().efqat_select_workspace_bytes(int(L), int(total_channels), C.byref(out)),
+           "efqat_select_workspace_bytes")
+    return out.value
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ---------------------------------------------------------------------------------------
+class SelectPlan:
+    """Pre-marshalled arguments of efqat_select_channels for a fixed set of layers."""
+
+    def __init__(self, ctx: Context, mode: int, weights: Sequence[torch.Tensor], k: Sequence[int],
+                 want_importance: bool = False):
+        self.ctx, self.mode = ctx, mode
+        self.weights = [_dev(w) for w in weights]
+        L = len(weights)
+        self.L = L
+        self.N = [int(w.shape[0]) for w in weights]
+        self.K = [int(w.numel() // w.shape[0]) for w in weights]
+        self.total = sum(self.N)
+        dev = weights[0].device
+        self.descs = (LayerDesc * L)(*[layer_desc(1, n, kk, F32) for n, kk in zip(self.N, self.K)])
+        self.wptrs = (C.c_void_p * L)(*[w.data_ptr() for w in self.weights])
+        self.k = (C.c_int64 * max(L, 1))(*[int(v) for v in k])
+        cap = {CWPL: sum(int(v) for v in k[:L]), CWPN: int(k[0]), LWPN: self.total}[mode]
+        self.idx = torch.empty(max(cap, 1), dtype=torch.int32, device=dev)
+        self.offsets = torch.empty(L + 1, dtype=torch.int32, device=dev)
+        n_imp = L if mode == LWPN else self.total
+        self.importance = torch.empty(n_imp, dtype=torch.float32, device=dev) if want_importance else None
+        self.ws = alloc_workspace(select_workspace_bytes(L, self.total), dev)
+
+    def run(self):
+        rc = load().efqat_select_channels(self.ctx.handle, self.mode, self.L, self.descs, self.wptrs, self.k,
+                                          _ptr(self.idx), _ptr(self.offsets), _ptr(self.importance),
+                                          _ptr(self.ws), self.ws.numel(), _stream())
+        _check(rc, "efqat_select_channels")
+        return self.idx, self.offsets, self.importance
+
+
+def select_channels(ctx: Context, mode: int, weights: Sequence[torch.Tensor], k: Sequence[int],
+                    want_importance: bool = False):
+    """Returns (list of per-layer int32 index tensors, offsets tensor, importance or None)."""
+    plan = SelectPlan(ctx, mode, weights, k, want_importance)
+    idx, offsets, imp = plan.run()
+    off = offsets.cpu().tolist()
+    per_layer = [idx[off[l]:off[l + 1]] for l in range(plan.L)]
+    return per_layer, offsets, imp
+
+
+# ---------------------------------------------------------------------------------------
+class LayerPlan:
+    """Pre-marshalled forward / backward calls of one layer: descriptor, quantizer spec,
+    workspace and output tensors allocated once, so a step is only the two C calls."""
+
+    def __init__(self, ctx: Context, M: int, N: int, K: int, act_dtype: torch.dtype, w_bits: int, x_bits: int,
+                 x_symmetric: bool, k_sel_max: int, device, conv: Optional[ConvGeom] = None,
+                 x_shape=None, y_shape=None):
+        self.ctx = ctx
+        self.M, self.N, self.K = M, N, K
+        self.act_dtype = act_dtype
+        code = F32 if act_dtype == torch.float32 else BF16
+        self.desc = layer_desc(M, N, K, code, conv)
+        self.spec = QSpec(w_bits, x_bits, 1 if x_symmetric else 0)
+        self.k_sel_max = k_sel_max
+        self.ws = alloc_workspace(workspace_bytes(self.desc, self.spec, k_sel_max), device)
+        xs = tuple(x_shape) if x_shape is not None else (M, K)
+        ys = tuple(y_shape) if y_shape is not None else (M, N)
+        self.Y = torch.empty(ys, dtype=act_dtype, device=device)
+        self.dX = torch.empty(xs, dtype=act_dtype, device=device)
+        self.dW_sel = torch.empty((max(k_sel_max, 1), K), dtype=torch.float32, device=device)
+        self.dS_w_sel = torch.empty(max(k_sel_max, 1), dtype=torch.float32, device=device)
+        self.dS_x = torch.empty(1, dtype=torch.float32, device=device)
+        self.dZ_x = torch.empty(1, dtype=torch.float32, device=device)
+        self.db = torch.empty(N, dtype=torch.float32, device=device)
+
+    def fwd(self, X, W, s_w, s_x, z_x, bias=None):
+        rc = load().efqat_fq_linear_fwd(self.ctx.handle, C.byref(self.desc), C.byref(self.spec), _ptr(X), _ptr(W),
+                                        _ptr(s_w), _ptr(s_x), _ptr(z_x), _ptr(bias), _ptr(self.Y), _ptr(self.ws),
+                                        self.ws.numel(), _stream())
+        _check(rc, "efqat_fq_linear_fwd")
+        return self.Y
+
+    def bwd(self, dY, X, W, s_w, s_x, z_x, idx, k_sel: int, want_db: bool = True, sgd: Optional[Sgd] = None):
+        rc = load().efqat_fq_linear_bwd(self.ctx.handle, C.byref(self.desc), C.byref(self.spec), _ptr(dY), _ptr(X),
+                                        _ptr(W), _ptr(s_w), _ptr(s_x), _ptr(z_x), _ptr(idx), int(k_sel),
+                                        _ptr(self.dX), _ptr(self.dW_sel), _ptr(self.dS_w_sel), _ptr(self.dS_x),
+                                        _ptr(self.dZ_x), _ptr(self.db) if want_db else None,
+                                        C.byref(sgd) if sgd is not None else None, _ptr(self.ws),
+                                        self.ws.numel(), _stream())
+        _check(rc, "efqat_fq_linear_bwd")
+        return dict(dX=self.dX, dW_sel=self.dW_sel[:k_sel], dS_w_sel=self.dS_w_sel[:k_sel], dS_x=self.dS_x,
+                    dZ_x=self.dZ_x, db=self.db if want_db else None)
+
+
+def _plan_for(ctx, X, W, w_bits, x_bits, x_symmetric, k_sel_max, conv):
+    N = int(W.shape[0])
+    K = int(W.numel() // N)
+    if conv is not None:
+        Ho = conv.H + 2 * conv.pad - conv.R + 1
+        Wo = conv.W + 2 * conv.pad - conv.S + 1
+        M = conv.B * Ho * Wo
+        return LayerPlan(ctx, M, N, K, X.dtype, w_bits, x_bits, x_symmetric, k_sel_max, X.device, conv,
+                         x_shape=X.shape, y_shape=(conv.B, Ho, Wo, N))
+    M = int(X.shape[0])
+    return LayerPlan(ctx, M, N, K, X.dtype, w_bits, x_bits, x_symmetric, k_sel_max, X.device)
+
+
+def fq_linear_fwd(ctx: Context, X, W, s_w, s_x, z_x, bias=None, w_bits=8, x_bits=8, x_symmetric=False,
+                  conv: Optional[ConvGeom] = None):
+    """efqat_fq_linear_fwd: returns Y (new tensor)."""
+    for t in (X, W, s_w, s_x):
+        _dev(t)
+    plan = _plan_for(ctx, X, W, w_bits, x_bits, x_symmetric, 0, conv)
+    return plan.fwd(X, W, s_w, s_x, z_x, bias)
+
+
+def fq_linear_bwd(ctx: Context, dY, X, W, s_w, s_x, z_x, idx, k_sel: int, w_bits=8, x_bits=8,
+                  x_symmetric=False, want_db=True, sgd: Optional[Sgd] = None, conv: Optional[ConvGeom] = None):
+    """efqat_fq_linear_bwd: returns dict(dX, dW_sel, dS_w_sel, dS_x, dZ_x, db)."""
+    for t in (dY, X, W, s_w, s_x):
+        _dev(t)
+    plan = _plan_for(ctx, X, W, w_bits, x_bits, x_symmetric, int(k_sel), conv)
+    return plan.bwd(dY, X, W, s_w, s_x, z_x, idx, int(k_sel), want_db, sgd)
+
+
+def make_sgd(lr: float, momentum: float, weight_decay: float, W: torch.Tensor, mom: torch.Tensor) -> Sgd:
+    return Sgd(lr, momentum, weight_decay, W.data_ptr(), mom.data_ptr())
+
+
+# ---------------------------------------------------------------------------------------
+def fake_quant_act(ctx: Context, x, s_x, z_x, x_bits=8, x_symmetric=False):
+    """efqat_fake_quant_act: returns (codes int32, clip uint8) shaped like x."""
+    _dev(x)
+    spec = QSpec(8, x_bits, 1 if x_symmetric else 0)
+    codes = torch.empty(x.shape, dtype=torch.int32, device=x.device)
+    clip = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    rc = load().efqat_fake_quant_act(ctx.handle, C.byref(spec), _dtype_code(x), _ptr(x), x.numel(), _ptr(s_x),
+                                     _ptr(z_x), _ptr(codes), _ptr(clip), _stream())
+    _check(rc, "efqat_fake_quant_act")
+    return codes, clip
+
+
+def fake_quant_weight(ctx: Context, W, s_w, w_bits=8):
+    """efqat_fake_quant_weight: returns (codes int32, clip uint8) shaped like W."""
+    _dev(W)
+    spec = QSpec(w_bits, 8, 0)
+    N = int(W.shape[0])
+    K = int(W.numel() // N)
+    codes = torch.empty(W.shape, dtype=torch.int32, device=W.device)
+    clip = torch.empty(W.shape, dtype=torch.uint8, device=W.device)
+    rc = load().efqat_fake_quant_weight(ctx.handle, C.byref(spec), _ptr(W), N, K, _ptr(s_w), _ptr(codes),
+                                        _ptr(clip), _stream())
+    _check(rc, "efqat_fake_quant_weight")
+    return codes, clip
+
+
+def init_act_qparams(ctx: Context, x, x_bits=8, x_symmetric=False):
+    """efqat_init_act_qparams: returns (s_x[1], z_x[1])."""
+    _dev(x)
+    spec = QSpec(8, x_bits, 1 if x_symmetric else 0)
+    s = torch.empty(1, dtype=torch.float32, device=x.device)
+    z = torch.empty(1, dtype=torch.float32, device=x.device)
+    ws = alloc_workspace(8192, x.device)
+    rc = load().efqat_init_act_qparams(ctx.handle, C.byref(spec), _dtype_code(x), _ptr(x), x.numel(), _ptr(s),
+                                       _ptr(z), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "efqat_init_act_qparams")
+    return s, z
+
+
+def init_weight_scales(ctx: Context, W, w_bits=8):
+    """efqat_init_weight_scales: returns s_w[N]."""
+    _dev(W)
+    spec = QSpec(w_bits, 8, 0)
+    N = int(W.shape[0])
+    K = int(W.numel() // N)
+    s = torch.empty(N, dtype=torch.float32, device=W.device)
+    rc = load().efqat_init_weight_scales(ctx.handle, C.byref(spec), _ptr(W), N, K, _ptr(s), _stream())
+    _check(rc, "efqat_init_weight_scales")
+    return s
+
+
+def gemm_bf16(ctx: Context, A, B, M: int, N: int, K: int, a_mn: bool, b_mn: bool, splits: int = 1):
+    """efqat_gemm_bf16: returns the fp32 slabs [splits, N, M] (transposed product per split)."""
+    _dev(A)
+    _dev(B)
+    out = torch.empty((splits, N, M), dtype=torch.float32, device=A.device)
+    rc = load().efqat_gemm_bf16(ctx.handle, _ptr(A), _ptr(B), M, N, K, int(a_mn), int(b_mn), int(splits),
+                                _ptr(out), _stream())
+    _check(rc, "efqat_gemm_bf16")
+    return out

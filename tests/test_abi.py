@@ -1,0 +1,88 @@
+"""CPU-only checks of the C ABI: the library loads, exports every symbol the header
+declares, and the host-side validation returns its error codes without touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2411_11038_b200 import binding as B
+from paper_2411_11038_b200 import build as build_mod
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_mod.build()
+    return B.load()
+
+
+def test_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "efqat.h")).read()
+    declared = set(re.findall(r"\b(efqat_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(B.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings(lib):
+    seen = set()
+    for code in list(range(-10, 1)) + [1, 2, 3]:
+        s = B.status_string(code)
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 14
+    assert B.status_string(-99) == "unknown status"
+
+
+def test_ratio_to_k(lib):
+    assert B.ratio_to_k(0.05, 512) == 25
+    assert B.ratio_to_k(0.1, 221184) == 22118
+    assert B.ratio_to_k(0.0, 768) == 0 and B.ratio_to_k(1.0, 768) == 768
+    assert B.ratio_to_k(0.25, 2304) == 576 and B.ratio_to_k(0.05, 3072) == 153
+
+
+def test_validate_layer_codes(lib):
+    ok = B.layer_desc(256, 512, 512, B.F32)
+    spec = B.QSpec(8, 8, 1)
+    assert B.validate_layer(ok, spec) == 0
+    assert B.validate_layer(B.layer_desc(0, 512, 512, B.F32), spec) == -2
+    assert B.validate_layer(B.layer_desc(256, 510, 512, B.F32), spec) == -3
+    assert B.validate_layer(B.layer_desc(256, 512, 100, B.F32), spec) == -3
+    assert B.validate_layer(B.layer_desc(256, 512, 512, 7), spec) == -4
+    assert B.validate_layer(ok, B.QSpec(9, 8, 0)) == -5
+    assert B.validate_layer(ok, B.QSpec(8, 1, 0)) == -5
+    conv = B.ConvGeom(B=2, H=8, W=8, Cin=16, R=1, S=1)
+    assert B.validate_layer(B.layer_desc(128, 32, 16, B.BF16, conv), spec) == 0
+    assert B.validate_layer(B.layer_desc(127, 32, 16, B.BF16, conv), spec) == -2
+    conv2 = B.ConvGeom(B=2, H=8, W=8, Cin=16, R=3, S=3, stride=2, pad=1)
+    assert B.validate_layer(B.layer_desc(32, 32, 144, B.BF16, conv2), spec) == -9
+
+
+def test_workspace_queries(lib):
+    d = B.layer_desc(4096, 768, 768, B.BF16)
+    spec = B.QSpec(8, 8, 0)
+    w0 = B.workspace_bytes(d, spec, 0)
+    w38 = B.workspace_bytes(d, spec, 38)
+    wN = B.workspace_bytes(d, spec, 768)
+    assert 0 < w0 <= w38 <= wN
+    assert w0 >= 4096 * 768 * 2 + 768 * 768 * 2
+    with pytest.raises(B.EfqatError) as e:
+        B.workspace_bytes(d, spec, 769)
+    assert e.value.code == -8
+    assert B.select_workspace_bytes(144, 221184) > 221184 * 16
+
+
+def test_null_context_is_rejected_before_any_launch(lib):
+    d = B.layer_desc(256, 512, 512, B.F32)
+    spec = B.QSpec(8, 8, 1)
+    rc = lib.efqat_fq_linear_fwd(None, C.byref(d), C.byref(spec), None, None, None, None, None, None, None,
+                                 None, 0, None)
+    assert rc == -1
+    rc = lib.efqat_fq_linear_bwd(None, C.byref(d), C.byref(spec), None, None, None, None, None, None, None, 0,
+                                 None, None, None, None, None, None, None, None, 0, None)
+    assert rc == -1
+    code = C.c_int(0)
+    assert lib.efqat_device_status(None, C.byref(code)) == -1
+    assert lib.efqat_destroy(None) == -1

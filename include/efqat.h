@@ -94,6 +94,19 @@ const char* efqat_status_string(int status);
  * stream work of interest was enqueued.  *code = 0 or an EFQAT_DEV_* value. */
 int efqat_device_status(efqat_ctx* ctx, int* code);
 
+/* ---- measurement aids --------------------------------------------------------- */
+/* Per-kernel timing for benchmarks.  While enabled, each of the three tensor-core
+ * launches (which = 0 forward GEMM, 1 grad-input GEMM, 2 weight-gradient GEMM) is
+ * bracketed by a pair of CUDA events on the caller's stream.  The events are created by
+ * the enabling call (never on the hot path); at most 8192 launches per kind are kept
+ * between two reads, later ones are not recorded. */
+int efqat_profile_enable(efqat_ctx* ctx, int enable);
+/* Synchronises the device, returns the summed duration (ms) and number of recorded
+ * launches of kernel `which` since the previous read, and clears the record. */
+int efqat_profile_read(efqat_ctx* ctx, int which, float* ms_total, int* launches);
+/* Number of kernels the library has launched in this process. */
+int64_t efqat_launch_count(void);
+
 /* ---- host-only helpers ---------------------------------------------------------- */
 /* floor(ratio * n): number of unfrozen channels for ratio r (Eq. 7). */
 int64_t efqat_ratio_to_k(double ratio, int64_t n);

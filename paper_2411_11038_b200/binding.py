@@ -26,6 +26,7 @@ EXPORTS = [
     "efqat_select_workspace_bytes", "efqat_select_channels", "efqat_fq_linear_fwd",
     "efqat_fq_linear_bwd", "efqat_fake_quant_act", "efqat_fake_quant_weight",
     "efqat_init_act_qparams", "efqat_init_weight_scales", "efqat_gemm_bf16",
+    "efqat_profile_enable", "efqat_profile_read", "efqat_launch_count",
 ]
 
 
@@ -83,9 +84,13 @@ def load() -> C.CDLL:
     lib.efqat_init_act_qparams.argtypes = [vp, C.POINTER(QSpec), i32, vp, i64, vp, vp, vp, sz, vp]
     lib.efqat_init_weight_scales.argtypes = [vp, C.POINTER(QSpec), vp, i64, i64, vp, vp]
     lib.efqat_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp]
+    lib.efqat_profile_enable.argtypes = [vp, i32]
+    lib.efqat_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]
+    lib.efqat_launch_count.argtypes = []
+    lib.efqat_launch_count.restype = i64
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("efqat_status_string", "efqat_ratio_to_k"):
+        if name not in ("efqat_status_string", "efqat_ratio_to_k", "efqat_launch_count"):
             fn.restype = i32
     _lib = lib
     return lib
@@ -138,6 +143,15 @@ class Context:
         _check(load().efqat_device_status(self.handle, C.byref(code)), "efqat_device_status")
         return code.value
 
+    def profile_enable(self, on: bool = True):
+        _check(load().efqat_profile_enable(self.handle, 1 if on else 0), "efqat_profile_enable")
+
+    def profile_read(self, which: int):
+        """(total ms, launches) of kernel `which` (0 fwd, 1 dX, 2 dW GEMM) since the last read."""
+        ms, n = C.c_float(0), C.c_int(0)
+        _check(load().efqat_profile_read(self.handle, int(which), C.byref(ms), C.byref(n)), "efqat_profile_read")
+        return ms.value, n.value
+
     def close(self):
         if getattr(self, "handle", None):
             load().efqat_destroy(self.handle)
@@ -170,6 +184,10 @@ def layer_desc(M: int, N: int, K: int, act_dtype: int, conv: Optional[ConvGeom] 
         d.B, d.H, d.W, d.Cin, d.R, d.S, d.stride, d.pad = (conv.B, conv.H, conv.W, conv.Cin, conv.R, conv.S,
                                                          conv.stride, conv.pad)
     return d
+
+
+def launch_count() -> int:
+    return int(load().efqat_launch_count())
 
 
 def ratio_to_k(ratio: float, n: int) -> int:

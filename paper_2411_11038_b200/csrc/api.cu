@@ -1,17 +1,30 @@
 // C ABI of the library: argument validation, workspace carving and the launch sequence
 // of each entry point.  Every step of the path runs in this library's kernels; there is
 // no host fallback.
+#include <atomic>
 #include <new>
+#include <vector>
 
 #include "internal.h"
 
 using namespace efqat;
 
+static const int PROF_KINDS = 3;       // 0 forward GEMM, 1 grad-input GEMM, 2 weight-grad GEMM
+static const int PROF_RING = 8192;     // event pairs kept per kind between two reads
+
 struct efqat_ctx {
   int device;
   int sm_count;
   int* d_status;
+  int prof_on;
+  std::vector<cudaEvent_t> ev[PROF_KINDS];   // start/stop pairs, created by efqat_profile_enable
+  int ev_used[PROF_KINDS];
 };
+
+static std::atomic<long long> g_launches{0};
+namespace efqat {
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace efqat
 
 namespace {
 
@@ -96,6 +109,19 @@ int guard_device(const efqat_ctx* ctx) {
 
 int last_error() { return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA; }
 
+// run_gemm, bracketed by a pair of events when per-kernel timing is switched on.
+int timed_gemm(efqat_ctx* ctx, int kind, const GemmArgs& g, cudaStream_t st, int* tiles = nullptr) {
+  const bool rec = ctx->prof_on && ctx->ev_used[kind] < PROF_RING;
+  const int slot = ctx->ev_used[kind];
+  if (rec) cudaEventRecord(ctx->ev[kind][2 * slot], st);
+  const int rc = run_gemm(g, ctx->sm_count, st, tiles);
+  if (rec) {
+    cudaEventRecord(ctx->ev[kind][2 * slot + 1], st);
+    ctx->ev_used[kind] = slot + 1;
+  }
+  return rc;
+}
+
 }  // namespace
 
 extern "C" {
@@ -111,6 +137,8 @@ int efqat_create(efqat_ctx** out, int device) {
   efqat_ctx* c = new (std::nothrow) efqat_ctx();
   if (!c) return EFQAT_ERR_CUDA;
   c->device = device;
+  c->prof_on = 0;
+  for (int k = 0; k < PROF_KINDS; ++k) c->ev_used[k] = 0;
   int rc = EFQAT_OK;
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
       cudaMalloc(&c->d_status, 256) != cudaSuccess || cudaMemset(c->d_status, 0, 256) != cudaSuccess)
@@ -128,6 +156,8 @@ int efqat_create(efqat_ctx** out, int device) {
 int efqat_destroy(efqat_ctx* ctx) {
   if (!ctx) return EFQAT_ERR_NULL;
   if (ctx->d_status) cudaFree(ctx->d_status);
+  for (int k = 0; k < PROF_KINDS; ++k)
+    for (cudaEvent_t e : ctx->ev[k]) cudaEventDestroy(e);
   delete ctx;
   return EFQAT_OK;
 }
@@ -159,6 +189,41 @@ int efqat_device_status(efqat_ctx* ctx, int* code) {
   if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) return EFQAT_ERR_CUDA;
   return EFQAT_OK;
 }
+
+int efqat_profile_enable(efqat_ctx* ctx, int enable) {
+  if (!ctx) return EFQAT_ERR_NULL;
+  int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  if (enable && ctx->ev[0].empty()) {
+    for (int k = 0; k < PROF_KINDS; ++k) {
+      ctx->ev[k].resize(2 * PROF_RING);
+      for (auto& e : ctx->ev[k])
+        if (cudaEventCreate(&e) != cudaSuccess) return EFQAT_ERR_CUDA;
+    }
+  }
+  for (int k = 0; k < PROF_KINDS; ++k) ctx->ev_used[k] = 0;
+  ctx->prof_on = enable ? 1 : 0;
+  return EFQAT_OK;
+}
+
+int efqat_profile_read(efqat_ctx* ctx, int which, float* ms_total, int* launches) {
+  if (!ctx || !ms_total || !launches) return EFQAT_ERR_NULL;
+  if (which < 0 || which >= PROF_KINDS) return EFQAT_ERR_MODE;
+  if (cudaDeviceSynchronize() != cudaSuccess) return EFQAT_ERR_CUDA;
+  double total = 0.0;
+  for (int i = 0; i < ctx->ev_used[which]; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->ev[which][2 * i], ctx->ev[which][2 * i + 1]) != cudaSuccess)
+      return EFQAT_ERR_CUDA;
+    total += ms;
+  }
+  *ms_total = static_cast<float>(total);
+  *launches = ctx->ev_used[which];
+  ctx->ev_used[which] = 0;
+  return EFQAT_OK;
+}
+
+int64_t efqat_launch_count(void) { return static_cast<int64_t>(g_launches.load()); }
 
 int64_t efqat_ratio_to_k(double ratio, int64_t n) {
   if (!(ratio > 0.0) || n <= 0) return 0;
@@ -248,7 +313,7 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   g.col_scale = s_w; g.col_bias = bias_or_null;
   g.xq = w.actq;
   g.status = ctx->d_status;
-  rc = run_gemm(g, ctx->sm_count, st);
+  rc = timed_gemm(ctx, 0, g, st);
   if (rc != EFQAT_OK) return rc;
   return last_error();
 }
@@ -300,7 +365,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.partials = w.dxpart;
     g.status = ctx->d_status;
     int tiles = 0;
-    rc = run_gemm(g, ctx->sm_count, st, &tiles);
+    rc = timed_gemm(ctx, 1, g, st, &tiles);
     if (rc != EFQAT_OK) return rc;
     launch_dx_finalize(w.dxpart, tiles, dS_x, dZ_x, st);
   }
@@ -328,7 +393,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.split_stride = k_sel * K;
     g.part_cols = k_sel;
     g.status = ctx->d_status;
-    rc = run_gemm(g, ctx->sm_count, st);
+    rc = timed_gemm(ctx, 2, g, st);
     if (rc != EFQAT_OK) return rc;
     launch_dw_finalize(w.P, w.splits, k_sel * K, k_sel, N, K, W, s_w, gathered ? idx : nullptr, w.actq,
                        q->w_bits, dW_sel, dS_w_sel, opt_or_null, ctx->d_status, st);

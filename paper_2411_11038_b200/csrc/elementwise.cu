@@ -33,6 +33,7 @@ __global__ void prep_act_kernel(const float* __restrict__ s_x, const float* __re
 
 void launch_prep_act(const float* s_x, const float* z_x, int x_bits, int x_sym, ActQ* out, int* status,
                      cudaStream_t st) {
+  count_launches(1);
   prep_act_kernel<<<1, 32, 0, st>>>(s_x, z_x, x_bits, x_sym, out, status);
 }
 
@@ -104,6 +105,7 @@ void launch_quant_act_operand(const void* X, int dtype, int64_t count, const Act
   const int64_t n8 = count / 8;
   if (n8 == 0) return;
   const int g = grid_for(n8, 256);
+  count_launches(1);
   if (dtype == EFQAT_BF16)
     quant_act_operand_kernel<bf16><<<g, 256, 0, st>>>(static_cast<const bf16*>(X), n8, q, out);
   else
@@ -126,6 +128,7 @@ void launch_quant_act_export(const void* X, int dtype, int64_t count, const ActQ
                              uint8_t* clip, cudaStream_t st) {
   if (count == 0) return;
   const int g = grid_for(count, 256);
+  count_launches(1);
   if (dtype == EFQAT_BF16)
     quant_act_export_kernel<bf16><<<g, 256, 0, st>>>(static_cast<const bf16*>(X), count, q, codes, clip);
   else
@@ -165,6 +168,7 @@ __global__ void __launch_bounds__(256) quant_weight_operand_kernel(const float* 
 void launch_quant_weight_operand(const float* W, int64_t N, int64_t K, const float* s_w, int w_bits, int mode,
                                  bf16* out, int* status, cudaStream_t st) {
   if (N == 0) return;
+  count_launches(1);
   if (mode == 0)
     quant_weight_operand_kernel<0><<<static_cast<unsigned>(N), 256, 0, st>>>(W, K, s_w, w_bits, out, status);
   else
@@ -191,6 +195,7 @@ __global__ void quant_weight_export_kernel(const float* __restrict__ W, int64_t 
 void launch_quant_weight_export(const float* W, int64_t N, int64_t K, const float* s_w, int w_bits,
                                 int32_t* codes, uint8_t* clip, int* status, cudaStream_t st) {
   if (N == 0) return;
+  count_launches(1);
   quant_weight_export_kernel<<<static_cast<unsigned>(N), 256, 0, st>>>(W, K, s_w, w_bits, codes, clip, status);
 }
 
@@ -207,6 +212,7 @@ __global__ void __launch_bounds__(256) to_bf16_kernel(const float* __restrict__ 
 void launch_to_bf16(const float* in, int64_t count, bf16* out, cudaStream_t st) {
   const int64_t n8 = count / 8;
   if (n8 == 0) return;
+  count_launches(1);
   to_bf16_kernel<<<grid_for(n8, 256), 256, 0, st>>>(in, n8, out);
 }
 
@@ -252,6 +258,7 @@ void launch_gather_cols(const void* dY, int dtype, int64_t M, int64_t N, const i
   if (M == 0 || pitch == 0) return;
   const int g = grid_for(ceil_div(M, 8), 1, 148 * 8);
   const size_t sm = static_cast<size_t>(pitch) * sizeof(int32_t);
+  count_launches(1);
   if (dtype == EFQAT_BF16)
     gather_cols_kernel<bf16><<<g, 256, sm, st>>>(static_cast<const bf16*>(dY), M, N, idx,
                                                  static_cast<int>(k_sel), static_cast<int>(pitch), out, status);
@@ -296,6 +303,7 @@ void launch_colsum(const void* dY, int dtype, int64_t M, int64_t N, float* ws, f
   if (slabs > COLSUM_SLABS) slabs = COLSUM_SLABS;
   if (slabs < 1) slabs = 1;
   dim3 g(static_cast<unsigned>(ceil_div(N, 128 * 8)), slabs);
+  count_launches(2);
   if (dtype == EFQAT_BF16)
     colsum_stage1_kernel<bf16><<<g, 128, 0, st>>>(static_cast<const bf16*>(dY), M, N, ws);
   else
@@ -328,6 +336,7 @@ __global__ void __launch_bounds__(256) dx_finalize_kernel(const float* __restric
   }
 }
 void launch_dx_finalize(const float* partials, int n, float* dS_x, float* dZ_x, cudaStream_t st) {
+  count_launches(1);
   dx_finalize_kernel<<<1, 256, 0, st>>>(partials, n, dS_x, dZ_x);
 }
 
@@ -388,6 +397,7 @@ void launch_dw_finalize(const float* P, int splits, int64_t split_stride, int64_
   if (k_sel == 0) return;
   efqat_sgd o = {};
   if (opt) o = *opt;
+  count_launches(1);
   dw_finalize_kernel<<<static_cast<unsigned>(k_sel), 256, 0, st>>>(P, splits, split_stride, K, W, s_w, idx_or_null,
                                                                   N, xq, w_bits, dW_sel, dS_w_sel, o,
                                                                   opt != nullptr, status);
@@ -445,6 +455,7 @@ __global__ void minmax_stage2_kernel(const float* __restrict__ ws, int nblocks, 
 void launch_minmax_act(const void* x, int dtype, int64_t count, int x_bits, int x_sym, float* s_x, float* z_x,
                        float* ws, cudaStream_t st) {
   const int g = grid_for(count, 256 * 8, 1024);
+  count_launches(2);
   if (dtype == EFQAT_BF16)
     minmax_stage1_kernel<bf16><<<g, 256, 0, st>>>(static_cast<const bf16*>(x), count, ws);
   else
@@ -472,6 +483,7 @@ __global__ void __launch_bounds__(256) absmax_rows_kernel(const float* __restric
 }
 void launch_absmax_rows(const float* W, int64_t N, int64_t K, int w_bits, float* s_w, cudaStream_t st) {
   if (N == 0) return;
+  count_launches(1);
   absmax_rows_kernel<<<static_cast<unsigned>(N), 256, 0, st>>>(W, K, w_bits, s_w);
 }
 

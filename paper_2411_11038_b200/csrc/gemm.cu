@@ -370,6 +370,7 @@ static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams
       return EFQAT_ERR_CUDA;
     configured[dev] = true;
   }
+  count_launches(1);
   kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, p);
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }

@@ -11,6 +11,9 @@ namespace efqat {
 
 typedef __nv_bfloat16 bf16;
 
+// Number of kernels this library has launched in this process (reported by efqat_launch_count).
+void count_launches(int n);
+
 // ---- elementwise.cu -----------------------------------------------------------------
 void launch_prep_act(const float* s_x, const float* z_x, int x_bits, int x_sym, ActQ* out, int* status,
                      cudaStream_t st);

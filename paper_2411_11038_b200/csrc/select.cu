@@ -335,15 +335,18 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
       row_off += layers[l].N;
       out_off += e.k;
     }
+    count_launches(1);
     table_write_kernel<<<1, TABLE_CHUNK, 0, st>>>(chunk, cnt, w.table + base);
   }
   const int tot = static_cast<int>(total);
   {
     int64_t blocks = ceil_div(total, 8);
     if (blocks > 148 * 8) blocks = 148 * 8;
+    count_launches(1);
     row_importance_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(w.table, L, tot, w.keys, w.rowsum);
   }
   if (mode == EFQAT_CWPL) {
+    count_launches(2);
     topk_kernel<<<L, TOPK_THREADS, 0, st>>>(w.keys, w.table, 0, 0, idx);
     cwpl_offsets_kernel<<<static_cast<unsigned>(ceil_div(L + 1, 256)), 256, 0, st>>>(w.table, L,
                                                                                     static_cast<int>(out_off),
@@ -351,6 +354,7 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
     if (importance) cudaMemcpyAsync(importance, w.keys, sizeof(float) * total, cudaMemcpyDeviceToDevice, st);
   } else if (mode == EFQAT_CWPN) {
     const int kt = static_cast<int>(k[0]);
+    count_launches(2);
     topk_kernel<<<1, TOPK_THREADS, 0, st>>>(w.keys, nullptr, tot, kt, w.sel);
     const int work = (kt > L + 1) ? kt : L + 1;
     cwpn_split_kernel<<<static_cast<unsigned>(ceil_div(work, 256)), 256, 0, st>>>(w.table, L, w.sel, kt, idx,
@@ -358,6 +362,7 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
     if (importance) cudaMemcpyAsync(importance, w.keys, sizeof(float) * total, cudaMemcpyDeviceToDevice, st);
   } else {
     const int kl = static_cast<int>(k[0]);
+    count_launches(4);
     layer_importance_kernel<<<L, 256, 0, st>>>(w.table, w.rowsum, w.layer_keys);
     topk_kernel<<<1, TOPK_THREADS, 0, st>>>(w.layer_keys, nullptr, L, kl, w.lsel);
     lwpn_offsets_kernel<<<1, 32, 0, st>>>(w.table, L, w.lsel, kl, w.keep, offsets);

@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the EfQAT layer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--frac R]
+
+Workload: the four BERT-base-shaped encoder linears at M = 32 x 128 = 4096 tokens with
+bf16 activations, W8A8, per-layer channel selection.  One step = one pass of the whole
+path over one batch: importance + Top-K selection for the four layers, then for each
+layer the fake-quantised forward and the partial backward (dX, dS_x, dZ_x, db, and dW /
+dS_w of the selected channels only).
+
+The printed JSON line reports the step throughput in algorithmic TFLOP/s
+(2MNK forward + 2MNK(1 + k/N) backward), the backward-only sweep over the unfrozen
+fractions with its speed-up over the library's own full-QAT backward, the tensor-core
+roofline of the dominant GEMM kernel, the oracle's CPU time on the same workload and the
+end-to-end number with host buffers.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2411_11038_b200 import inputs as I  # noqa: E402
+
+FRACS = (0.0, 0.05, 0.25, 1.0)
+METRIC = "fq-linear step TFLOP/s (select + fwd + partial bwd); bwd TFLOP/s and speedup vs full-QAT bwd per unfrozen % in 'bwd'"
+L2_FLUSH_BYTES = 256 << 20
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture of the current kernel exists).
+DOMINANT_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(tflops=float(d["bf16_tflops"]), tflops_sustained=float(d.get("bf16_tflops_sustained", 0)),
+                    hbm_gbs=float(d["hbm_gbs"]), source="measured")
+    return dict(tflops=1590.0, tflops_sustained=1400.0, hbm_gbs=6650.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+        }
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def summary(self):
+        return dict(sm_mhz=(statistics.median(self.samples) if self.samples else None),
+                    sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=len(self.samples))
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ----------------------------------------------------------------------------------------
+class Workload:
+    """Device-resident tensors and pre-marshalled calls of the four layers."""
+
+    def __init__(self, ctx, device):
+        from paper_2411_11038_b200 import binding as B
+        self.B, self.ctx, self.device = B, ctx, device
+        self.cases = I.config2()
+        self.layers = []
+        for c in self.cases:
+            T = I.make_tensors(c)
+            D = {k: v.to(device) for k, v in T.items()}
+            D["s_w"] = B.init_weight_scales(ctx, D["W"], c.w_bits)
+            D["s_x"], D["z_x"] = B.init_act_qparams(ctx, D["X"], c.x_bits, c.x_symmetric)
+            D["host_X"] = T["X"].pin_memory()
+            D["host_dY"] = T["dY"].pin_memory()
+            plan = B.LayerPlan(ctx, c.M, c.N, c.K, c.act_dtype, c.w_bits, c.x_bits, c.x_symmetric, c.N, device)
+            D["host_dW"] = torch.empty((c.N, c.K), dtype=torch.float32).pin_memory()
+            D["host_small"] = torch.empty(2 * c.N + 2, dtype=torch.float32).pin_memory()
+            self.layers.append((c, D, plan))
+        self.sel = {}
+        for f in FRACS:
+            ks = [B.ratio_to_k(f, c.N) for c in self.cases]
+            plan = B.SelectPlan(ctx, B.CWPL, [D["W"] for _, D, _ in self.layers], ks)
+            offs = np.concatenate([[0], np.cumsum(ks)]).astype(int)
+            views = [plan.idx[offs[i]:offs[i + 1]] if ks[i] else None for i in range(len(ks))]
+            self.sel[f] = (plan, ks, views)
+        self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+
+    def flops(self, frac, fwd=True, bwd=True):
+        tot = 0.0
+        _, ks, _ = self.sel[frac]
+        for (c, _, _), k in zip(self.layers, ks):
+            g = 2.0 * c.M * c.N * c.K
+            if fwd:
+                tot += g
+            if bwd:
+                tot += g + 2.0 * c.M * k * c.K
+        return tot
+
+    def gemm_flops(self, frac):
+        """Algorithmic FLOPs of the three GEMM kinds per step: fwd, dX, dW."""
+        _, ks, _ = self.sel[frac]
+        full = sum(2.0 * c.M * c.N * c.K for c, _, _ in self.layers)
+        dw = sum(2.0 * c.M * k * c.K for (c, _, _), k in zip(self.layers, ks))
+        return [full, full, dw]
+
+    def select(self, frac):
+        self.sel[frac][0].run()
+
+    def backward(self, frac):
+        _, ks, views = self.sel[frac]
+        for (c, D, plan), k, idx in zip(self.layers, ks, views):
+            plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True)
+
+    def step(self, frac):
+        self.select(frac)
+        for c, D, plan in self.layers:
+            plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"])
+        self.backward(frac)
+
+    def step_e2e(self, frac):
+        """Same step with this step's activations coming from pinned host memory and the
+        parameter gradients going back to it."""
+        _, ks, _ = self.sel[frac]
+        for c, D, plan in self.layers:
+            D["X"].copy_(D["host_X"], non_blocking=True)
+            D["dY"].copy_(D["host_dY"], non_blocking=True)
+        self.step(frac)
+        for (c, D, plan), k in zip(self.layers, ks):
+            if k:
+                D["host_dW"][:k].copy_(plan.dW_sel[:k], non_blocking=True)
+                D["host_small"][:k].copy_(plan.dS_w_sel[:k], non_blocking=True)
+            D["host_small"][c.N:2 * c.N].copy_(plan.db, non_blocking=True)
+            D["host_small"][2 * c.N:2 * c.N + 1].copy_(plan.dS_x, non_blocking=True)
+            D["host_small"][2 * c.N + 1:].copy_(plan.dZ_x, non_blocking=True)
+
+    def e2e_bytes(self, frac):
+        _, ks, _ = self.sel[frac]
+        bi = sum(D["host_X"].numel() * 2 + D["host_dY"].numel() * 2 for _, D, _ in self.layers)
+        bo = sum(k * c.K * 4 + k * 4 + c.N * 4 + 8 for (c, _, _), k in zip(self.layers, ks))
+        return bi, bo
+
+
+def timed(fn, steps, warmup, flush, sync_all=None, after_warmup=None):
+    """Sum of per-step device durations (ms); L2 is flushed, untimed, before every step."""
+    for _ in range(warmup):
+        flush.zero_()
+        fn()
+    if sync_all:
+        sync_all()
+    torch.cuda.synchronize()
+    if after_warmup:
+        after_warmup()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for i in range(steps):
+        flush.zero_()
+        starts[i].record()
+        fn()
+        ends[i].record()
+    torch.cuda.synchronize()
+    if sync_all:
+        sync_all()
+    return sum(s.elapsed_time(e) for s, e in zip(starts, ends))
+
+
+# ----------------------------------------------------------------------------------------
+def oracle_step_seconds(frac, layers=None, rows=None):
+    """One pass of the oracle, as it stands, over the same workload (CPU, fp64)."""
+    from oracle import efqat_oracle as O
+    cases = I.config2()
+    if layers is not None:
+        cases = [cases[i] for i in layers]
+    if rows is not None:
+        cases = [I.shrink(c, rows) for c in cases]
+    flops = 0.0
+    t0 = time.perf_counter()
+    for c in cases:
+        T = I.make_tensors(c)
+        X, W, dY, b = (I.as_f64(T[k]) for k in ("X", "W", "dY", "bias"))
+        s_w = O.init_minmax_w(W, c.w_bits)
+        s_x, z_x = O.init_minmax_x(X, c.x_bits, c.x_symmetric)
+        k = O.ratio_to_k(frac, c.N)
+        idx = O.select_cwpl([W], [k])[0]
+        O.forward(X, W, s_w, s_x, z_x, b, c.w_bits, c.x_bits, c.x_symmetric)
+        O.backward_efqat(dY, X, W, s_w, s_x, z_x, idx, c.w_bits, c.x_bits, c.x_symmetric)
+        flops += 2.0 * c.M * c.N * c.K * 2 + 2.0 * c.M * k * c.K
+    return time.perf_counter() - t0, flops, [c.name for c in cases]
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    frac = args.frac
+    layers, rows = [1], 1024    # bounded sample: 1024 tokens of the 768 -> 768 attention-output layer
+    for _ in range(min(args.warmup, 3)):
+        oracle_step_seconds(frac, layers, rows)
+    tot, fl, names = 0.0, 0.0, []
+    for _ in range(args.steps):
+        s, f, names = oracle_step_seconds(frac, layers, rows)
+        tot += s
+        fl += f
+    val = fl / tot / 1e12
+    cores = os.cpu_count()
+    sample = f"oracle fwd + EfQAT bwd (fp64 numpy) on layer {names[0]} (first {rows} tokens), {int(frac * 100)}% unfrozen"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "configs[1] BERT-base-shaped linears (bounded sample)", "unfrozen": frac},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    from paper_2411_11038_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if dist is None:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    ctx = B.Context(local)
+    wl = Workload(ctx, dev)
+    frac = args.frac
+    peaks = load_peaks()
+
+    # ---- headline: K steps of the whole path, device-resident inputs
+    sampler = ClockSampler(physical_gpu_index(local))
+    mark = {}
+
+    def start_counting():
+        mark["launches"] = B.launch_count()
+        ctx.profile_enable(True)
+        sampler.start()
+
+    total_ms = timed(lambda: wl.step(frac), args.steps, args.warmup, wl.flush, sync_all, start_counting)
+    sampler.stop_flag = True
+    kinds = [ctx.profile_read(i) for i in range(3)]      # (total ms, launches) of the timed steps only
+    ctx.profile_enable(False)
+    launches = B.launch_count() - mark["launches"]
+    sampler.join(timeout=2)
+    total_ms = max_over_ranks(total_ms)
+    ms_per_step = total_ms / args.steps
+    value = world * wl.flops(frac) / (ms_per_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (largest share of GEMM time in the timed region)
+    gf = wl.gemm_flops(frac)
+    names = ["gemm_kernel<fwd epilogue>", "gemm_kernel<dX epilogue>", "gemm_kernel<dW partial epilogue>"]
+    dom = max(range(3), key=lambda i: kinds[i][0])
+    dom_ms, dom_n = kinds[dom]
+    avg_launch_ms = dom_ms / max(dom_n, 1)
+    # algorithmic FLOPs of all launches of that kind in the timed region / their summed duration
+    achieved = (gf[dom] * args.steps) / (dom_ms * 1e-3) / 1e12 if dom_n else None
+    roofline = {"bound": "tensor", "kernel": names[dom], "achieved": achieved, "peak": peaks["tflops"],
+                "unit": "TFLOP/s", "frac": (achieved / peaks["tflops"]) if achieved else None,
+                "traffic": DOMINANT_TRAFFIC_BYTES, "peak_source": f"{peaks['source']} burst bf16 GEMM",
+                "launches": dom_n, "avg_launch_ms": avg_launch_ms,
+                "gemm_ms_per_step": {n: kinds[i][0] / args.steps for i, n in enumerate(names)}}
+
+    # ---- backward-only sweep over the unfrozen fractions
+    sweep_steps = max(20, args.steps // 4)
+    bwd = {}
+    for f in FRACS:
+        wl.select(f)
+        ms = timed(lambda: wl.backward(f), sweep_steps, 5, wl.flush, sync_all) / sweep_steps
+        ms = max_over_ranks(ms)
+        bwd[f] = ms
+    bwd_report = {}
+    for f in FRACS:
+        fl = wl.flops(f, fwd=False)
+        bwd_report[f"{int(round(f * 100))}%"] = {
+            "ms": bwd[f], "tflops": fl / (bwd[f] * 1e-3) / 1e12, "speedup_vs_full_qat": bwd[1.0] / bwd[f],
+            "ideal_speedup": 2.0 / (1.0 + f)}
+    sel_ms = max_over_ranks(timed(lambda: wl.select(frac), sweep_steps, 5, wl.flush, sync_all) / sweep_steps)
+
+    # ---- end to end: inputs from pinned host memory, parameter gradients back to it
+    e2e_steps = max(10, args.steps // 4)
+    e2e_ms = max_over_ranks(timed(lambda: wl.step_e2e(frac), e2e_steps, 3, wl.flush, sync_all) / e2e_steps)
+    bi, bo = wl.e2e_bytes(frac)
+    e2e_val = world * wl.flops(frac) / (e2e_ms * 1e-3) / 1e12
+    status = ctx.device_status()
+
+    # ---- the oracle on this machine's host cores (rank 0, single GPU only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        s, fl, names_c = oracle_step_seconds(frac)
+        cpu = {"value": fl / s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+               "seconds": s, "sample": f"one full step of the workload ({', '.join(names_c)}), oracle fwd + EfQAT bwd "
+                                        f"in fp64 numpy, {int(frac * 100)}% unfrozen"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "configs[1]: BERT-base-shaped linears 768->2304, 768->768, 768->3072, 3072->768 "
+                                   "at M=4096, bf16 activations, W8A8, CWPL",
+                       "unfrozen": frac, "l2": "256 MiB buffer written between timed steps",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": sampler.summary(),
+            "e2e": {"value": e2e_val, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": bi,
+                    "d2h_bytes_per_step": bo},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+            "bwd": bwd_report,
+            "select_ms": sel_ms,
+            "device_status": status,
+            "paper_context": "paper reports 1.44-1.64x backward speed-up on A10/A100 (whole network)",
+        }))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--frac", type=float, default=0.05, choices=list(FRACS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -330,21 +330,23 @@ def run_ours(args):
     # ---- backward-only sweep over the unfrozen fractions
     sweep_steps = max(20, args.steps // 4)
     bwd = {}
-    for f in FRACS:
+    for f in (() if args.skip_extras else FRACS):
         wl.select(f)
         ms = timed(lambda: wl.backward(f), sweep_steps, 5, wl.flush, sync_all) / sweep_steps
         ms = max_over_ranks(ms)
         bwd[f] = ms
     bwd_report = {}
-    for f in FRACS:
+    for f in (() if args.skip_extras else FRACS):
         fl = wl.flops(f, fwd=False)
         bwd_report[f"{int(round(f * 100))}%"] = {
             "ms": bwd[f], "tflops": fl / (bwd[f] * 1e-3) / 1e12, "speedup_vs_full_qat": bwd[1.0] / bwd[f],
             "ideal_speedup": 2.0 / (1.0 + f)}
-    sel_ms = max_over_ranks(timed(lambda: wl.select(frac), sweep_steps, 5, wl.flush, sync_all) / sweep_steps)
+    sel_ms = None
+    if not args.skip_extras:
+        sel_ms = max_over_ranks(timed(lambda: wl.select(frac), sweep_steps, 5, wl.flush, sync_all) / sweep_steps)
 
     # ---- end to end: inputs from pinned host memory, parameter gradients back to it
-    e2e_steps = max(10, args.steps // 4)
+    e2e_steps = 3 if args.skip_extras else max(10, args.steps // 4)
     e2e_ms = max_over_ranks(timed(lambda: wl.step_e2e(frac), e2e_steps, 3, wl.flush, sync_all) / e2e_steps)
     bi, bo = wl.e2e_bytes(frac)
     e2e_val = world * wl.flops(frac) / (e2e_ms * 1e-3) / 1e12
@@ -352,7 +354,7 @@ def run_ours(args):
 
     # ---- the oracle on this machine's host cores (rank 0, single GPU only)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.skip_extras:
         s, fl, names_c = oracle_step_seconds(frac)
         cpu = {"value": fl / s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
                "seconds": s, "sample": f"one full step of the workload ({', '.join(names_c)}), oracle fwd + EfQAT bwd "
@@ -390,6 +392,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--frac", type=float, default=0.05, choices=list(FRACS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="only the headline timed steps and a 3-step end-to-end leg (short run for profilers)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -45,6 +45,7 @@ typedef enum {
   EFQAT_ERR_K_RANGE = -8,    /* k_sel / budget outside its range */
   EFQAT_ERR_UNIMPL = -9,     /* combination not built (e.g. conv stride != 1) */
   EFQAT_ERR_CUDA = -10,      /* a CUDA runtime / driver call failed */
+  EFQAT_ERR_TOO_LARGE = -11, /* a size exceeds a fixed built-in maximum (efqat_colsum_noalloc) */
   /* device-side conditions, reported by efqat_device_status (positive) */
   EFQAT_DEV_BAD_SCALE = 1,   /* a scale was <= 0 or not finite */
   EFQAT_DEV_BAD_INDEX = 2,   /* idx entry outside [0,N) or not strictly ascending */
@@ -174,6 +175,26 @@ int efqat_init_act_qparams(efqat_ctx* ctx, const efqat_qspec* q, int dtype, cons
 /* Eq. 4 (weights, per output channel) -> s_w[N]. */
 int efqat_init_weight_scales(efqat_ctx* ctx, const efqat_qspec* q, const float* W, int64_t N, int64_t K,
                              float* s_w, efqat_stream_t stream);
+
+/* ---- allocation-free bias gradient ------------------------------------------------- */
+/* The paper has no counterpart to this call; it exists for integration reasons only.
+ * db[n] = sum_m dY[m,n] (fp32), the same column sums efqat_fq_linear_bwd writes to
+ * db_or_null, for callers that cannot allocate device memory at all and therefore can
+ * neither create a context nor provide a workspace: an enqueue hook of a runtime that hands
+ * out a fixed arena and forbids further allocation, a latency-critical loop that must not
+ * enter the allocator, a process whose device memory pool belongs to another component.
+ * The partial sums live in a 4 MiB device array built into the library (held on every
+ * GPU that loads it, for the life of the process).  Needs no efqat_ctx.  The call
+ * allocates nothing and frees nothing.
+ *   dY: device, [M,N] row-major in `dtype` (EFQAT_F32 / EFQAT_BF16), 16-byte aligned;
+ *   db: device, fp32 [N];  N % 8 == 0 and N <= 16384, else EFQAT_ERR_ALIGN /
+ *   EFQAT_ERR_TOO_LARGE; the CUDA device owning dY must be current.
+ * The first call on each device looks up the array's device address; make that call
+ * before starting any stream capture.  All calls share the one array and it keeps what the
+ * previous call left there (each call overwrites every element it reads, so nothing needs
+ * clearing), hence two calls whose kernels may overlap on the GPU -- different streams
+ * without ordering -- race with each other: serialise them. */
+int efqat_colsum_noalloc(int dtype, const void* dY, int64_t M, int64_t N, float* db, efqat_stream_t stream);
 
 /* ---- helper: the tensor-core contraction shared by a3, a4 and a6 (Eq. 5 shapes) -------- */
 /* out[n*M + m] = sum_k A(m,k) * B(n,k) in fp32, bf16 operands (device), i.e. the product is

@@ -26,7 +26,7 @@ EXPORTS = [
     "efqat_select_workspace_bytes", "efqat_select_channels", "efqat_fq_linear_fwd",
     "efqat_fq_linear_bwd", "efqat_fake_quant_act", "efqat_fake_quant_weight",
     "efqat_init_act_qparams", "efqat_init_weight_scales", "efqat_gemm_bf16",
-    "efqat_profile_enable", "efqat_profile_read", "efqat_launch_count",
+    "efqat_profile_enable", "efqat_profile_read", "efqat_launch_count", "efqat_colsum_noalloc",
 ]
 
 
@@ -86,6 +86,7 @@ def load() -> C.CDLL:
     lib.efqat_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp]
     lib.efqat_profile_enable.argtypes = [vp, i32]
     lib.efqat_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]
+    lib.efqat_colsum_noalloc.argtypes = [i32, vp, i64, i64, vp, vp]
     lib.efqat_launch_count.argtypes = []
     lib.efqat_launch_count.restype = i64
     for name in EXPORTS:
@@ -398,4 +399,16 @@ def gemm_bf16(ctx: Context, A, B, M: int, N: int, K: int, a_mn: bool, b_mn: bool
     rc = load().efqat_gemm_bf16(ctx.handle, _ptr(A), _ptr(B), M, N, K, int(a_mn), int(b_mn), int(splits),
                                 _ptr(out), _stream())
     _check(rc, "efqat_gemm_bf16")
+    return out
+
+
+def colsum_noalloc(dY: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """efqat_colsum_noalloc: column sums of a 2-D dY without context or workspace.  The
+    library call allocates nothing; `out` (fp32 [N]) is created here only if not given."""
+    _dev(dY)
+    M, N = int(dY.shape[0]), int(dY.shape[1])
+    if out is None:
+        out = torch.empty(N, dtype=torch.float32, device=dY.device)
+    rc = load().efqat_colsum_noalloc(_dtype_code(dY), _ptr(dY), M, N, _ptr(out), _stream())
+    _check(rc, "efqat_colsum_noalloc")
     return out

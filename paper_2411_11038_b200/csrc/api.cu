@@ -175,6 +175,7 @@ const char* efqat_status_string(int s) {
     case EFQAT_ERR_K_RANGE: return "selection count out of range";
     case EFQAT_ERR_UNIMPL: return "combination not implemented";
     case EFQAT_ERR_CUDA: return "CUDA call failed";
+    case EFQAT_ERR_TOO_LARGE: return "size exceeds a built-in maximum";
     case EFQAT_DEV_BAD_SCALE: return "device: scale not positive and finite";
     case EFQAT_DEV_BAD_INDEX: return "device: channel index out of range or not ascending";
     case EFQAT_DEV_WAIT_TIMEOUT: return "device: bounded wait expired";

@@ -28,11 +28,11 @@ def test_exports_every_declared_symbol(lib):
 
 def test_status_strings(lib):
     seen = set()
-    for code in list(range(-10, 1)) + [1, 2, 3]:
+    for code in list(range(-11, 1)) + [1, 2, 3]:
         s = B.status_string(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 14
+    assert len(seen) == 15
     assert B.status_string(-99) == "unknown status"
 
 

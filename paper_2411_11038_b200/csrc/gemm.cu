@@ -4,15 +4,16 @@
 //   EPI_DX  : dX = acc * [x not clipped]; partial sums of dS_x, dZ_x   (Eq. 5 + STE)
 //   EPI_PART: fp32 partial products of the (partial) weight gradient   (Algorithm 1)
 //
-// One CTA computes one 128 x BN output tile (optionally one split of the contraction):
+// Persistent kernel, one CTA per SM, looping over 128 x BN output tiles:
 //   warp 0  lane 0 : TMA producer over a ring of shared-memory stages
-//   warp 1  lane 0 : issues tcgen05.mma; warp 1 also owns the TMEM allocation
-//   warps 2..5     : epilogue, each reading its 32-lane quarter of the accumulator
+//   warp 1  lane 0 : issues tcgen05.mma into one of two TMEM accumulators; warp 1 owns TMEM
+//   warps 2..5     : epilogue of the previous tile, overlapped with the next tile's main loop;
+//                    each warp reads its 32-lane quarter of the accumulator, fetches its slice
+//                    of X with TMA (EPI_DX) and writes its slice of the output with TMA stores
+//                    from a swizzled staging buffer, so global traffic is in whole 128-byte rows
 // Either operand may be stored with the contraction dimension contiguous ("K-major") or
 // with the other dimension contiguous ("MN-major"); the shared-memory and instruction
 // descriptors carry the difference, so no transposed copies are ever made.
-#include <stdio.h>
-
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -27,6 +28,9 @@ static const int MAX_STAGES = 8;
 static const int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB
 static const int CHUNK_BYTES = 64 * BK * 2;     // one 64-wide MN-major chunk, 8 KiB
 static const int GEMM_THREADS = 192;
+static const int ACC_STRIDE = 256;              // TMEM columns between the two accumulators
+static const int TMEM_COLS = 512;
+static const int STG_BYTES = 32 * 128;          // staging slice of one epilogue warp: 32 rows x 128 B
 
 struct GemmParams {
   int64_t Mr, Nc;
@@ -34,17 +38,15 @@ struct GemmParams {
   int BN;             // tile columns (multiple of 16, <= 256)
   int stages;
   int b_stage_bytes;
-  int tmem_cols;
   int splits;
-  int out_bf16;
-  void* out;
-  int64_t ldo;
+  int tiles_m, tiles_n;
+  int chunk_cols;     // output columns per 128-byte staging row: 64 (bf16) or 32 (fp32)
   const float* col_scale;
   const float* col_bias;
   const ActQ* xq;
-  const void* X;
-  int x_dtype;
-  float* partials;
+  float* partials;    // EPI_DX: [tile][quarter][2]
+  float* out;         // EPI_PART
+  int64_t ldo;
   int64_t split_stride;
   int64_t part_cols;
   int* status;
@@ -53,82 +55,64 @@ struct GemmParams {
 struct __align__(8) SmemCtl {
   uint64_t full[MAX_STAGES];
   uint64_t empty[MAX_STAGES];
-  uint64_t acc_full;
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint64_t xbar[4][2];
   uint32_t tmem_base;
   int abort_flag;
-  float red[4][2];
 };
-
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Stores 8 consecutive outputs of one row (16-byte aligned by the N % 8 / K % 8 contract).
-__device__ __forceinline__ void store8(void* base, int64_t elem_off, const float* v, int as_bf16) {
-  if (as_bf16) {
-    uint4 o;
-    o.x = pack2(v[0], v[1]); o.y = pack2(v[2], v[3]); o.z = pack2(v[4], v[5]); o.w = pack2(v[6], v[7]);
-    *reinterpret_cast<uint4*>(static_cast<bf16*>(base) + elem_off) = o;
-  } else {
-    float4* p = reinterpret_cast<float4*>(static_cast<float*>(base) + elem_off);
-    p[0] = make_float4(v[0], v[1], v[2], v[3]);
-    p[1] = make_float4(v[4], v[5], v[6], v[7]);
-  }
-}
-__device__ __forceinline__ void load8(const void* base, int64_t elem_off, float* v, int is_bf16) {
-  if (is_bf16) {
-    const uint4 r = __ldg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(base) + elem_off));
-    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(w[i] << 16);
-      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  } else {
-    const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(base) + elem_off);
-    const float4 a = __ldg(p), b = __ldg(p + 1);
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-  }
+// 16-byte piece `piece` (0..7) of row `row` (0..31) inside a 128-byte-swizzled staging slice.
+__device__ __forceinline__ uint8_t* stg_addr(uint8_t* base, int row, int piece) {
+  return base + row * 128 + ((piece ^ (row & 7)) << 4);
 }
 
 template <int A_MN, int B_MN, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmX,
+            const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms of TMA and UMMA
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
-  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + p.stages * stage_bytes);
-  float* s_scale = reinterpret_cast<float*>(ctl + 1);   // [BN] (EPI_FWD)
-  float* s_bias = s_scale + 256;                         // [BN]
+  uint8_t* out_stg = smem + p.stages * stage_bytes;          // [4 warps][STG_BYTES]
+  uint8_t* x_stg = out_stg + 4 * STG_BYTES;                  // [4 warps][2][STG_BYTES]   (EPI_DX)
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? 8 * STG_BYTES : 0));
+  float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [4 warps][256] (EPI_FWD), warp-private
+  float* s_bias = s_scale + 4 * 256;                         // [4 warps][256]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * p.BN;
-  const int m0 = blockIdx.y * BM;
-  const int split = blockIdx.z;
-  const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
-  const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
-  // columns of this tile that exist, rounded up to the UMMA N granularity
-  int n_eff = static_cast<int>(p.Nc - n0);
-  if (n_eff > p.BN) n_eff = p.BN;
-  n_eff = (n_eff + 15) & ~15;
+  const int tiles_mn = p.tiles_m * p.tiles_n;
+  const int total_items = tiles_mn * p.splits;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&ctl->full[s], 1);
       mbar_init(&ctl->empty[s], 1);
     }
-    mbar_init(&ctl->acc_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&ctl->acc_full[b], 1);
+      mbar_init(&ctl->acc_empty[b], 4);
+    }
+    for (int w = 0; w < 4; ++w) {
+      mbar_init(&ctl->xbar[w][0], 1);
+      mbar_init(&ctl->xbar[w][1], 1);
+    }
     ctl->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
+    if (EPI != EPI_PART) prefetch_tmap(&tmOut);
+    if (EPI == EPI_DX) prefetch_tmap(&tmX);
   }
   if (warp == 1) {
-    tmem_alloc(&ctl->tmem_base, static_cast<uint32_t>(p.tmem_cols));
+    tmem_alloc(&ctl->tmem_base, TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -140,31 +124,40 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      const int b_chunks = (n_eff + 63) >> 6;
-      const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : p.BN * BK * 2);
       int it = 0;
-      for (int kb = kb_begin; kb < kb_end && !*abort_flag; ++kb, ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        if (!mbar_wait(&ctl->empty[s], ph ^ 1)) {
-          record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
-          *abort_flag = 1;
-          break;
-        }
-        uint8_t* sa = smem + s * stage_bytes;
-        uint8_t* sb = sa + A_STAGE_BYTES;
-        mbar_arrive_expect_tx(&ctl->full[s], tx);
-        if (A_MN) {
-          tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
-          tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
-        } else {
-          tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
-        }
-        if (B_MN) {
-          for (int c = 0; c < b_chunks; ++c)
-            tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
-        } else {
-          tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+      for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x) {
+        const int split = w / tiles_mn, t = w - split * tiles_mn;
+        const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * p.BN;
+        int n_eff = static_cast<int>(p.Nc - n0);
+        if (n_eff > p.BN) n_eff = p.BN;
+        n_eff = (n_eff + 15) & ~15;
+        const int b_chunks = (n_eff + 63) >> 6;
+        const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : p.BN * BK * 2);
+        const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
+        const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1;
+          if (*abort_flag || !mbar_wait(&ctl->empty[s], ph ^ 1)) {
+            record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
+            *abort_flag = 1;
+            break;
+          }
+          uint8_t* sa = smem + s * stage_bytes;
+          uint8_t* sb = sa + A_STAGE_BYTES;
+          mbar_arrive_expect_tx(&ctl->full[s], tx);
+          if (A_MN) {
+            tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
+            tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+          } else {
+            tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
+          }
+          if (B_MN) {
+            for (int c = 0; c < b_chunks; ++c)
+              tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
+          } else {
+            tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+          }
         }
       }
       // Make sure none of this CTA's bulk copies is still in flight when it exits (only
@@ -176,123 +169,227 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = instr_desc_bf16(BM, n_eff, A_MN, B_MN);
-      int it = 0;
+      int it = 0, acc_it = 0;
       bool ok = true;
-      for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        if (*abort_flag || !mbar_wait(&ctl->full[s], ph)) {
+      for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x, ++acc_it) {
+        const int split = w / tiles_mn, t = w - split * tiles_mn;
+        const int n0 = (t % p.tiles_n) * p.BN;
+        int n_eff = static_cast<int>(p.Nc - n0);
+        if (n_eff > p.BN) n_eff = p.BN;
+        n_eff = (n_eff + 15) & ~15;
+        const uint32_t idesc = instr_desc_bf16(BM, n_eff, A_MN, B_MN);
+        const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
+        const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
+        const int buf = acc_it & 1;
+        // wait until the epilogue has drained this accumulator (two tiles ago)
+        if (*abort_flag || !mbar_wait(&ctl->acc_empty[buf], ((acc_it >> 1) & 1) ^ 1)) {
           record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
           *abort_flag = 1;
           ok = false;
           break;
         }
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-        const uint32_t b_addr = a_addr + A_STAGE_BYTES;
+        const uint32_t d_tmem = tmem_base + buf * ACC_STRIDE;
+        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1;
+          if (*abort_flag || !mbar_wait(&ctl->full[s], ph)) {
+            record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
+            *abort_flag = 1;
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+          const uint32_t b_addr = a_addr + A_STAGE_BYTES;
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k) {
-          // K-major: 16 contraction elements = 32 bytes inside the swizzled 128-byte row.
-          // MN-major: 16 contraction elements = 16 rows of 128 bytes = two 8-row groups.
-          const uint64_t adesc = A_MN ? smem_desc_sw128(a_addr + k * 2048, CHUNK_BYTES, 1024)
-                                      : smem_desc_sw128(a_addr + k * 32, 16, 1024);
-          const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
-                                      : smem_desc_sw128(b_addr + k * 32, 16, 1024);
-          umma_bf16(tmem_base, adesc, bdesc, idesc, (it > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // K-major: 16 contraction elements = 32 bytes inside the swizzled 128-byte row.
+            // MN-major: 16 contraction elements = 16 rows of 128 bytes = two 8-row groups.
+            const uint64_t adesc = A_MN ? smem_desc_sw128(a_addr + k * 2048, CHUNK_BYTES, 1024)
+                                        : smem_desc_sw128(a_addr + k * 32, 16, 1024);
+            const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
+                                        : smem_desc_sw128(b_addr + k * 32, 16, 1024);
+            umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+          }
+          umma_commit(&ctl->empty[s]);   // frees the stage once these MMAs have read it
         }
-        umma_commit(&ctl->empty[s]);   // frees the stage once these MMAs have read it
+        if (ok) umma_commit(&ctl->acc_full[buf]);
       }
-      if (ok) umma_commit(&ctl->acc_full);
     }
   } else {
     // ------------------------------------------------------------- epilogue (warps 2..5)
     const int q = warp & 3;                  // TMEM lane quarter this warp may read
-    const int row_in_tile = q * 32 + lane;
-    const int64_t row = static_cast<int64_t>(m0) + row_in_tile;
-    const int et = threadIdx.x - 64;         // 0..127
-    if (EPI == EPI_FWD) {
-      for (int j = et; j < p.BN; j += 128) {
-        const int64_t c = static_cast<int64_t>(n0) + j;
-        s_scale[j] = (c < p.Nc) ? p.col_scale[c] : 0.f;
-        s_bias[j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
-      }
-      epi_bar_sync();
-    }
+    uint8_t* my_out = out_stg + q * STG_BYTES;
+    uint8_t* my_x = x_stg + q * 2 * STG_BYTES;
+    const int cc = p.chunk_cols;
     ActQ xq;
     if (EPI != EPI_PART) xq = *p.xq;
-    float acc_s = 0.f, acc_z = 0.f;
-    bool ok = mbar_wait(&ctl->acc_full, 0);
-    if (!ok) {
-      record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
-      *abort_flag = 1;
-    }
-    // all lanes of a warp see the same outcome of the wait, so the branch is warp-uniform
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    int acc_it = 0;
+    int x_it = 0;                            // X slices consumed so far by this warp (EPI_DX)
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x, ++acc_it) {
+      const int split = w / tiles_mn, t = w - split * tiles_mn;
+      const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * p.BN;
+      int n_eff = static_cast<int>(p.Nc - n0);
+      if (n_eff > p.BN) n_eff = p.BN;
+      n_eff = (n_eff + 15) & ~15;
+      const int buf = acc_it & 1;
+      const int row0 = m0 + q * 32;
+      if (EPI == EPI_FWD) {
+        // this warp's own copy of the tile's column scales and biases (no cross-warp barrier)
+        float* sc = s_scale + q * 256;
+        float* sb = s_bias + q * 256;
+        __syncwarp();
+        for (int j = lane; j < p.BN; j += 32) {
+          const int64_t c = static_cast<int64_t>(n0) + j;
+          sc[j] = (c < p.Nc) ? p.col_scale[c] : 0.f;
+          sb[j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
+        }
+        __syncwarp();
+      }
+      if (EPI == EPI_DX && lane == 0) {
+        // first X slice of this tile: in flight while the main loop of the tile finishes
+        uint64_t* xb = &ctl->xbar[q][x_it & 1];
+        mbar_arrive_expect_tx(xb, STG_BYTES);
+        tma_load_2d(my_x + (x_it & 1) * STG_BYTES, &tmX, xb, n0, row0);
+      }
+      bool got = *abort_flag ? false : mbar_wait(&ctl->acc_full[buf], (acc_it >> 1) & 1);
+      got = __all_sync(0xffffffffu, got);
+      if (!got) {
+        record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
+        *abort_flag = 1;
+        ok = false;
+        break;
+      }
       tc_fence_after();
-      for (int c0 = 0; c0 < n_eff; c0 += 32) {
-        uint32_t r[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c0);
-        const int ncols = (n_eff - c0 >= 32) ? 32 : 16;
-        if (ncols == 32) tmem_ld_32x32(taddr, r); else tmem_ld_32x16(taddr, r);
-        tmem_wait_ld();
-        if (EPI == EPI_PART) {
+      const uint32_t t_row = tmem_base + buf * ACC_STRIDE + (static_cast<uint32_t>(q * 32) << 16);
+      float acc_s = 0.f, acc_z = 0.f;
+
+      if (EPI == EPI_PART) {
+        const int64_t row = static_cast<int64_t>(row0) + lane;
+        for (int c0 = 0; c0 < n_eff; c0 += 32) {
+          uint32_t r[32];
+          const int ncols = (n_eff - c0 >= 32) ? 32 : 16;
+          if (ncols == 32) tmem_ld_32x32(t_row + c0, r); else tmem_ld_32x16(t_row + c0, r);
+          tmem_wait_ld();
           if (row < p.Mr) {
-            float* outp = static_cast<float*>(p.out) + split * p.split_stride + row;
+            float* outp = p.out + split * p.split_stride + row;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int64_t col = static_cast<int64_t>(n0) + c0 + j;
               if (j < ncols && col < p.part_cols) outp[col * p.ldo] = __uint_as_float(r[j]);
             }
           }
-        } else if (row < p.Mr) {
+        }
+      } else {
+        const float* sc = s_scale + q * 256;
+        const float* sb = s_bias + q * 256;
+        for (int c0 = 0; c0 < n_eff && ok; c0 += cc) {
+          uint8_t* xs = nullptr;
+          if (EPI == EPI_DX) {
+            const int xb_i = x_it & 1;
+            if (lane == 0 && c0 + cc < n_eff) {       // prefetch the next slice of this tile
+              uint64_t* xb = &ctl->xbar[q][xb_i ^ 1];
+              mbar_arrive_expect_tx(xb, STG_BYTES);
+              tma_load_2d(my_x + (xb_i ^ 1) * STG_BYTES, &tmX, xb, n0 + c0 + cc, row0);
+            }
+            bool gx = mbar_wait(&ctl->xbar[q][xb_i], (x_it >> 1) & 1);
+            gx = __all_sync(0xffffffffu, gx);
+            if (!gx) {
+              record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
+              *abort_flag = 1;
+              ok = false;
+              break;
+            }
+            xs = my_x + xb_i * STG_BYTES;
+            ++x_it;
+          }
+          // the previous TMA store must have finished reading the staging slice
+          if (lane == 0) tma_store_wait_read0();
+          __syncwarp();
+          for (int h = 0; h < cc; h += 32) {
+            const int left = n_eff - c0 - h;
+            if (left <= 0) break;
+            uint32_t r[32];
+            const int ncols = (left >= 32) ? 32 : 16;
+            if (ncols == 32) tmem_ld_32x32(t_row + c0 + h, r); else tmem_ld_32x16(t_row + c0 + h, r);
+            tmem_wait_ld();
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int64_t col = static_cast<int64_t>(n0) + c0 + g * 8;
-            if (g * 8 < ncols && col < p.Nc) {
-              float v[8];
-              if (EPI == EPI_FWD) {
+            for (int g = 0; g < 4; ++g) {
+              if (g * 8 < ncols) {
+                float v[8];
+                if (EPI == EPI_FWD) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                  v[j] = fmaf(__uint_as_float(r[g * 8 + j]) * xq.s, s_scale[c0 + g * 8 + j],
-                              s_bias[c0 + g * 8 + j]);
-              } else {
-                float x[8];
-                load8(p.X, row * p.ldo + col, x, p.x_dtype == EFQAT_BF16);
+                  for (int j = 0; j < 8; ++j) {
+                    const int cj = c0 + h + g * 8 + j;
+                    v[j] = fmaf(__uint_as_float(r[g * 8 + j]) * xq.s, sc[cj], sb[cj]);
+                  }
+                } else {
+                  float x[8];
+                  if (cc == 64) {      // bf16 activations: 8 values in one 16-byte piece
+                    const uint4 u = *reinterpret_cast<const uint4*>(stg_addr(xs, lane, (h >> 3) + g));
+                    const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float gx = __uint_as_float(r[g * 8 + j]);
-                  const QElem e = quant_act(x[j], xq);
-                  v[j] = e.flag ? 0.f : gx;
-                  acc_s = fmaf(gx, e.t, acc_s);
-                  acc_z += e.flag ? -gx * xq.s : 0.f;
+                    for (int i = 0; i < 4; ++i) {
+                      x[2 * i] = __uint_as_float(wv[i] << 16);
+                      x[2 * i + 1] = __uint_as_float(wv[i] & 0xffff0000u);
+                    }
+                  } else {             // fp32 activations: two 16-byte pieces
+                    const float4 a = *reinterpret_cast<const float4*>(stg_addr(xs, lane, 2 * g));
+                    const float4 b = *reinterpret_cast<const float4*>(stg_addr(xs, lane, 2 * g + 1));
+                    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+                    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+                  }
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    const float gx = __uint_as_float(r[g * 8 + j]);
+                    const QElem e = quant_act(x[j], xq);
+                    v[j] = e.flag ? 0.f : gx;
+                    acc_s = fmaf(gx, e.t, acc_s);
+                    acc_z += e.flag ? -gx * xq.s : 0.f;
+                  }
+                }
+                if (cc == 64) {
+                  uint4 o;
+                  o.x = pack2(v[0], v[1]); o.y = pack2(v[2], v[3]);
+                  o.z = pack2(v[4], v[5]); o.w = pack2(v[6], v[7]);
+                  *reinterpret_cast<uint4*>(stg_addr(my_out, lane, (h >> 3) + g)) = o;
+                } else {
+                  *reinterpret_cast<float4*>(stg_addr(my_out, lane, 2 * g)) = make_float4(v[0], v[1], v[2], v[3]);
+                  *reinterpret_cast<float4*>(stg_addr(my_out, lane, 2 * g + 1)) =
+                      make_float4(v[4], v[5], v[6], v[7]);
                 }
               }
-              store8(p.out, row * p.ldo + col, v, p.out_bf16);
             }
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0 && row0 < p.Mr && n0 + c0 < p.Nc) {
+            tma_store_2d(&tmOut, my_out, n0 + c0, row0);   // clipped at the tensor's edges
+            tma_store_commit();
           }
         }
       }
-    }
-    if (EPI == EPI_DX) {
-      acc_s = warp_sum(acc_s);
-      acc_z = warp_sum(acc_z);
-      if (lane == 0) {
-        ctl->red[q][0] = acc_s;
-        ctl->red[q][1] = acc_z;
+      // every TMEM read of this accumulator is complete: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctl->acc_empty[buf]);
+      if (EPI == EPI_DX && ok) {
+        acc_s = warp_sum(acc_s);
+        acc_z = warp_sum(acc_z);
+        if (lane == 0) {
+          float* pp = p.partials + (static_cast<int64_t>(t) * 4 + q) * 2;
+          pp[0] = acc_s;
+          pp[1] = acc_z;
+        }
       }
-      epi_bar_sync();
-      if (et == 0) {
-        const int64_t tile = static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x;
-        p.partials[2 * tile] = (ctl->red[0][0] + ctl->red[1][0]) + (ctl->red[2][0] + ctl->red[3][0]);
-        p.partials[2 * tile + 1] = (ctl->red[0][1] + ctl->red[1][1]) + (ctl->red[2][1] + ctl->red[3][1]);
-      }
     }
+    if (EPI != EPI_PART && lane == 0) tma_store_wait_all();
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 // ------------------------------------------------------------------ host side
@@ -312,25 +409,30 @@ int gemm_init() {
   return EFQAT_OK;
 }
 
-// 2-D bf16 row-major matrix [rows, cols] with pitch ld (elements); box = 64 columns x box_rows rows.
-static int make_map(CUtensorMap* m, const bf16* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+// 2-D row-major matrix [rows, cols] with pitch ld (elements); box = 128 bytes of columns x box_rows rows.
+static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
+                    int box_rows) {
+  const int es = is_bf16 ? 2 : 4;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
-  const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
-  const cuuint32_t es[2] = {1u, 1u};
-  const CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(base), dims, strides, box,
-                              es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * es};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / es), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1u, 1u};
+  const CUresult r = g_encode(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
-static int choose_bn(int64_t Mr, int64_t Nc, int splits, int sm_count) {
-  if (Nc <= 64) return static_cast<int>(round_up(Nc, 16));
+// Tile width for the forward / grad-input GEMMs: multiples of 64 so that every 128-byte
+// staging row of the epilogue lies inside one tile.
+static int choose_bn(int64_t Mr, int64_t Nc, int sm_count) {
+  if (Nc <= 64) return 64;
   const int64_t mt = ceil_div(Mr, BM);
   int best = 64;
   double best_cost = 1e300;
-  for (int bn = 256; bn >= 64; bn -= 32) {
-    const int64_t tiles = mt * ceil_div(Nc, bn) * splits;
+  for (int bn = 256; bn >= 64; bn -= 64) {
+    const int64_t tiles = mt * ceil_div(Nc, bn);
     const double cost = static_cast<double>(ceil_div(tiles, sm_count)) * (bn + 24);
     if (cost < best_cost) {
       best_cost = cost;
@@ -341,14 +443,17 @@ static int choose_bn(int64_t Mr, int64_t Nc, int splits, int sm_count) {
 }
 
 int gemm_dx_num_partials(int64_t Mr, int64_t Nc) {
-  // upper bound over every tile width the heuristic may pick
-  return static_cast<int>(ceil_div(Mr, BM) * ceil_div(Nc, 64));
+  // upper bound over every tile width the heuristic may pick: 4 quarter-warps per tile
+  return static_cast<int>(ceil_div(Mr, BM) * ceil_div(Nc, 64) * 4);
+}
+
+static int part_bn(int64_t Nc) {
+  return (Nc <= 64) ? static_cast<int>(round_up(Nc, 16)) : (Nc <= 128 ? 128 : 256);
 }
 
 int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
   const int64_t nkb = ceil_div(Kc, BK);
-  const int bn = (Nc <= 64) ? static_cast<int>(round_up(Nc, 16)) : (Nc <= 128 ? 128 : 256);
-  const int64_t tiles = ceil_div(Mr, BM) * ceil_div(Nc, bn);
+  const int64_t tiles = ceil_div(Mr, BM) * ceil_div(Nc, part_bn(Nc));
   int64_t s = ceil_div(sm_count, tiles);
   const int64_t max_s = nkb / 4 > 0 ? nkb / 4 : 1;   // at least four contraction blocks per split
   if (s > max_s) s = max_s;
@@ -358,8 +463,8 @@ int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
 }
 
 template <int A_MN, int B_MN, int EPI>
-static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, dim3 grid, size_t smem,
-                  cudaStream_t st) {
+static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const CUtensorMap& tx,
+                  const GemmParams& p, int grid, size_t smem, cudaStream_t st) {
   auto kern = gemm_kernel<A_MN, B_MN, EPI>;
   static bool configured[64] = {};   // per instantiation and device
   int dev = 0;
@@ -371,7 +476,7 @@ static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams
     configured[dev] = true;
   }
   count_launches(1);
-  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, p);
+  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, to, tx, p);
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
@@ -385,47 +490,52 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.nkb = static_cast<int>(ceil_div(a.Kc, BK));
   p.splits = (a.epi == EPI_PART) ? a.splits : 1;
   if (p.splits < 1 || p.splits > p.nkb) return EFQAT_ERR_SHAPE;
-  if (a.epi == EPI_PART) {
-    p.BN = (a.Nc <= 64) ? static_cast<int>(round_up(a.Nc, 16)) : (a.Nc <= 128 ? 128 : 256);
-  } else {
-    p.BN = choose_bn(a.Mr, a.Nc, 1, sm_count);
-  }
+  p.BN = (a.epi == EPI_PART) ? part_bn(a.Nc) : choose_bn(a.Mr, a.Nc, sm_count);
+  p.tiles_m = static_cast<int>(ceil_div(a.Mr, BM));
+  p.tiles_n = static_cast<int>(ceil_div(a.Nc, p.BN));
+  p.chunk_cols = a.out_bf16 ? 64 : 32;
   p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(p.BN, 64) * CHUNK_BYTES : p.BN * BK * 2);
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
   const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
-  const int ctl_bytes = static_cast<int>(sizeof(SmemCtl)) + 2 * 256 * 4;
-  int stages = (227 * 1024 - 1024 - ctl_bytes) / stage_bytes;
+  const int fixed_bytes = 4 * STG_BYTES + (a.epi == EPI_DX ? 8 * STG_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
+                          (a.epi == EPI_FWD ? 2 * 4 * 256 * 4 : 0);
+  int stages = (227 * 1024 - 1024 - fixed_bytes) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return EFQAT_ERR_SHAPE;
   p.stages = stages;
-  int cols = 32;
-  while (cols < p.BN) cols <<= 1;
-  p.tmem_cols = cols;
-  p.out_bf16 = a.out_bf16;
-  p.out = a.out;
-  p.ldo = a.ldo;
   p.col_scale = a.col_scale;
   p.col_bias = a.col_bias;
   p.xq = a.xq;
-  p.X = a.X;
-  p.x_dtype = a.x_dtype;
   p.partials = a.partials;
+  p.out = static_cast<float*>(a.out);
+  p.ldo = a.ldo;
   p.split_stride = a.split_stride;
   p.part_cols = a.part_cols;
   p.status = a.status;
 
-  CUtensorMap ta, tb;
-  rc = a.a_mn ? make_map(&ta, a.A, a.Kc, a.Mr, a.lda, BK) : make_map(&ta, a.A, a.Mr, a.Kc, a.lda, BM);
+  CUtensorMap ta, tb, to, tx;
+  rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
   if (rc != EFQAT_OK) return rc;
-  rc = a.b_mn ? make_map(&tb, a.B, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, a.Nc, a.Kc, a.ldb, p.BN);
+  rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, p.BN);
   if (rc != EFQAT_OK) return rc;
+  to = ta;
+  tx = ta;
+  if (a.epi != EPI_PART) {
+    rc = make_map(&to, a.out, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+    if (rc != EFQAT_OK) return rc;
+  }
+  if (a.epi == EPI_DX) {
+    if ((a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;
+    rc = make_map(&tx, a.X, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+    if (rc != EFQAT_OK) return rc;
+  }
 
-  const dim3 grid(static_cast<unsigned>(ceil_div(a.Nc, p.BN)), static_cast<unsigned>(ceil_div(a.Mr, BM)),
-                  static_cast<unsigned>(p.splits));
-  const size_t smem = static_cast<size_t>(stages) * stage_bytes + ctl_bytes + 1024;
-  if (tiles_out) *tiles_out = static_cast<int>(grid.x * grid.y);
+  const int64_t items = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
+  const int grid = static_cast<int>(items < sm_count ? items : sm_count);
+  const size_t smem = static_cast<size_t>(stages) * stage_bytes + fixed_bytes + 1024;
+  if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * 4;
 
-#define EFQAT_LAUNCH(AM, BMj, E) return launch<AM, BMj, E>(ta, tb, p, grid, smem, st)
+#define EFQAT_LAUNCH(AM, BMj, E) return launch<AM, BMj, E>(ta, tb, to, tx, p, grid, smem, st)
   if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) EFQAT_LAUNCH(0, 0, EPI_FWD);
   if (a.epi == EPI_DX && !a.a_mn && a.b_mn) EFQAT_LAUNCH(0, 1, EPI_DX);
   if (a.epi == EPI_PART && a.a_mn && a.b_mn) EFQAT_LAUNCH(1, 1, EPI_PART);

@@ -1,0 +1,98 @@
+"""Full-size parity: the benchmark's own workload (BERT-base-shaped linears at M = 4096),
+in the launch configuration bench.py times, compared element by element with the oracle;
+and a larger GEMM shape checked on sampled rows / channels plus size-independent properties."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import efqat_oracle as O
+from paper_2411_11038_b200 import binding as B
+from paper_2411_11038_b200 import inputs as I
+from tests import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    return B.Context(0)
+
+
+@pytest.mark.parametrize("li", [0, 1, 2, 3])
+def test_config2_layer_full_size(ctx, li):
+    case = I.config2()[li]
+    T = I.make_tensors(case)
+    s_w, s_x, z_x = U.oracle_qparams(case, T, (0.8, 0.85, 1.4))
+    D = U.to_dev(T, s_w, s_x, z_x)
+    U.check_forward(ctx, case, T, D, s_w, s_x, z_x)
+    k = B.ratio_to_k(0.05, case.N)
+    sel, _, _ = B.select_channels(ctx, B.CWPL, [D["W"]], [k])
+    idx = sel[0].cpu().numpy()
+    assert idx.tolist() == O.select_cwpl([T["W"].numpy()], [k])[0].tolist()
+    U.check_backward(ctx, case, T, D, s_w, s_x, z_x, idx)
+
+
+def test_config2_full_qat_backward(ctx):
+    case = I.config2()[1]
+    T = I.make_tensors(case)
+    s_w, s_x, z_x = U.oracle_qparams(case, T)
+    D = U.to_dev(T, s_w, s_x, z_x)
+    U.check_backward(ctx, case, T, D, s_w, s_x, z_x, np.arange(case.N, dtype=np.int32))
+
+
+def test_large_shape_sampled(ctx):
+    """M = 16384, K = N = 4096 (GEMM-sweep family): sampled rows of Y and dX, sampled selected
+    channels of dW, and the invariants that hold at any size."""
+    case = I.config5()[1]
+    T = I.make_tensors(case)
+    X64, W64, dY64 = (I.as_f64(T[k]) for k in ("X", "W", "dY"))
+    s_w = O.init_minmax_w(W64, case.w_bits)
+    s_x, z_x = O.init_minmax_x(X64, case.x_bits, False)
+    D = U.to_dev(T, s_w, s_x, z_x)
+    # MinMax initialisation on the device agrees exactly
+    assert np.array_equal(B.init_weight_scales(ctx, D["W"], 8).cpu().numpy(), s_w)
+    ds, dz = B.init_act_qparams(ctx, D["X"], 8, False)
+    assert ds.item() == float(s_x) and dz.item() == float(z_x)
+    k = B.ratio_to_k(0.05, case.N)
+    sel, _, _ = B.select_channels(ctx, B.CWPL, [D["W"]], [k])
+    idx = sel[0].cpu().numpy()
+    assert idx.tolist() == O.select_cwpl([T["W"].numpy()], [k])[0].tolist()
+
+    plan = B.LayerPlan(ctx, case.M, case.N, case.K, case.act_dtype, 8, 8, False, case.N, "cuda")
+    Y = plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"]).float().cpu().numpy()
+    out = plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], sel[0], k)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    dX = out["dX"].float().cpu().numpy()
+    dW = out["dW_sel"].cpu().numpy().copy()
+    dSx, dZx = out["dS_x"].item(), out["dZ_x"].item()
+
+    rng = np.random.default_rng(0)
+    rows = np.sort(rng.choice(case.M, 64, replace=False))
+    rows[0], rows[-1] = 0, case.M - 1
+    b64 = I.as_f64(T["bias"])
+    Yr = O.forward(X64[rows], W64, s_w, s_x, z_x, b64, 8, 8)
+    U.assert_bf16_class(Y[rows], Yr, "Y rows")
+    ref = O.backward_full(dY64[rows], X64[rows], W64, s_w, s_x, z_x, 8, 8, operand_model="bf16")
+    U.assert_fp32_class(dX[rows], ref["dX"], ref["G_x_abs"], "dX rows", out_is_bf16=True)
+    ex = O.backward_full(dY64[rows], X64[rows], W64, s_w, s_x, z_x, 8, 8)
+    U.assert_bf16_class(dX[rows], ex["dX"], "dX rows")
+    pick = np.sort(rng.choice(k, 16, replace=False))
+    d = O.backward_efqat_direct(dY64, X64, W64, s_w, s_x, z_x, idx[pick], 8, 8)
+    U.assert_bf16_class(dW[pick], d["dW_sel"], "dW_sel rows")
+    assert np.abs(dW[pick] - d["dW_sel"]).max() <= 1e-4 * np.abs(d["dW_sel"]).max()
+    np.testing.assert_allclose(out["dS_w_sel"].cpu().numpy()[pick], d["dS_w_sel"], rtol=2e-3, atol=1e-2)
+    np.testing.assert_allclose(out["db"].cpu().numpy(), dY64.sum(axis=0), rtol=0,
+                               atol=1e-5 * np.abs(dY64).sum(axis=0).max())
+    # properties at full size: dX, dS_x, dZ_x do not depend on the selection; a second
+    # selection returns the same rows for the channels both contain
+    idx2 = np.arange(0, case.N, 16, dtype=np.int32)
+    out2 = plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], torch.from_numpy(idx2).cuda(), len(idx2))
+    torch.cuda.synchronize()
+    assert np.array_equal(out2["dX"].float().cpu().numpy(), dX)
+    assert out2["dS_x"].item() == dSx and out2["dZ_x"].item() == dZx
+    common = np.intersect1d(idx, idx2)
+    if len(common):
+        a = dW[np.searchsorted(idx, common)]
+        b = out2["dW_sel"].cpu().numpy()[np.searchsorted(idx2, common)]
+        assert np.abs(a - b).max() <= 1e-5 * np.abs(a).max()

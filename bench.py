@@ -236,8 +236,7 @@ def oracle_step_seconds(frac, layers=None, rows=None):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     frac = args.frac
     layers, rows = [1], 1024    # bounded sample: 1024 tokens of the 768 -> 768 attention-output layer
@@ -263,31 +262,15 @@ def run_reference(args):
 
 def run_ours(args):
     from paper_2411_11038_b200 import binding as B
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2411_11038_b200.replicas import Replicas, env_ranks
+    rank, local, world = env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    def max_over_ranks(v):
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    reps = Replicas(backend="nccl", device=dev)       # replicas only: no data-path collective
+    sync_all = reps.barrier
+    max_over_ranks = reps.max_over_ranks
 
     ctx = B.Context(local)
     wl = Workload(ctx, dev)
@@ -380,8 +363,7 @@ def run_ours(args):
             "device_status": status,
             "paper_context": "paper reports 1.44-1.64x backward speed-up on A10/A100 (whole network)",
         }))
-    if dist is not None:
-        dist.destroy_process_group()
+    reps.close()
 
 
 def main():

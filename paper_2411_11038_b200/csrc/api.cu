@@ -300,9 +300,14 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   const int64_t M = layer->M, N = layer->N, K = layer->K;
   cudaStream_t st = stream;
 
-  launch_prep_act(s_x, z_x, q->x_bits, q->x_symmetric, w.actq, ctx->d_status, st);
-  launch_quant_act_operand(X, layer->act_dtype, M * K, w.actq, w.Xc, st);
-  launch_quant_weight_operand(W, N, K, s_w, q->w_bits, 0, w.Wq, ctx->d_status, st);
+  const int act_bf16 = layer->act_dtype == EFQAT_BF16;
+  // a2: both quantizers in one launch
+  PrepArgs pa = {};
+  pa.M = M; pa.N = N; pa.K = K;
+  pa.W = W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
+  pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric; pa.Xc = w.Xc;
+  pa.status = ctx->d_status;
+  launch_prepare(pa, 0, act_bf16, st);
   GemmArgs g = {};
   g.A = w.Xc; g.B = w.Wq;
   g.Mr = M; g.Nc = N; g.Kc = K;
@@ -312,7 +317,7 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   g.out_bf16 = layer->act_dtype == EFQAT_BF16;
   g.out = Y; g.ldo = N;
   g.col_scale = s_w; g.col_bias = bias_or_null;
-  g.xq = w.actq;
+  g.s_x = s_x; g.z_x = z_x; g.x_bits = q->x_bits; g.x_sym = q->x_symmetric;
   g.status = ctx->d_status;
   rc = timed_gemm(ctx, 0, g, st);
   if (rc != EFQAT_OK) return rc;
@@ -333,6 +338,9 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   if (k_sel > 0 && (!dW_sel || !dS_w_sel)) return EFQAT_ERR_NULL;
   if (k_sel > 0 && k_sel < N && !idx) return EFQAT_ERR_NULL;
   if (opt_or_null && k_sel > 0 && (!opt_or_null->W_inout || !opt_or_null->mom_inout)) return EFQAT_ERR_NULL;
+  if (opt_or_null && k_sel > 0 && (!aligned16(opt_or_null->W_inout) || !aligned16(opt_or_null->mom_inout)))
+    return EFQAT_ERR_ALIGN;
+  if (dS_w_sel == nullptr && k_sel > 0) return EFQAT_ERR_NULL;
   if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(dX) || (dW_sel && !aligned16(dW_sel)))
     return EFQAT_ERR_ALIGN;
   if (!ws) return EFQAT_ERR_WORKSPACE;
@@ -343,15 +351,22 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   cudaStream_t st = stream;
   const int act_bf16 = layer->act_dtype == EFQAT_BF16;
 
-  // a2: quantizer parameters, dequantised weight operand, bf16 view of dY
-  launch_prep_act(s_x, z_x, q->x_bits, q->x_symmetric, w.actq, ctx->d_status, st);
-  launch_quant_weight_operand(W, N, K, s_w, q->w_bits, 1, w.Wq, ctx->d_status, st);
-  const bf16* dYb = static_cast<const bf16*>(dY);
-  if (!act_bf16) {
-    launch_to_bf16(static_cast<const float*>(dY), M * N, w.dYb, st);
-    dYb = w.dYb;
-  }
+  const bool gathered = k_sel > 0 && k_sel < N;
+  // a2: one launch: dequantised weight operand, activation codes (only when some channel is
+  // unfrozen) and one pass over dY (column-sum partials, gathered columns, bf16 copy)
+  const bf16* dYb = act_bf16 ? static_cast<const bf16*>(dY) : w.dYb;
+  PrepArgs pa = {};
+  pa.M = M; pa.N = N; pa.K = K;
+  pa.W = W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
+  pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric;
+  pa.Xc = k_sel > 0 ? w.Xc : nullptr;
+  pa.dY = dY; pa.dYb = act_bf16 ? nullptr : w.dYb;
+  pa.colsum_ws = db_or_null ? w.colsum : nullptr;
+  pa.idx = idx; pa.k_sel = k_sel; pa.pitch = w.pitch; pa.dYsel = gathered ? w.dYsel : nullptr;
+  pa.status = ctx->d_status;
+  launch_prepare(pa, 1, act_bf16, st);
   // a4 + a5: dX = (dY W^) masked, with the dS_x / dZ_x partial sums in the epilogue
+  int tiles = 0;
   {
     GemmArgs g = {};
     g.A = dYb; g.B = w.Wq;
@@ -361,32 +376,20 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.epi = EPI_DX;
     g.out_bf16 = act_bf16;
     g.out = dX; g.ldo = K;
-    g.xq = w.actq;
+    g.s_x = s_x; g.z_x = z_x; g.x_bits = q->x_bits; g.x_sym = q->x_symmetric;
     g.X = X; g.x_dtype = layer->act_dtype;
     g.partials = w.dxpart;
     g.status = ctx->d_status;
-    int tiles = 0;
     rc = timed_gemm(ctx, 1, g, st, &tiles);
     if (rc != EFQAT_OK) return rc;
-    launch_dx_finalize(w.dxpart, tiles, dS_x, dZ_x, st);
   }
-  if (db_or_null) launch_colsum(dY, layer->act_dtype, M, N, w.colsum, db_or_null, st);
-  // a6 (+ a7): weight gradient of the unfrozen channels only
+  // a6: weight gradient of the unfrozen channels only, as split partial products
   if (k_sel > 0) {
-    launch_quant_act_operand(X, layer->act_dtype, M * K, w.actq, w.Xc, st);
-    const bool gathered = k_sel < N;
-    const bf16* Bop = dYb;
-    int64_t ldb = N, nc = N;
-    if (gathered) {
-      launch_gather_cols(dY, layer->act_dtype, M, N, idx, k_sel, w.pitch, w.dYsel, ctx->d_status, st);
-      Bop = w.dYsel;
-      ldb = w.pitch;
-      nc = round_up(k_sel, 16);
-    }
     GemmArgs g = {};
-    g.A = w.Xc; g.B = Bop;           // D[k, i] = sum_m Xc[m,k] * dYsel[m,i]
-    g.Mr = K; g.Nc = nc; g.Kc = M;
-    g.lda = K; g.ldb = ldb;
+    g.A = w.Xc;                       // D[k, i] = sum_m Xc[m,k] * dYsel[m,i]
+    g.B = gathered ? w.dYsel : dYb;
+    g.Mr = K; g.Nc = gathered ? round_up(k_sel, 16) : N; g.Kc = M;
+    g.lda = K; g.ldb = gathered ? w.pitch : N;
     g.a_mn = 1; g.b_mn = 1;
     g.epi = EPI_PART;
     g.out = w.P; g.ldo = K;
@@ -396,9 +399,20 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.status = ctx->d_status;
     rc = timed_gemm(ctx, 2, g, st);
     if (rc != EFQAT_OK) return rc;
-    launch_dw_finalize(w.P, w.splits, k_sel * K, k_sel, N, K, W, s_w, gathered ? idx : nullptr, w.actq,
-                       q->w_bits, dW_sel, dS_w_sel, opt_or_null, ctx->d_status, st);
   }
+  // a5 (+ a7): one launch: dW rows (mask, dS_w, optional SGD), dS_x / dZ_x, db
+  FinArgs fa = {};
+  fa.N = N; fa.K = K; fa.k_sel = k_sel;
+  fa.P = w.P; fa.splits = w.splits; fa.split_stride = k_sel * K;
+  fa.W = W; fa.s_w = s_w; fa.s_x = s_x; fa.w_bits = q->w_bits;
+  fa.idx = gathered ? idx : nullptr;
+  fa.dW_sel = dW_sel; fa.dS_w_sel = dS_w_sel;
+  if (opt_or_null) fa.opt = *opt_or_null;
+  fa.has_opt = opt_or_null != nullptr;
+  fa.dx_partials = w.dxpart; fa.n_partials = tiles; fa.dS_x = dS_x; fa.dZ_x = dZ_x;
+  fa.colsum_ws = w.colsum; fa.slabs = prepare_slabs(M); fa.db = db_or_null;
+  fa.status = ctx->d_status;
+  launch_finalize(fa, st);
   return last_error();
 }
 

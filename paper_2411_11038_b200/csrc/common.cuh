@@ -51,6 +51,33 @@ __device__ __forceinline__ QElem quant_act(float x, const ActQ& p) {
   return e;
 }
 
+// Derived activation-quantizer constants from the learnable scale / zero point.  A scale
+// that is not positive and finite is replaced by 1 (and reported through *bad).
+__device__ __forceinline__ ActQ make_actq(const float* __restrict__ s_x, const float* __restrict__ z_x,
+                                          int x_bits, int x_sym, bool* bad) {
+  ActQ p;
+  float s = s_x[0];
+  const bool ok = s > 0.f && isfinite(s);
+  if (bad) *bad = !ok;
+  if (!ok) s = 1.f;
+  p.s = s;
+  const double inv = 1.0 / static_cast<double>(s);
+  p.rinv = static_cast<float>(inv);
+  p.rinv_lo = static_cast<float>(inv - static_cast<double>(p.rinv));
+  if (x_sym) {
+    const float qs = static_cast<float>((1 << (x_bits - 1)) - 1);
+    p.lo = -qs;
+    p.hi = qs;
+    p.zr = 0.f;
+  } else {
+    p.lo = 0.f;
+    p.hi = static_cast<float>((1 << x_bits) - 1);
+    p.zr = fminf(fmaxf(rintf(z_x[0]), p.lo), p.hi);
+  }
+  p.pad0 = p.pad1 = 0.f;
+  return p;
+}
+
 struct RowQ {
   float s, rinv, rinv_lo, qmax;
 };

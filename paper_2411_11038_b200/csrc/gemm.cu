@@ -11,6 +11,10 @@
 //                    each warp reads its 32-lane quarter of the accumulator, fetches its slice
 //                    of X with TMA (EPI_DX) and writes its slice of the output with TMA stores
 //                    from a swizzled staging buffer, so global traffic is in whole 128-byte rows
+// With CTA2 = 1 two CTAs of a cluster work as a pair on a 256 x BN tile (tcgen05 cta_group::2):
+// each CTA stages its own 128 rows of A and one half of the B tile, the leader CTA issues the
+// MMAs for both, and every CTA runs the epilogue of its own 128 rows.  This halves the B
+// traffic from L2 per FLOP, which is what bounds the one-CTA tiles.  No TMA multicast is used.
 // Either operand may be stored with the contraction dimension contiguous ("K-major") or
 // with the other dimension contiguous ("MN-major"); the shared-memory and instruction
 // descriptors carry the difference, so no transposed copies are ever made.
@@ -43,7 +47,7 @@ struct GemmParams {
   int chunk_cols;     // output columns per 128-byte staging row: 64 (bf16) or 32 (fp32)
   const float* col_scale;
   const float* col_bias;
-  const ActQ* xq;
+  const float* s_x; const float* z_x; int x_bits, x_sym;
   float* partials;    // EPI_DX: [tile][quarter][2]
   float* out;         // EPI_PART
   int64_t ldo;
@@ -72,7 +76,7 @@ __device__ __forceinline__ uint8_t* stg_addr(uint8_t* base, int row, int piece) 
   return base + row * 128 + ((piece ^ (row & 7)) << 4);
 }
 
-template <int A_MN, int B_MN, int EPI>
+template <int A_MN, int B_MN, int EPI, int CTA2>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmX,
@@ -90,6 +94,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_mn = p.tiles_m * p.tiles_n;
   const int total_items = tiles_mn * p.splits;
+  // CTA pair bookkeeping: `rank` inside the pair, `unit` = index of this CTA / pair in the grid
+  const int rank = CTA2 ? static_cast<int>(cluster_ctarank()) : 0;
+  const int unit = CTA2 ? (blockIdx.x >> 1) : blockIdx.x;
+  const int num_units = CTA2 ? (gridDim.x >> 1) : gridDim.x;
+  const int TILE_M = CTA2 ? 2 * BM : BM;
+  const int bn_cta = CTA2 ? (p.BN >> 1) : p.BN;     // B columns staged by this CTA
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -98,7 +108,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&ctl->acc_full[b], 1);
-      mbar_init(&ctl->acc_empty[b], 4);
+      mbar_init(&ctl->acc_empty[b], CTA2 ? 8 : 4);
     }
     for (int w = 0; w < 4; ++w) {
       mbar_init(&ctl->xbar[w][0], 1);
@@ -112,11 +122,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (EPI == EPI_DX) prefetch_tmap(&tmX);
   }
   if (warp == 1) {
-    tmem_alloc(&ctl->tmem_base, TMEM_COLS);
-    tmem_relinquish();
+    if (CTA2) {
+      tmem_alloc_pair(&ctl->tmem_base, TMEM_COLS);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(&ctl->tmem_base, TMEM_COLS);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CTA2) cluster_sync();     // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   volatile int* abort_flag = &ctl->abort_flag;
@@ -125,14 +141,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
       int it = 0;
-      for (int w = blockIdx.x; w < total_items && !*abort_flag; w += gridDim.x) {
+      for (int w = unit; w < total_items && !*abort_flag; w += num_units) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
-        const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * p.BN;
+        const int m0 = (t / p.tiles_n) * TILE_M + rank * BM;
+        const int n0 = (t % p.tiles_n) * p.BN + rank * bn_cta;     // first B column staged by this CTA
         int n_eff = static_cast<int>(p.Nc - n0);
-        if (n_eff > p.BN) n_eff = p.BN;
+        if (n_eff > bn_cta) n_eff = bn_cta;
         n_eff = (n_eff + 15) & ~15;
         const int b_chunks = (n_eff + 63) >> 6;
-        const uint32_t tx = A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : p.BN * BK * 2);
+        // bytes credited to the (leader's) full barrier per stage: both CTAs' copies in pair mode
+        const uint32_t tx = (CTA2 ? 2u : 1u) * (A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : bn_cta * BK * 2));
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
         for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
@@ -145,39 +163,58 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           uint8_t* sa = smem + s * stage_bytes;
           uint8_t* sb = sa + A_STAGE_BYTES;
-          mbar_arrive_expect_tx(&ctl->full[s], tx);
-          if (A_MN) {
-            tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
-            tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+          if (CTA2) {
+            // the leader's barrier collects the bytes of both CTAs; only the leader arrives on it
+            const uint32_t fb = mapa_u32(smem_u32(&ctl->full[s]), 0);
+            if (rank == 0) mbar_arrive_expect_tx(&ctl->full[s], tx);
+            if (A_MN) {
+              tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
+              tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
+            } else {
+              tma_load_2d_pair(sa, &tmA, fb, kb * BK, m0);
+            }
+            if (B_MN) {
+              for (int c = 0; c < b_chunks; ++c)
+                tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
+            } else {
+              tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
+            }
           } else {
-            tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
-          }
-          if (B_MN) {
-            for (int c = 0; c < b_chunks; ++c)
-              tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
-          } else {
-            tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+            mbar_arrive_expect_tx(&ctl->full[s], tx);
+            if (A_MN) {
+              tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
+              tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+            } else {
+              tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
+            }
+            if (B_MN) {
+              for (int c = 0; c < b_chunks; ++c)
+                tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
+            } else {
+              tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+            }
           }
         }
       }
       // Make sure none of this CTA's bulk copies is still in flight when it exits (only
       // relevant after an abort: otherwise the MMA warp has consumed every stage).
       const int issued = it;
-      for (int j = (issued > p.stages ? issued - p.stages : 0); j < issued; ++j)
-        mbar_wait(&ctl->full[j % p.stages], (j / p.stages) & 1, 20000000ull);
+      if (rank == 0)
+        for (int j = (issued > p.stages ? issued - p.stages : 0); j < issued; ++j)
+          mbar_wait(&ctl->full[j % p.stages], (j / p.stages) & 1, 20000000ull);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       int it = 0, acc_it = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x, ++acc_it) {
+      for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
         const int n0 = (t % p.tiles_n) * p.BN;
         int n_eff = static_cast<int>(p.Nc - n0);
         if (n_eff > p.BN) n_eff = p.BN;
         n_eff = (n_eff + 15) & ~15;
-        const uint32_t idesc = instr_desc_bf16(BM, n_eff, A_MN, B_MN);
+        const uint32_t idesc = instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
         const int buf = acc_it & 1;
@@ -210,11 +247,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                         : smem_desc_sw128(a_addr + k * 32, 16, 1024);
             const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
                                         : smem_desc_sw128(b_addr + k * 32, 16, 1024);
-            umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            if (CTA2) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            else umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
           }
-          umma_commit(&ctl->empty[s]);   // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (CTA2) umma_commit_pair(&ctl->empty[s], 3); else umma_commit(&ctl->empty[s]);
         }
-        if (ok) umma_commit(&ctl->acc_full[buf]);
+        if (ok) {
+          if (CTA2) umma_commit_pair(&ctl->acc_full[buf], 3); else umma_commit(&ctl->acc_full[buf]);
+        }
       }
     }
   } else {
@@ -223,14 +264,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint8_t* my_out = out_stg + q * STG_BYTES;
     uint8_t* my_x = x_stg + q * 2 * STG_BYTES;
     const int cc = p.chunk_cols;
-    ActQ xq;
-    if (EPI != EPI_PART) xq = *p.xq;
+    ActQ xq = {};
+    if (EPI != EPI_PART) xq = make_actq(p.s_x, p.z_x, p.x_bits, p.x_sym, nullptr);
     int acc_it = 0;
     int x_it = 0;                            // X slices consumed so far by this warp (EPI_DX)
     bool ok = true;
-    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x, ++acc_it) {
+    for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
       const int split = w / tiles_mn, t = w - split * tiles_mn;
-      const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * p.BN;
+      const int m0 = (t / p.tiles_n) * TILE_M + rank * BM, n0 = (t % p.tiles_n) * p.BN;
       int n_eff = static_cast<int>(p.Nc - n0);
       if (n_eff > p.BN) n_eff = p.BN;
       n_eff = (n_eff + 15) & ~15;
@@ -374,12 +415,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // every TMEM read of this accumulator is complete: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&ctl->acc_empty[buf]);
+      if (lane == 0) {
+        if (CTA2) mbar_arrive_cluster(mapa_u32(smem_u32(&ctl->acc_empty[buf]), 0));   // leader's barrier
+        else mbar_arrive(&ctl->acc_empty[buf]);
+      }
       if (EPI == EPI_DX && ok) {
         acc_s = warp_sum(acc_s);
         acc_z = warp_sum(acc_z);
         if (lane == 0) {
-          float* pp = p.partials + (static_cast<int64_t>(t) * 4 + q) * 2;
+          float* pp = p.partials + ((static_cast<int64_t>(t) * (CTA2 ? 2 : 1) + rank) * 4 + q) * 2;
           pp[0] = acc_s;
           pp[1] = acc_z;
         }
@@ -389,7 +433,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+  if (CTA2) cluster_sync();     // neither CTA leaves while its peer may still signal its barriers
+  if (warp == 1) {
+    if (CTA2) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
+  }
 }
 
 // ------------------------------------------------------------------ host side
@@ -462,10 +509,10 @@ int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
   return static_cast<int>(s);
 }
 
-template <int A_MN, int B_MN, int EPI>
+template <int A_MN, int B_MN, int EPI, int CTA2>
 static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const CUtensorMap& tx,
                   const GemmParams& p, int grid, size_t smem, cudaStream_t st) {
-  auto kern = gemm_kernel<A_MN, B_MN, EPI>;
+  auto kern = gemm_kernel<A_MN, B_MN, EPI, CTA2>;
   static bool configured[64] = {};   // per instantiation and device
   int dev = 0;
   cudaGetDevice(&dev);
@@ -476,7 +523,23 @@ static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMa
     configured[dev] = true;
   }
   count_launches(1);
-  kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, to, tx, p);
+  if (CTA2) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, ta, tb, to, tx, p) != cudaSuccess) return EFQAT_ERR_CUDA;
+  } else {
+    kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, to, tx, p);
+  }
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
@@ -491,10 +554,22 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.splits = (a.epi == EPI_PART) ? a.splits : 1;
   if (p.splits < 1 || p.splits > p.nkb) return EFQAT_ERR_SHAPE;
   p.BN = (a.epi == EPI_PART) ? part_bn(a.Nc) : choose_bn(a.Mr, a.Nc, sm_count);
-  p.tiles_m = static_cast<int>(ceil_div(a.Mr, BM));
+  // CTA pairs (256 x BN tiles) whenever the tiles are full in N: half the B traffic per FLOP
+  int pair = 0;
+  if (a.epi != EPI_PART && a.Mr >= 256 && a.Nc % 128 == 0) {
+    pair = 1;
+    const int units = sm_count / 2;
+    const int64_t mt = ceil_div(a.Mr, 2 * BM);
+    const bool can256 = a.Nc % 256 == 0;
+    const double c256 = can256 ? static_cast<double>(ceil_div(mt * (a.Nc / 256), units)) * (256 + 24) : 1e300;
+    const double c128 = static_cast<double>(ceil_div(mt * (a.Nc / 128), units)) * (128 + 24);
+    p.BN = (c256 <= c128) ? 256 : 128;
+  }
+  const int bn_cta = pair ? p.BN / 2 : p.BN;
+  p.tiles_m = static_cast<int>(ceil_div(a.Mr, pair ? 2 * BM : BM));
   p.tiles_n = static_cast<int>(ceil_div(a.Nc, p.BN));
   p.chunk_cols = a.out_bf16 ? 64 : 32;
-  p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(p.BN, 64) * CHUNK_BYTES : p.BN * BK * 2);
+  p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2);
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
   const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
   const int fixed_bytes = 4 * STG_BYTES + (a.epi == EPI_DX ? 8 * STG_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
@@ -505,7 +580,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.stages = stages;
   p.col_scale = a.col_scale;
   p.col_bias = a.col_bias;
-  p.xq = a.xq;
+  p.s_x = a.s_x; p.z_x = a.z_x; p.x_bits = a.x_bits; p.x_sym = a.x_sym;
   p.partials = a.partials;
   p.out = static_cast<float*>(a.out);
   p.ldo = a.ldo;
@@ -516,7 +591,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   CUtensorMap ta, tb, to, tx;
   rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
   if (rc != EFQAT_OK) return rc;
-  rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, p.BN);
+  rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, bn_cta);
   if (rc != EFQAT_OK) return rc;
   to = ta;
   tx = ta;
@@ -531,17 +606,25 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   }
 
   const int64_t items = static_cast<int64_t>(p.tiles_m) * p.tiles_n * p.splits;
-  const int grid = static_cast<int>(items < sm_count ? items : sm_count);
+  const int max_units = pair ? sm_count / 2 : sm_count;
+  const int units = static_cast<int>(items < max_units ? items : max_units);
+  const int grid = pair ? 2 * units : units;
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + fixed_bytes + 1024;
-  if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * 4;
+  if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * 4;
 
-#define EFQAT_LAUNCH(AM, BMj, E) return launch<AM, BMj, E>(ta, tb, to, tx, p, grid, smem, st)
-  if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) EFQAT_LAUNCH(0, 0, EPI_FWD);
-  if (a.epi == EPI_DX && !a.a_mn && a.b_mn) EFQAT_LAUNCH(0, 1, EPI_DX);
-  if (a.epi == EPI_PART && a.a_mn && a.b_mn) EFQAT_LAUNCH(1, 1, EPI_PART);
-  if (a.epi == EPI_PART && !a.a_mn && !a.b_mn) EFQAT_LAUNCH(0, 0, EPI_PART);
-  if (a.epi == EPI_PART && !a.a_mn && a.b_mn) EFQAT_LAUNCH(0, 1, EPI_PART);
-  if (a.epi == EPI_PART && a.a_mn && !a.b_mn) EFQAT_LAUNCH(1, 0, EPI_PART);
+#define EFQAT_LAUNCH(AM, BMj, E, P2) return launch<AM, BMj, E, P2>(ta, tb, to, tx, p, grid, smem, st)
+  if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) {
+    if (pair) EFQAT_LAUNCH(0, 0, EPI_FWD, 1);
+    EFQAT_LAUNCH(0, 0, EPI_FWD, 0);
+  }
+  if (a.epi == EPI_DX && !a.a_mn && a.b_mn) {
+    if (pair) EFQAT_LAUNCH(0, 1, EPI_DX, 1);
+    EFQAT_LAUNCH(0, 1, EPI_DX, 0);
+  }
+  if (a.epi == EPI_PART && a.a_mn && a.b_mn) EFQAT_LAUNCH(1, 1, EPI_PART, 0);
+  if (a.epi == EPI_PART && !a.a_mn && !a.b_mn) EFQAT_LAUNCH(0, 0, EPI_PART, 0);
+  if (a.epi == EPI_PART && !a.a_mn && a.b_mn) EFQAT_LAUNCH(0, 1, EPI_PART, 0);
+  if (a.epi == EPI_PART && a.a_mn && !a.b_mn) EFQAT_LAUNCH(1, 0, EPI_PART, 0);
 #undef EFQAT_LAUNCH
   return EFQAT_ERR_UNIMPL;
 }

@@ -39,6 +39,36 @@ void launch_minmax_act(const void* x, int dtype, int64_t count, int x_bits, int 
                        float* ws, cudaStream_t st);
 void launch_absmax_rows(const float* W, int64_t N, int64_t K, int w_bits, float* s_w, cudaStream_t st);
 
+// ---- fused.cu -----------------------------------------------------------------------
+// One launch in front of the GEMMs: weight rows -> bf16 operand, activations -> centred codes
+// (skipped when Xc is null), and one pass over dY (skipped when dY is null or nothing of it
+// is wanted) producing column-sum partials, the gathered selected columns and a bf16 copy.
+struct PrepArgs {
+  int64_t M, N, K;
+  const float* W; const float* s_w; int w_bits; bf16* Wq;
+  const void* X; const float* s_x; const float* z_x; int x_bits, x_sym; bf16* Xc;
+  const void* dY; bf16* dYb; float* colsum_ws;
+  const int32_t* idx; int64_t k_sel, pitch; bf16* dYsel;
+  int* status;
+  int nb_w, nb_x, col_blocks, slabs;   // filled by launch_prepare
+};
+int prepare_slabs(int64_t M);
+void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st);
+// One launch behind the GEMMs: dW rows (split reduction, clip mask, dS_w, optional SGD),
+// dS_x / dZ_x from the per-tile partials, db from the column-sum partials.
+struct FinArgs {
+  int64_t N, K, k_sel;
+  const float* P; int splits; int64_t split_stride;
+  const float* W; const float* s_w; const float* s_x; int w_bits;
+  const int32_t* idx;
+  float* dW_sel; float* dS_w_sel;
+  efqat_sgd opt; int has_opt;
+  const float* dx_partials; int n_partials; float* dS_x; float* dZ_x;
+  const float* colsum_ws; int slabs; float* db;
+  int* status;
+};
+void launch_finalize(FinArgs a, cudaStream_t st);
+
 // ---- select.cu ----------------------------------------------------------------------
 size_t select_workspace_bytes(int L, int64_t total_channels);
 int run_select(int mode, int L, const efqat_layer_desc* layers, const float* const* weights, const int64_t* k,
@@ -64,8 +94,8 @@ struct GemmArgs {
   // EPI_FWD
   const float* col_scale;  // s_w[Nc]
   const float* col_bias;   // bias[Nc] or null
-  // EPI_FWD / EPI_DX
-  const ActQ* xq;
+  // EPI_FWD / EPI_DX: learnable activation scale / zero point and their bit-width
+  const float* s_x; const float* z_x; int x_bits, x_sym;
   // EPI_DX
   const void* X;     // raw activations [Mr,Nc] in x_dtype
   int x_dtype;

@@ -53,7 +53,7 @@ int check_layer(const efqat_layer_desc* l, const efqat_qspec* q) {
     if (Ho < 1 || Wo < 1) return EFQAT_ERR_SHAPE;
     if (l->M != static_cast<int64_t>(l->B) * Ho * Wo) return EFQAT_ERR_SHAPE;
     if (l->K != static_cast<int64_t>(l->R) * l->S * l->Cin) return EFQAT_ERR_SHAPE;
-    if (l->R != 1 || l->S != 1 || l->pad != 0) return EFQAT_ERR_UNIMPL;   // 1x1 convolutions only so far
+    if ((l->R != 1 || l->S != 1 || l->pad != 0) && (l->Cin & 63)) return EFQAT_ERR_UNIMPL;   // tap-wise tiles need Cin % 64 == 0
   }
   return EFQAT_OK;
 }
@@ -75,6 +75,31 @@ struct LayerWs {
 
 int64_t sel_pitch(int64_t k_sel) { return round_up(k_sel, 64); }
 
+// A 1x1 convolution without padding is the linear layer on the [B*H*W, Cin] matrix.
+bool spatial_conv(const efqat_layer_desc* l) { return l->is_conv && (l->R != 1 || l->S != 1 || l->pad != 0); }
+
+ConvArgs conv_args(const efqat_layer_desc* l, int mode) {
+  ConvArgs c = {};
+  c.mode = mode;
+  c.B = l->B; c.H = l->H; c.W = l->W; c.Cin = l->Cin;
+  c.Ho = l->H + 2 * l->pad - l->R + 1;
+  c.Wo = l->W + 2 * l->pad - l->S + 1;
+  c.N = static_cast<int>(l->N);
+  c.R = l->R; c.S = l->S; c.pad = l->pad;
+  return c;
+}
+
+int64_t x_elems(const efqat_layer_desc* l) {
+  return spatial_conv(l) ? static_cast<int64_t>(l->B) * l->H * l->W * l->Cin : l->M * l->K;
+}
+
+int dx_partials(const efqat_layer_desc* l) {
+  if (!spatial_conv(l)) return gemm_dx_num_partials(l->M, l->K);
+  int tw, th, tb;
+  conv_pixel_box(l->W, l->H, l->B, 128, &tw, &th, &tb);
+  return static_cast<int>(ceil_div(l->W, tw) * ceil_div(l->H, th) * ceil_div(l->B, tb) * ceil_div(l->Cin, 64) * 4);
+}
+
 LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, int64_t p_elems_override) {
   LayerWs w = {};
   char* base = ws ? reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~uintptr_t(255)) : nullptr;
@@ -86,7 +111,7 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   };
   const int64_t M = l->M, N = l->N, K = l->K;
   w.actq = reinterpret_cast<ActQ*>(take(sizeof(ActQ)));
-  w.Xc = reinterpret_cast<bf16*>(take(M * K * 2));
+  w.Xc = reinterpret_cast<bf16*>(take(x_elems(l) * 2));
   w.Wq = reinterpret_cast<bf16*>(take(N * K * 2));
   w.dYb = reinterpret_cast<bf16*>(take(l->act_dtype == EFQAT_F32 ? M * N * 2 : 0));
   const bool gathered = k_sel > 0 && k_sel < N;
@@ -95,7 +120,7 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   w.splits = k_sel > 0 ? gemm_choose_splits(K, gathered ? round_up(k_sel, 16) : N, M, sm_count) : 1;
   const int64_t p_elems = p_elems_override >= 0 ? p_elems_override : static_cast<int64_t>(w.splits) * k_sel * K;
   w.P = reinterpret_cast<float*>(take(p_elems * 4));
-  w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(gemm_dx_num_partials(M, K)) * 8));
+  w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(dx_partials(l)) * 8));
   w.colsum = reinterpret_cast<float*>(take(static_cast<int64_t>(COLSUM_SLABS) * N * 4));
   w.bytes = off + 256;
   return w;
@@ -306,8 +331,10 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   pa.M = M; pa.N = N; pa.K = K;
   pa.W = W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric; pa.Xc = w.Xc;
+  pa.x_count = x_elems(layer);
   pa.status = ctx->d_status;
   launch_prepare(pa, 0, act_bf16, st);
+  ConvArgs cva;
   GemmArgs g = {};
   g.A = w.Xc; g.B = w.Wq;
   g.Mr = M; g.Nc = N; g.Kc = K;
@@ -318,6 +345,10 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   g.out = Y; g.ldo = N;
   g.col_scale = s_w; g.col_bias = bias_or_null;
   g.s_x = s_x; g.z_x = z_x; g.x_bits = q->x_bits; g.x_sym = q->x_symmetric;
+  if (spatial_conv(layer)) {
+    cva = conv_args(layer, 1);
+    g.conv = &cva;
+  }
   g.status = ctx->d_status;
   rc = timed_gemm(ctx, 0, g, st);
   if (rc != EFQAT_OK) return rc;
@@ -360,6 +391,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   pa.W = W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric;
   pa.Xc = k_sel > 0 ? w.Xc : nullptr;
+  pa.x_count = x_elems(layer);
   pa.dY = dY; pa.dYb = act_bf16 ? nullptr : w.dYb;
   pa.colsum_ws = db_or_null ? w.colsum : nullptr;
   pa.idx = idx; pa.k_sel = k_sel; pa.pitch = w.pitch; pa.dYsel = gathered ? w.dYsel : nullptr;
@@ -367,15 +399,20 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   launch_prepare(pa, 1, act_bf16, st);
   // a4 + a5: dX = (dY W^) masked, with the dS_x / dZ_x partial sums in the epilogue
   int tiles = 0;
+  const bool sconv = spatial_conv(layer);
+  ConvArgs cv_dx = conv_args(layer, 2), cv_dw = conv_args(layer, 3);
   {
     GemmArgs g = {};
+    if (sconv) g.conv = &cv_dx;
     g.A = dYb; g.B = w.Wq;
-    g.Mr = M; g.Nc = K; g.Kc = N;
+    g.Mr = sconv ? x_elems(layer) / layer->Cin : M;
+    g.Nc = sconv ? layer->Cin : K;
+    g.Kc = sconv ? static_cast<int64_t>(layer->R) * layer->S * N : N;
     g.lda = N; g.ldb = K;
     g.a_mn = 0; g.b_mn = 1;
     g.epi = EPI_DX;
     g.out_bf16 = act_bf16;
-    g.out = dX; g.ldo = K;
+    g.out = dX; g.ldo = sconv ? layer->Cin : K;
     g.s_x = s_x; g.z_x = z_x; g.x_bits = q->x_bits; g.x_sym = q->x_symmetric;
     g.X = X; g.x_dtype = layer->act_dtype;
     g.partials = w.dxpart;
@@ -386,6 +423,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   // a6: weight gradient of the unfrozen channels only, as split partial products
   if (k_sel > 0) {
     GemmArgs g = {};
+    if (sconv) g.conv = &cv_dw;
     g.A = w.Xc;                       // D[k, i] = sum_m Xc[m,k] * dYsel[m,i]
     g.B = gathered ? w.dYsel : dYb;
     g.Mr = K; g.Nc = gathered ? round_up(k_sel, 16) : N; g.Kc = M;

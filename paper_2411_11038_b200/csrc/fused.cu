@@ -66,7 +66,7 @@ __device__ __forceinline__ void job_quant_x(const PrepArgs& a, int block, int nb
   const ActQ p = make_actq(a.s_x, a.z_x, a.x_bits, a.x_sym, &bad);
   if (bad && block == 0 && threadIdx.x == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
   const T* X = static_cast<const T*>(a.X);
-  const int64_t n8 = a.M * a.K / 8;
+  const int64_t n8 = a.x_count / 8;
   for (int64_t i = static_cast<int64_t>(block) * blockDim.x + threadIdx.x; i < n8;
        i += static_cast<int64_t>(nblocks) * blockDim.x) {
     float v[8];
@@ -264,7 +264,7 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   a.nb_w = static_cast<int>(a.N);
   a.nb_x = 0;
   if (a.Xc) {
-    int64_t nb = ceil_div(a.M * a.K / 8, 256 * 2);
+    int64_t nb = ceil_div(a.x_count / 8, 256 * 2);
     if (nb > 148 * 8) nb = 148 * 8;
     if (nb < 1) nb = 1;
     a.nb_x = static_cast<int>(nb);

@@ -36,7 +36,19 @@ static const int ACC_STRIDE = 256;              // TMEM columns between the two 
 static const int TMEM_COLS = 512;
 static const int STG_BYTES = 32 * 128;          // staging slice of one epilogue warp: 32 rows x 128 B
 
+// Convolution geometry as the kernel needs it (mode 0 = plain matrices).
+struct ConvP {
+  int mode;                 // 1 forward, 2 grad-input, 3 grad-weight
+  int tw, th, tb;           // pixel box: one 128-row tile (modes 1, 2) or one 64-row contraction block (mode 3)
+  int tiles_w, tiles_h;     // boxes along W and H (boxes along B follow from the tile / block count)
+  int dimH, dimB;           // extent of the tiled pixel space in H and B (store / load guards)
+  int R, S, pad;
+  int C;                    // channels of the 4-D A tensor (Cin for modes 1 and 3, N for mode 2)
+  int cchunks;              // 64-channel chunks of C
+};
+
 struct GemmParams {
+  ConvP cv;
   int64_t Mr, Nc;
   int nkb;            // number of BK blocks along the contraction
   int BN;             // tile columns (multiple of 16, <= 256)
@@ -179,7 +191,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             } else {
               tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
             }
-          } else {
+          } else if (p.cv.mode == 0) {
             mbar_arrive_expect_tx(&ctl->full[s], tx);
             if (A_MN) {
               tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
@@ -192,6 +204,40 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
             } else {
               tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+            }
+          } else if (p.cv.mode == 3) {
+            // grad-weight: contraction block kb = one box of 64 output pixels; tile rows = (tap, channel)
+            mbar_arrive_expect_tx(&ctl->full[s], tx);
+            const int bw = kb % p.cv.tiles_w, bh = (kb / p.cv.tiles_w) % p.cv.tiles_h;
+            const int bb = kb / (p.cv.tiles_w * p.cv.tiles_h);
+            const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
+            for (int j = 0; j < 2; ++j) {
+              const int k = m0 + 64 * j;
+              int rs = k / p.cv.C, c = k - rs * p.cv.C;
+              if (rs >= p.cv.R * p.cv.S) { rs = 0; c = p.cv.C; }     // past the last tap: all zeros
+              const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
+              tma_load_4d(sa + j * CHUNK_BYTES, &tmA, &ctl->full[s], c, w0 + sx - p.cv.pad, h0 + r - p.cv.pad, b0);
+            }
+            for (int c = 0; c < b_chunks; ++c)
+              tma_load_4d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, w0, h0, b0);
+          } else {
+            // forward / grad-input: tile rows = one box of 128 pixels; contraction block kb = (tap, 64 channels)
+            mbar_arrive_expect_tx(&ctl->full[s], tx);
+            const int tmi = t / p.tiles_n;
+            const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
+            const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
+            const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
+            const int rs = kb / p.cv.cchunks, cc = kb - rs * p.cv.cchunks;
+            const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
+            const int dw = (p.cv.mode == 1) ? sx - p.cv.pad : p.cv.pad - sx;
+            const int dh = (p.cv.mode == 1) ? r - p.cv.pad : p.cv.pad - r;
+            tma_load_4d(sa, &tmA, &ctl->full[s], cc * 64, w0 + dw, h0 + dh, b0);
+            if (B_MN) {     // W^ viewed as [N rows, R*S*Cin columns]: rows = contraction, Nc = Cin
+              for (int c = 0; c < b_chunks; ++c)
+                tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s],
+                            rs * static_cast<int>(p.Nc) + n0 + 64 * c, cc * 64);
+            } else {        // weight codes [N, R*S*Cin]
+              tma_load_2d(sb, &tmB, &ctl->full[s], rs * p.cv.C + cc * 64, n0);
             }
           }
         }
@@ -277,6 +323,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       n_eff = (n_eff + 15) & ~15;
       const int buf = acc_it & 1;
       const int row0 = m0 + q * 32;
+      // convolution: this warp's 32 rows are a sub-box of the tile's pixel box
+      int pw0 = 0, ph0 = 0, pb0 = 0;
+      bool rows_live = row0 < p.Mr;
+      if (EPI != EPI_PART && p.cv.mode != 0) {
+        const int tmi = t / p.tiles_n;
+        const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
+        const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
+        const int pix = q * 32;
+        pw0 = bw * p.cv.tw;
+        ph0 = bh * p.cv.th + (pix / p.cv.tw) % p.cv.th;
+        pb0 = bb * p.cv.tb + pix / (p.cv.tw * p.cv.th);
+        rows_live = ph0 < p.cv.dimH && pb0 < p.cv.dimB;
+      }
       if (EPI == EPI_FWD) {
         // this warp's own copy of the tile's column scales and biases (no cross-warp barrier)
         float* sc = s_scale + q * 256;
@@ -293,7 +352,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // first X slice of this tile: in flight while the main loop of the tile finishes
         uint64_t* xb = &ctl->xbar[q][x_it & 1];
         mbar_arrive_expect_tx(xb, STG_BYTES);
-        tma_load_2d(my_x + (x_it & 1) * STG_BYTES, &tmX, xb, n0, row0);
+        if (p.cv.mode != 0) tma_load_4d(my_x + (x_it & 1) * STG_BYTES, &tmX, xb, n0, pw0, ph0, pb0);
+        else tma_load_2d(my_x + (x_it & 1) * STG_BYTES, &tmX, xb, n0, row0);
       }
       bool got = *abort_flag ? false : mbar_wait(&ctl->acc_full[buf], (acc_it >> 1) & 1);
       got = __all_sync(0xffffffffu, got);
@@ -333,7 +393,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (lane == 0 && c0 + cc < n_eff) {       // prefetch the next slice of this tile
               uint64_t* xb = &ctl->xbar[q][xb_i ^ 1];
               mbar_arrive_expect_tx(xb, STG_BYTES);
-              tma_load_2d(my_x + (xb_i ^ 1) * STG_BYTES, &tmX, xb, n0 + c0 + cc, row0);
+              if (p.cv.mode != 0)
+                tma_load_4d(my_x + (xb_i ^ 1) * STG_BYTES, &tmX, xb, n0 + c0 + cc, pw0, ph0, pb0);
+              else
+                tma_load_2d(my_x + (xb_i ^ 1) * STG_BYTES, &tmX, xb, n0 + c0 + cc, row0);
             }
             bool gx = mbar_wait(&ctl->xbar[q][xb_i], (x_it >> 1) & 1);
             gx = __all_sync(0xffffffffu, gx);
@@ -406,8 +469,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           fence_proxy_async();
           __syncwarp();
-          if (lane == 0 && row0 < p.Mr && n0 + c0 < p.Nc) {
-            tma_store_2d(&tmOut, my_out, n0 + c0, row0);   // clipped at the tensor's edges
+          if (lane == 0 && rows_live && n0 + c0 < p.Nc) {     // stores are clipped at the tensor's edges
+            if (p.cv.mode != 0) tma_store_4d(&tmOut, my_out, n0 + c0, pw0, ph0, pb0);
+            else tma_store_2d(&tmOut, my_out, n0 + c0, row0);
             tma_store_commit();
           }
         }
@@ -469,6 +533,43 @@ static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows,
                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? EFQAT_OK : EFQAT_ERR_CUDA;
+}
+
+// 4-D NHWC tensor [B,H,W,C] (pitch C elements per pixel); box = 128 bytes of channels x bw x bh x bb pixels.
+static int make_map_4d(CUtensorMap* m, const void* base, int is_bf16, int64_t B, int64_t H, int64_t W, int64_t C,
+                       int64_t pitch, int bw, int bh, int bb) {
+  const int es = is_bf16 ? 2 : 4;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
+                              static_cast<cuuint64_t>(B)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(pitch) * es, static_cast<cuuint64_t>(pitch) * W * es,
+                                 static_cast<cuuint64_t>(pitch) * W * H * es};
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / es), static_cast<cuuint32_t>(bw),
+                             static_cast<cuuint32_t>(bh), static_cast<cuuint32_t>(bb)};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r = g_encode(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+                              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? EFQAT_OK : EFQAT_ERR_CUDA;
+}
+
+// Pixel box (power-of-two sides, tw * th * tb = target) that wastes the least work on a
+// W x H x B pixel space; tw <= 32 so that a quarter of a 128-pixel box is a sub-box.
+void conv_pixel_box(int W, int H, int B, int target, int* tw, int* th, int* tb) {
+  double best = 1e300;
+  *tw = 1; *th = 1; *tb = target;
+  for (int a = 1; a <= target && a <= 32; a <<= 1)
+    for (int b = 1; a * b <= target; b <<= 1) {
+      const int c = target / (a * b);
+      const double vol = static_cast<double>(ceil_div(W, a) * a) * static_cast<double>(ceil_div(H, b) * b) *
+                         static_cast<double>(ceil_div(B, c) * c);
+      // prefer wider boxes at equal volume: longer contiguous runs per TMA row
+      const double score = vol - 1e-3 * a - 1e-6 * b;
+      if (score < best) {
+        best = score;
+        *tw = a; *th = b; *tb = c;
+      }
+    }
 }
 
 // Tile width for the forward / grad-input GEMMs: multiples of 64 so that every 128-byte
@@ -554,9 +655,16 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.splits = (a.epi == EPI_PART) ? a.splits : 1;
   if (p.splits < 1 || p.splits > p.nkb) return EFQAT_ERR_SHAPE;
   p.BN = (a.epi == EPI_PART) ? part_bn(a.Nc) : choose_bn(a.Mr, a.Nc, sm_count);
+  const ConvArgs* cv = a.conv;
+  if (cv) {
+    if (cv->mode < 1 || cv->mode > 3 || (cv->Cin & 63)) return EFQAT_ERR_UNIMPL;
+    if (cv->mode == 2) {           // grad-input tiles must not straddle the end of Cin (B is not zero there)
+      p.BN = (cv->Cin % 256 == 0) ? 256 : (cv->Cin % 192 == 0) ? 192 : (cv->Cin % 128 == 0) ? 128 : 64;
+    }
+  }
   // CTA pairs (256 x BN tiles) whenever the tiles are full in N: half the B traffic per FLOP
   int pair = 0;
-  if (a.epi != EPI_PART && a.Mr >= 256 && a.Nc % 128 == 0) {
+  if (!cv && a.epi != EPI_PART && a.Mr >= 256 && a.Nc % 128 == 0) {
     pair = 1;
     const int units = sm_count / 2;
     const int64_t mt = ceil_div(a.Mr, 2 * BM);
@@ -568,6 +676,27 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   const int bn_cta = pair ? p.BN / 2 : p.BN;
   p.tiles_m = static_cast<int>(ceil_div(a.Mr, pair ? 2 * BM : BM));
   p.tiles_n = static_cast<int>(ceil_div(a.Nc, p.BN));
+  if (cv) {
+    ConvP& c = p.cv;
+    c.mode = cv->mode;
+    c.R = cv->R; c.S = cv->S; c.pad = cv->pad;
+    // pixel space that is tiled: outputs for forward and grad-weight, inputs for grad-input
+    const int pW = (cv->mode == 2) ? cv->W : cv->Wo, pH = (cv->mode == 2) ? cv->H : cv->Ho;
+    conv_pixel_box(pW, pH, cv->B, cv->mode == 3 ? BK : BM, &c.tw, &c.th, &c.tb);
+    c.tiles_w = static_cast<int>(ceil_div(pW, c.tw));
+    c.tiles_h = static_cast<int>(ceil_div(pH, c.th));
+    const int tiles_b = static_cast<int>(ceil_div(cv->B, c.tb));
+    c.dimH = pH; c.dimB = cv->B;
+    c.C = (cv->mode == 2) ? cv->N : cv->Cin;
+    c.cchunks = static_cast<int>(ceil_div(c.C, 64));
+    if (cv->mode == 3) {
+      p.nkb = c.tiles_w * c.tiles_h * tiles_b;                 // contraction over boxes of 64 output pixels
+      if (p.splits > p.nkb) return EFQAT_ERR_SHAPE;
+    } else {
+      p.tiles_m = c.tiles_w * c.tiles_h * tiles_b;             // one tile per box of 128 pixels
+      p.nkb = cv->R * cv->S * c.cchunks;
+    }
+  }
   p.chunk_cols = a.out_bf16 ? 64 : 32;
   p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2);
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
@@ -589,19 +718,47 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.status = a.status;
 
   CUtensorMap ta, tb, to, tx;
-  rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
-  if (rc != EFQAT_OK) return rc;
-  rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, bn_cta);
-  if (rc != EFQAT_OK) return rc;
-  to = ta;
-  tx = ta;
-  if (a.epi != EPI_PART) {
-    rc = make_map(&to, a.out, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+  if (a.epi == EPI_DX && (a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;
+  if (!cv) {
+    rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
     if (rc != EFQAT_OK) return rc;
-  }
-  if (a.epi == EPI_DX) {
-    if ((a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;
-    rc = make_map(&tx, a.X, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+    rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, bn_cta);
+    if (rc != EFQAT_OK) return rc;
+    to = ta;
+    tx = ta;
+    if (a.epi != EPI_PART) {
+      rc = make_map(&to, a.out, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+      if (rc != EFQAT_OK) return rc;
+    }
+    if (a.epi == EPI_DX) {
+      rc = make_map(&tx, a.X, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+      if (rc != EFQAT_OK) return rc;
+    }
+  } else {
+    const ConvP& c = p.cv;
+    const int64_t KK = static_cast<int64_t>(cv->R) * cv->S * cv->Cin;
+    // quarter of a 128-pixel box: the 32 rows one epilogue warp owns
+    const int qh = (32 / c.tw < c.th) ? 32 / c.tw : c.th;
+    const int qb = 32 / (c.tw * qh);
+    if (cv->mode == 1) {
+      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, c.th, c.tb);
+      if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, bn_cta);
+      if (rc == EFQAT_OK)
+        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, qh, qb);
+      tx = ta;
+    } else if (cv->mode == 2) {
+      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, c.th, c.tb);
+      if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, BK);
+      if (rc == EFQAT_OK)
+        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb);
+      if (rc == EFQAT_OK)
+        rc = make_map_4d(&tx, a.X, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb);
+    } else {
+      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, c.th, c.tb);
+      if (rc == EFQAT_OK) rc = make_map_4d(&tb, a.B, 1, cv->B, cv->Ho, cv->Wo, a.Nc, a.ldb, c.tw, c.th, c.tb);
+      to = ta;
+      tx = ta;
+    }
     if (rc != EFQAT_OK) return rc;
   }
 

@@ -47,6 +47,7 @@ struct PrepArgs {
   int64_t M, N, K;
   const float* W; const float* s_w; int w_bits; bf16* Wq;
   const void* X; const float* s_x; const float* z_x; int x_bits, x_sym; bf16* Xc;
+  int64_t x_count;   // elements of X (B*H*W*Cin for convolutions, M*K otherwise)
   const void* dY; bf16* dYb; float* colsum_ws;
   const int32_t* idx; int64_t k_sel, pitch; bf16* dYsel;
   int* status;
@@ -78,7 +79,22 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
 // ---- gemm.cu ------------------------------------------------------------------------
 enum GemmEpi { EPI_FWD = 0, EPI_DX = 1, EPI_PART = 2 };
 
+// Implicit-GEMM convolution geometry (stride 1).  The activation operand is read through a
+// 4-D tensor map over its NHWC tensor with a box of pixels shifted by the filter tap; pixels
+// that fall into the padding come back as zeros from the TMA unit.
+//   mode 1 forward : A = Xc [B,H,W,Cin] patches, B = weight codes [N, R*S*Cin], D = Y [B,Ho,Wo,N]
+//   mode 2 grad-in : A = dY [B,Ho,Wo,N] patches, B = W^ [N, R*S*Cin] (MN-major), D = dX [B,H,W,Cin]
+//   mode 3 grad-w  : A = Xc patches (MN-major), B = gathered dY [B,Ho,Wo,pitch] (MN-major),
+//                    D[(r,s,c), i] partial products, contraction over output pixels
+struct ConvArgs {
+  int mode;
+  int B, H, W, Cin;     // input activation tensor
+  int Ho, Wo, N;        // output activation tensor
+  int R, S, pad;
+};
+
 struct GemmArgs {
+  const ConvArgs* conv;  // null for linear layers
   // D[Mr, Nc] = A * B over contraction length Kc.
   // a_mn = 0: A is stored [Mr, Kc] row-major; a_mn = 1: A is stored [Kc, Mr] row-major.
   // b_mn = 0: B is stored [Nc, Kc] row-major; b_mn = 1: B is stored [Kc, Nc] row-major.
@@ -111,6 +127,7 @@ int gemm_dx_num_partials(int64_t Mr, int64_t Nc);
 // Split count along the contraction for EPI_PART.
 int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count);
 int gemm_init();  // resolves the tensor-map encoder; returns an efqat_status
+void conv_pixel_box(int W, int H, int B, int target, int* tw, int* th, int* tb);
 // tiles_out (optional): number of output tiles = number of partial pairs EPI_DX wrote.
 int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out = nullptr);
 

@@ -1,0 +1,112 @@
+"""GPU parity of the convolution form of the layer step (implicit GEMM over NHWC tensors,
+stride 1) against the oracle: forward, grad-input with the STE mask and dS_x / dZ_x, and the
+partial grad-weight, including padded borders with a non-zero activation zero point."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import efqat_oracle as O
+from paper_2411_11038_b200 import binding as B
+from paper_2411_11038_b200 import inputs as I
+from tests import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    return B.Context(0)
+
+
+def _case(name, Bn, H, Wd, Cin, N, R, pad, dtype=torch.bfloat16, w_bits=4, seed=0):
+    Ho, Wo = H + 2 * pad - R + 1, Wd + 2 * pad - R + 1
+    return I.LayerCase(name, Bn * Ho * Wo, R * R * Cin, N, act_dtype=dtype, w_bits=w_bits, x_bits=8, w_std=None,
+                       x_abs=True, seed=seed, conv=True, B=Bn, H=H, Wd=Wd, Cin=Cin, R=R, S=R, stride=1, pad=pad)
+
+
+CASES = [
+    _case("c3x3_small", 2, 9, 10, 64, 72, 3, 1, seed=1),
+    _case("c3x3_valid_f32", 3, 8, 8, 64, 64, 3, 0, dtype=torch.float32, seed=2),
+    _case("c5x5", 2, 7, 7, 128, 136, 5, 2, w_bits=8, seed=3),
+    _case("c3x3_14", 4, 14, 14, 128, 256, 3, 1, seed=4),
+    _case("c1x1", 2, 12, 12, 72, 64, 1, 0, seed=5),
+    _case("resnet_56_64to256_3x3_b2", 2, 56, 56, 64, 256, 3, 1, seed=6),
+]
+
+
+def _abs_bounds(case, T, s_w, s_x, z_x):
+    """Sum of |terms| of every output of the three contractions (same loops as the definition)."""
+    X64, W64, dY64 = (I.as_f64(T[k]) for k in ("X", "W", "dY"))
+    qx = O.fake_quant_x(X64, s_x, z_x, case.x_bits)
+    qw = O.fake_quant_w(W64, s_w, case.w_bits)
+    N, R, S, C = W64.shape
+    Bn, H, Wd, _ = X64.shape
+    Ho, Wo = dY64.shape[1:3]
+    pad = case.pad
+    P = O._patches(np.abs(qx["deq"]), R, S, 1, pad).reshape(-1, R * S * C)
+    Yabs = (P @ np.abs(qw["deq"]).reshape(N, -1).T).reshape(Bn, Ho, Wo, N)
+    dY2 = np.abs(dY64).reshape(-1, N)
+    Pc = O._patches(np.abs(qx["c0"]), R, S, 1, pad).reshape(-1, R * S * C)
+    Gw_abs = (float(s_x) * (dY2.T @ Pc)).reshape(N, R, S, C)
+    Gp = (dY2 @ np.abs(qw["deq"]).reshape(N, -1)).reshape(Bn, Ho, Wo, R, S, C)
+    Gxp = np.zeros((Bn, H + 2 * pad, Wd + 2 * pad, C))
+    for r in range(R):
+        for s in range(S):
+            Gxp[:, r:r + Ho, s:s + Wo, :] += Gp[:, :, :, r, s, :]
+    return Yabs, Gxp[:, pad:pad + H, pad:pad + Wd, :], Gw_abs
+
+
+@pytest.mark.parametrize("case", CASES, ids=lambda c: c.name)
+def test_conv_forward_backward_parity(ctx, case):
+    T = I.make_tensors(case)
+    T["X"] = (T["X"].float() - 0.3).to(case.act_dtype)        # asymmetric range: Z != 0, pad must act as x^ = 0
+    X64, W64, dY64, b64 = (I.as_f64(T[k]) for k in ("X", "W", "dY", "bias"))
+    s_w = (O.init_minmax_w(W64, case.w_bits) * np.float32(0.9)).astype(np.float32)
+    s_x, z_x = O.init_minmax_x(X64, case.x_bits)
+    s_x = np.float32(s_x * np.float32(0.8))
+    assert float(np.clip(np.rint(z_x), 0, 255)) > 0
+    D = U.to_dev(T, s_w, s_x, z_x)
+    geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, 1, case.pad)
+    is_bf16 = case.act_dtype == torch.bfloat16
+    Yabs, Gx_abs, Gw_abs = _abs_bounds(case, T, s_w, s_x, z_x)
+
+    Y = B.fq_linear_fwd(ctx, D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"], case.w_bits, case.x_bits,
+                        False, conv=geom)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ref = O.conv_forward(X64, W64, s_w, s_x, z_x, b64, case.w_bits, case.x_bits, 1, case.pad)
+    got = U.np32(Y)
+    U.assert_bf16_class(got, ref, case.name + " Y")
+    U.assert_fp32_class(got, ref, Yabs + np.abs(b64), case.name + " Y", out_is_bf16=is_bf16)
+
+    N = case.N
+    sets = [np.zeros(0, np.int32), O.select_cwpl([W64], [max(1, N // 10)])[0], np.arange(N, dtype=np.int32)]
+    outs = []
+    for idx in sets:
+        k = len(idx)
+        idx_dev = torch.from_numpy(idx).cuda() if 0 < k < N else None
+        out = B.fq_linear_bwd(ctx, D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx_dev, k,
+                              case.w_bits, case.x_bits, False, want_db=True, conv=geom)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        g = {kk: (U.np32(v) if v is not None else None) for kk, v in out.items()}
+        outs.append(g)
+        args = (dY64, X64, W64, s_w, s_x, z_x, idx, case.w_bits, case.x_bits, 1, case.pad)
+        ex = O.conv_backward_efqat(*args, operand_model="exact")
+        bm = O.conv_backward_efqat(*args, operand_model="bf16")
+        name = f"{case.name} k_sel={k}"
+        clip_x = O.fake_quant_x(X64, s_x, z_x, case.x_bits)["flag"] != 0
+        assert clip_x.any() and np.all(g["dX"][clip_x] == 0)
+        U.assert_bf16_class(g["dX"], ex["dX"], name + " dX")
+        U.assert_fp32_class(g["dX"], bm["dX"], Gx_abs, name + " dX", out_is_bf16=is_bf16)
+        for key in ("dS_x", "dZ_x"):
+            U.assert_fp32_class(g[key][0], bm[key], bm[key + "_abs"], name + " " + key, atol=1e-30)
+        U.assert_fp32_class(g["db"], bm["db"], np.abs(dY64).reshape(-1, N).sum(axis=0), name + " db")
+        dW = g["dW_sel"].reshape((k,) + W64.shape[1:])
+        if k:
+            U.assert_bf16_class(dW, ex["dW_sel"], name + " dW_sel")
+            U.assert_fp32_class(dW, bm["dW_sel"], Gw_abs[idx], name + " dW_sel")
+            U.assert_fp32_class(g["dS_w_sel"], bm["dS_w_sel"], bm["dS_w_sel_abs"], name + " dS_w", atol=1e-30)
+    for o in outs[1:]:
+        for key in ("dX", "dS_x", "dZ_x", "db"):
+            assert np.array_equal(o[key], outs[0][key]), key

@@ -1,0 +1,144 @@
+"""Per-layer timing sweep over the five workload families (single GPU).
+
+    python -m paper_2411_11038_b200.sweep [--configs 1,2,3,4,5] [--iters 30] [--out file.jsonl]
+
+For every layer: forward ms, backward ms at each unfrozen fraction, algorithmic TFLOP/s
+(2MNK forward, 2MNK(1 + k/N) backward, Eq. 7-8 of the paper), the speed-up of the partial
+backward over this library's own full-QAT backward next to the ideal 2/(1+r), and the
+selection time.  Every number is the median over `iters` runs timed with CUDA events, with a
+256 MiB buffer written between runs so that nothing is served from a warm L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+import sys
+
+import torch
+
+from . import binding as B
+from . import inputs as I
+
+FRACS = {1: (0.0, 26 / 512, 1.0), 2: (0.0, 0.05, 0.25, 1.0), 3: (0.0, 0.10, 1.0), 4: (0.0, 0.10, 1.0),
+         5: (0.0, 0.01, 0.05, 0.10, 0.25, 0.50, 1.0)}
+
+
+class Timer:
+    def __init__(self, iters: int, device):
+        self.iters = iters
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def ms(self, fn, warmup: int = 5) -> float:
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        out = []
+        for _ in range(self.iters):
+            self.flush.zero_()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            fn()
+            e.record()
+            torch.cuda.synchronize()
+            out.append(s.elapsed_time(e))
+        return statistics.median(out)
+
+
+def layer_on_device(ctx, case: I.LayerCase, dev):
+    T = I.make_tensors(case)
+    D = {k: (v.to(dev) if v is not None else None) for k, v in T.items()}
+    D["s_w"] = B.init_weight_scales(ctx, D["W"], case.w_bits)
+    D["s_x"], D["z_x"] = B.init_act_qparams(ctx, D["X"], case.x_bits, case.x_symmetric)
+    conv = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, case.stride, case.pad) if case.conv else None
+    if conv is not None:
+        Ho, Wo = case.H + 2 * case.pad - case.R + 1, case.Wd + 2 * case.pad - case.S + 1
+        plan = B.LayerPlan(ctx, case.M, case.N, case.K, case.act_dtype, case.w_bits, case.x_bits, case.x_symmetric,
+                           case.N, dev, conv, x_shape=D["X"].shape, y_shape=(case.B, Ho, Wo, case.N))
+    else:
+        plan = B.LayerPlan(ctx, case.M, case.N, case.K, case.act_dtype, case.w_bits, case.x_bits, case.x_symmetric,
+                           case.N, dev)
+    return D, plan
+
+
+def sweep_layer(ctx, case, fracs, timer, dev, ks=None):
+    D, plan = layer_on_device(ctx, case, dev)
+    g = 2.0 * case.M * case.N * case.K
+    rec = {"layer": case.name, "M": case.M, "N": case.N, "K": case.K, "w_bits": case.w_bits, "x_bits": case.x_bits}
+    t = timer.ms(lambda: plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"]))
+    rec["fwd_ms"], rec["fwd_tflops"] = t, g / t / 1e9
+    rec["bwd"] = {}
+    full_ms = None
+    for f in sorted(set(fracs), reverse=True):
+        k = B.ratio_to_k(f, case.N) if ks is None else ks[f]
+        sel = B.SelectPlan(ctx, B.CWPL, [D["W"]], [k])
+        sel.run()
+        idx = sel.idx[:k] if 0 < k < case.N else None
+        t = timer.ms(lambda: plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True))
+        if f == 1.0:
+            full_ms = t
+        rec["bwd"][f"{f:.4g}"] = {"k_sel": k, "ms": t, "tflops": (g + 2.0 * case.M * k * case.K) / t / 1e9,
+                                  "speedup_vs_full_qat": (full_ms / t) if full_ms else None,
+                                  "ideal": 2.0 / (1.0 + k / case.N)}
+    sel = B.SelectPlan(ctx, B.CWPL, [D["W"]], [B.ratio_to_k(0.05, case.N)])
+    t = timer.ms(sel.run)
+    rec["select_ms"], rec["select_gbs"] = t, case.N * case.K * 4 / t / 1e6
+    return rec
+
+
+def sweep_network(ctx, timer, dev):
+    """Config 4: one global ranking over the 144 layers, then the per-layer steps with the
+    counts that ranking assigns (the 4096->1024 layers end up fully frozen)."""
+    cases = I.config4()
+    Ws = []
+    for c in cases:
+        g = torch.Generator().manual_seed(c.seed)
+        Ws.append((torch.randn((c.N, c.K), generator=g) * (2.0 / c.K) ** 0.5).to(dev))
+    total = sum(c.N for c in cases)
+    budget = B.ratio_to_k(0.1, total)
+    plan = B.SelectPlan(ctx, B.CWPN, Ws, [budget])
+    t = timer.ms(plan.run)
+    nbytes = sum(w.numel() * 4 for w in Ws)
+    counts = (plan.offsets[1:] - plan.offsets[:-1]).cpu().tolist()
+    out = [{"layer": "cfg4_cwpn_selection_144_layers", "select_ms": t, "select_gbs": nbytes / t / 1e6,
+            "channels": total, "budget": budget, "per_layer_counts_block0": counts[:6]}]
+    del Ws, plan
+    torch.cuda.empty_cache()
+    for j in (0, 4, 5):                       # one of each shape: 1024->1024, 1024->4096, 4096->1024
+        c = cases[j]
+        ks = {0.0: 0, 0.10: counts[j], 1.0: c.N}
+        out.append(sweep_layer(ctx, c, (0.0, 0.10, 1.0), timer, dev, ks))
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="1,2,3,4,5")
+    ap.add_argument("--iters", type=int, default=30)
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    ctx = B.Context(0)
+    timer = Timer(args.iters, dev)
+    sink = open(args.out, "w") if args.out else sys.stdout
+    for cfg in (int(c) for c in args.configs.split(",")):
+        if cfg == 4:
+            recs = sweep_network(ctx, timer, dev)
+        else:
+            cases = {1: I.config1, 2: I.config2, 3: I.config3, 5: I.config5}[cfg]()
+            if cfg == 5:
+                cases = cases + I.config5(4, 4)
+            recs = []
+            for c in cases:
+                recs.append(sweep_layer(ctx, c, FRACS[cfg], timer, dev))
+                torch.cuda.empty_cache()
+        for r in recs:
+            r["config"] = cfg
+            sink.write(json.dumps(r) + "\n")
+            sink.flush()
+    assert ctx.device_status() == 0
+
+
+if __name__ == "__main__":
+    main()

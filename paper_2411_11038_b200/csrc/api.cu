@@ -121,7 +121,7 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   const int64_t p_elems = p_elems_override >= 0 ? p_elems_override : static_cast<int64_t>(w.splits) * k_sel * K;
   w.P = reinterpret_cast<float*>(take(p_elems * 4));
   w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(dx_partials(l)) * 8));
-  w.colsum = reinterpret_cast<float*>(take(static_cast<int64_t>(COLSUM_SLABS) * N * 4));
+  w.colsum = reinterpret_cast<float*>(take(static_cast<int64_t>(prepare_slabs(M, N)) * N * 4));
   w.bytes = off + 256;
   return w;
 }
@@ -448,7 +448,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   if (opt_or_null) fa.opt = *opt_or_null;
   fa.has_opt = opt_or_null != nullptr;
   fa.dx_partials = w.dxpart; fa.n_partials = tiles; fa.dS_x = dS_x; fa.dZ_x = dZ_x;
-  fa.colsum_ws = w.colsum; fa.slabs = prepare_slabs(M); fa.db = db_or_null;
+  fa.colsum_ws = w.colsum; fa.slabs = prepare_slabs(M, N); fa.db = db_or_null;
   fa.status = ctx->d_status;
   launch_finalize(fa, st);
   return last_error();

@@ -116,7 +116,24 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
   if (col_ok) {
-    for (int64_t m = m_lo + warp; m < m_hi; m += 8) {
+    int64_t m = m_lo + warp;
+    for (; m + 24 < m_hi; m += 32) {       // four independent 16-byte loads in flight per thread
+      float v[4][8];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) ld8<T>(dY + (m + 8 * u) * a.N + c0, v[u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] += v[u][j];
+        if (a.dYb) st8(a.dYb + (m + 8 * u) * a.N + c0, v[u]);
+        if (gather) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (pos[j] >= 0) a.dYsel[(m + 8 * u) * a.pitch + pos[j]] = __float2bfloat16_rn(v[u][j]);
+        }
+      }
+    }
+    for (; m < m_hi; m += 8) {
       float v[8];
       ld8<T>(dY + m * a.N + c0, v);
 #pragma unroll
@@ -242,20 +259,33 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
       a.dZ_x[0] = static_cast<float>(shd[1][0]);
     }
   } else {
-    const int64_t n = static_cast<int64_t>(b - a.k_sel - 1) * 256 + threadIdx.x;
-    if (n < a.N) {
-      double acc = 0.0;
-      for (int s = 0; s < a.slabs; ++s) acc += static_cast<double>(a.colsum_ws[static_cast<int64_t>(s) * a.N + n]);
-      a.db[n] = static_cast<float>(acc);
+    // db: 32 columns per block, 8 threads per column over the slabs, fixed combination order
+    const int c = threadIdx.x & 31, j = threadIdx.x >> 5;
+    const int64_t n = static_cast<int64_t>(b - a.k_sel - 1) * 32 + c;
+    double acc = 0.0;
+    if (n < a.N)
+      for (int s = j; s < a.slabs; s += 8) acc += static_cast<double>(a.colsum_ws[static_cast<int64_t>(s) * a.N + n]);
+    shd[0][threadIdx.x] = acc;
+    __syncthreads();
+    if (j == 0 && n < a.N) {
+      double t = 0.0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) t += shd[0][w * 32 + c];
+      a.db[n] = static_cast<float>(t);
     }
   }
 }
 
 }  // namespace
 
-int prepare_slabs(int64_t M) {
-  int64_t s = ceil_div(M, 32);
-  if (s > COLSUM_SLABS) s = COLSUM_SLABS;
+// Row slabs of the dY pass: enough blocks (column blocks x slabs) to fill the GPU about four
+// times over, at least 32 rows per slab.
+int prepare_slabs(int64_t M, int64_t N) {
+  const int64_t col_blocks = ceil_div(N, 256);
+  int64_t s = ceil_div(4 * 148, col_blocks);
+  const int64_t by_rows = ceil_div(M, 32);
+  if (s > by_rows) s = by_rows;
+  if (s > 2048) s = 2048;
   if (s < 1) s = 1;
   return static_cast<int>(s);
 }
@@ -272,7 +302,7 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   const bool gather = a.k_sel > 0 && a.k_sel < a.N;
   int nb_y = 0;
   a.col_blocks = static_cast<int>(ceil_div(a.N, 256));
-  a.slabs = prepare_slabs(a.M);
+  a.slabs = prepare_slabs(a.M, a.N);
   if (a.dY && (a.colsum_ws || gather || a.dYb)) nb_y = a.col_blocks * a.slabs;
   const int grid = a.nb_w + a.nb_x + nb_y;
   count_launches(1);
@@ -286,7 +316,7 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
 }
 
 void launch_finalize(FinArgs a, cudaStream_t st) {
-  const int nb_db = a.db ? static_cast<int>(ceil_div(a.N, 256)) : 0;
+  const int nb_db = a.db ? static_cast<int>(ceil_div(a.N, 32)) : 0;
   const int grid = static_cast<int>(a.k_sel) + 1 + nb_db;
   count_launches(1);
   finalize_kernel<<<grid, 256, 0, st>>>(a);

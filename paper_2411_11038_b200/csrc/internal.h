@@ -53,7 +53,7 @@ struct PrepArgs {
   int* status;
   int nb_w, nb_x, col_blocks, slabs;   // filled by launch_prepare
 };
-int prepare_slabs(int64_t M);
+int prepare_slabs(int64_t M, int64_t N);
 void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st);
 // One launch behind the GEMMs: dW rows (split reduction, clip mask, dS_w, optional SGD),
 // dS_x / dZ_x from the per-tile partials, db from the column-sum partials.

@@ -137,6 +137,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
                                                             const LayerEntry* __restrict__ table, int single_len,
                                                             int single_k, int32_t* __restrict__ out) {
   __shared__ int hist[256];
+  __shared__ int suf[257];
   __shared__ int scan_sh[64];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
@@ -167,14 +168,23 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
       if (digit < 256 && (threadIdx.x & 31) == (__ffs(peers) - 1)) atomicAdd(&hist[digit], __popc(peers));
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int cum = 0, d = 255;
-      for (; d > 0; --d) {
-        if (cum + hist[d] >= remaining) break;
-        cum += hist[d];
+    // digit of the k-th largest candidate: largest d whose suffix count reaches `remaining`
+    // (suffix sums over the 256 bins, Hillis-Steele in shared memory)
+    {
+      const int d = threadIdx.x;
+      if (d < 256) suf[d] = hist[d];
+      if (d == 0) suf[256] = 0;
+      __syncthreads();
+      for (int o = 1; o < 256; o <<= 1) {
+        const int v = (d < 256 && d + o < 256) ? suf[d + o] : 0;
+        __syncthreads();
+        if (d < 256) suf[d] += v;
+        __syncthreads();
       }
-      sh_prefix = prefix | (static_cast<uint32_t>(d) << shift);
-      sh_remaining = remaining - cum;
+      if (d < 256 && ((suf[d] >= remaining && suf[d + 1] < remaining) || (d == 0 && suf[0] < remaining))) {
+        sh_prefix = prefix | (static_cast<uint32_t>(d) << shift);
+        sh_remaining = remaining - suf[d + 1];
+      }
     }
     __syncthreads();
     prefix = sh_prefix;
@@ -205,6 +215,122 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
       ++erank;
     }
     if (take) op[pos++] = i;
+  }
+}
+
+// ---- Top-K of one large segment (per-network ranking) spread over many blocks ------------
+// Same radix select, but every pass is a grid-wide histogram followed by a one-block digit
+// pick, and the order-preserving compaction uses per-block counts and a scan over them.
+struct TopkState {
+  uint32_t prefix, mask;
+  int remaining, pad;
+};
+static const int BIG_CHUNK = 4096;      // keys per block in the count / write kernels
+
+__global__ void topk_big_init_kernel(TopkState* st, int k, int* ghist) {
+  if (threadIdx.x < 256) ghist[threadIdx.x] = 0;
+  if (threadIdx.x == 0) {
+    st->prefix = 0; st->mask = 0; st->remaining = k; st->pad = 0;
+  }
+}
+__global__ void __launch_bounds__(256) topk_big_hist_kernel(const float* __restrict__ keys, int n,
+                                                            const TopkState* __restrict__ st, int shift,
+                                                            int* __restrict__ ghist) {
+  __shared__ int sh[256];
+  sh[threadIdx.x] = 0;
+  __syncthreads();
+  const uint32_t prefix = st->prefix, mask = st->mask;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const uint32_t kb = key_bits(keys[i]);
+    if ((kb & mask) == prefix) atomicAdd(&sh[(kb >> shift) & 255], 1);
+  }
+  __syncthreads();
+  if (sh[threadIdx.x]) atomicAdd(&ghist[threadIdx.x], sh[threadIdx.x]);
+}
+__global__ void __launch_bounds__(256) topk_big_pick_kernel(TopkState* st, int shift, int* ghist) {
+  __shared__ int suf[257];
+  const int d = threadIdx.x;
+  suf[d] = ghist[d];
+  if (d == 0) suf[256] = 0;
+  __syncthreads();
+  // inclusive suffix sums: suf[d] = number of candidate keys whose digit is >= d
+  for (int o = 1; o < 256; o <<= 1) {
+    const int v = (d + o < 256) ? suf[d + o] : 0;
+    __syncthreads();
+    suf[d] += v;
+    __syncthreads();
+  }
+  const int remaining = st->remaining;
+  __syncthreads();
+  const bool mine = suf[d] >= remaining && suf[d + 1] < remaining;
+  if (mine || (d == 0 && suf[0] < remaining)) {
+    st->prefix |= static_cast<uint32_t>(d) << shift;
+    st->mask |= 255u << shift;
+    st->remaining = remaining - suf[d + 1];
+  }
+  ghist[d] = 0;
+}
+__global__ void __launch_bounds__(TOPK_THREADS) topk_big_count_kernel(const float* __restrict__ keys, int n,
+                                                                      const TopkState* __restrict__ st,
+                                                                      int* __restrict__ counts) {
+  __shared__ int red[2][32];
+  const uint32_t thr = st->prefix;
+  const int lo = blockIdx.x * BIG_CHUNK, hi = min(n, lo + BIG_CHUNK);
+  int gt = 0, eq = 0;
+  for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+    const uint32_t kb = key_bits(keys[i]);
+    gt += kb > thr;
+    eq += kb == thr;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    gt += __shfl_xor_sync(0xffffffffu, gt, o);
+    eq += __shfl_xor_sync(0xffffffffu, eq, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = gt; red[1][threadIdx.x >> 5] = eq; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int a = 0, b = 0;
+    for (int w = 0; w < 32; ++w) { a += red[0][w]; b += red[1][w]; }
+    counts[2 * blockIdx.x] = a;
+    counts[2 * blockIdx.x + 1] = b;
+  }
+}
+__global__ void topk_big_scan_kernel(const int* __restrict__ counts, int blocks, int* __restrict__ offs) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int a = 0, b = 0;
+  for (int i = 0; i < blocks; ++i) {
+    offs[2 * i] = a;
+    offs[2 * i + 1] = b;
+    a += counts[2 * i];
+    b += counts[2 * i + 1];
+  }
+}
+__global__ void __launch_bounds__(TOPK_THREADS) topk_big_write_kernel(const float* __restrict__ keys, int n,
+                                                                      const TopkState* __restrict__ st,
+                                                                      const int* __restrict__ offs,
+                                                                      int32_t* __restrict__ out) {
+  __shared__ int scan_sh[64];
+  __shared__ int carry[2];
+  const uint32_t thr = st->prefix;
+  const int R = st->remaining;
+  const int lo = blockIdx.x * BIG_CHUNK, hi = min(n, lo + BIG_CHUNK);
+  if (threadIdx.x == 0) { carry[0] = offs[2 * blockIdx.x]; carry[1] = offs[2 * blockIdx.x + 1]; }
+  __syncthreads();
+  for (int base = lo; base < hi; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    int gt = 0, eq = 0;
+    if (i < hi) {
+      const uint32_t kb = key_bits(keys[i]);
+      gt = kb > thr;
+      eq = kb == thr;
+    }
+    int pg, pe;
+    block_scan2(gt, eq, pg, pe, scan_sh);
+    const int g_before = carry[0] + pg, e_before = carry[1] + pe;
+    if (gt || (eq && e_before < R)) out[g_before + min(e_before, R)] = i;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) { carry[0] = g_before + gt; carry[1] = e_before + eq; }
+    __syncthreads();
   }
 }
 
@@ -267,6 +393,10 @@ struct SelectWs {
   float* layer_keys;
   int32_t* lsel;
   int32_t* keep;
+  TopkState* big_state;
+  int* big_hist;
+  int* big_counts;
+  int* big_offs;
   size_t bytes;
 };
 
@@ -286,6 +416,11 @@ static SelectWs carve(void* ws, int L, int64_t total) {
   w.layer_keys = reinterpret_cast<float*>(take(sizeof(float) * static_cast<size_t>(L)));
   w.lsel = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * static_cast<size_t>(L)));
   w.keep = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * static_cast<size_t>(L)));
+  const size_t big_blocks = static_cast<size_t>(ceil_div(total, BIG_CHUNK));
+  w.big_state = reinterpret_cast<TopkState*>(take(sizeof(TopkState)));
+  w.big_hist = reinterpret_cast<int*>(take(256 * sizeof(int)));
+  w.big_counts = reinterpret_cast<int*>(take(2 * big_blocks * sizeof(int)));
+  w.big_offs = reinterpret_cast<int*>(take(2 * big_blocks * sizeof(int)));
   w.bytes = off;
   return w;
 }
@@ -354,8 +489,24 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
     if (importance) cudaMemcpyAsync(importance, w.keys, sizeof(float) * total, cudaMemcpyDeviceToDevice, st);
   } else if (mode == EFQAT_CWPN) {
     const int kt = static_cast<int>(k[0]);
-    count_launches(2);
-    topk_kernel<<<1, TOPK_THREADS, 0, st>>>(w.keys, nullptr, tot, kt, w.sel);
+    if (tot > 4 * BIG_CHUNK && kt > 0) {
+      const int blocks = static_cast<int>(ceil_div(tot, BIG_CHUNK));
+      int hgrid = static_cast<int>(ceil_div(tot, 256 * 4));
+      if (hgrid > 148 * 4) hgrid = 148 * 4;
+      count_launches(13);
+      topk_big_init_kernel<<<1, 256, 0, st>>>(w.big_state, kt, w.big_hist);
+      for (int shift = 24; shift >= 0; shift -= 8) {
+        topk_big_hist_kernel<<<hgrid, 256, 0, st>>>(w.keys, tot, w.big_state, shift, w.big_hist);
+        topk_big_pick_kernel<<<1, 256, 0, st>>>(w.big_state, shift, w.big_hist);
+      }
+      topk_big_count_kernel<<<blocks, TOPK_THREADS, 0, st>>>(w.keys, tot, w.big_state, w.big_counts);
+      topk_big_scan_kernel<<<1, 32, 0, st>>>(w.big_counts, blocks, w.big_offs);
+      topk_big_write_kernel<<<blocks, TOPK_THREADS, 0, st>>>(w.keys, tot, w.big_state, w.big_offs, w.sel);
+    } else {
+      count_launches(1);
+      topk_kernel<<<1, TOPK_THREADS, 0, st>>>(w.keys, nullptr, tot, kt, w.sel);
+    }
+    count_launches(1);
     const int work = (kt > L + 1) ? kt : L + 1;
     cwpn_split_kernel<<<static_cast<unsigned>(ceil_div(work, 256)), 256, 0, st>>>(w.table, L, w.sel, kt, idx,
                                                                                  offsets);

@@ -167,7 +167,7 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
 }
 
 template <int W_MODE, typename TX>
-__global__ void __launch_bounds__(256) prepare_kernel(const PrepArgs a) {
+__global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
   __shared__ float sh[8 * 256];
   const int b = blockIdx.x;
   if (b < a.nb_w) {

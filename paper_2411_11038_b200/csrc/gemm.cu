@@ -605,7 +605,7 @@ int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
   int64_t s = ceil_div(sm_count, tiles);
   const int64_t max_s = nkb / 4 > 0 ? nkb / 4 : 1;   // at least four contraction blocks per split
   if (s > max_s) s = max_s;
-  if (s > 64) s = 64;
+  if (s > sm_count) s = sm_count;
   if (s < 1) s = 1;
   return static_cast<int>(s);
 }

@@ -116,6 +116,7 @@ def main():
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--out", default=None)
+    ap.add_argument("--only", default=None, help="run only layers whose name contains this string")
     args = ap.parse_args()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
@@ -130,6 +131,8 @@ def main():
             if cfg == 5:
                 cases = cases + I.config5(4, 4)
             recs = []
+            if args.only:
+                cases = [c for c in cases if args.only in c.name]
             for c in cases:
                 recs.append(sweep_layer(ctx, c, FRACS[cfg], timer, dev))
                 torch.cuda.empty_cache()

@@ -92,17 +92,44 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
   int pos[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) pos[j] = -1;
-  if (gather && col_ok) {
-    // compact position of each of this thread's columns: binary search in the ascending idx
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int c = static_cast<int>(c0) + j;
+  if (gather) {
+    // Compact position of each of this thread's 8 consecutive columns in the ascending idx:
+    // one binary search for the first column, then a merge walk.  The slice of idx that this
+    // block's 256 columns can hit is staged in shared memory first (it holds at most 256 entries).
+    __shared__ int s_lo, s_cnt;
+    __shared__ int32_t s_idx[256];
+    if (threadIdx.x == 0) {
+      const int cfirst = cb * 256;
       int lo = 0, hi = static_cast<int>(a.k_sel);
       while (lo < hi) {
         const int mid = (lo + hi) >> 1;
-        if (a.idx[mid] < c) lo = mid + 1; else hi = mid;
+        if (a.idx[mid] < cfirst) lo = mid + 1; else hi = mid;
       }
-      if (lo < a.k_sel && a.idx[lo] == c) pos[j] = lo;
+      s_lo = lo;
+      int l2 = lo, h2 = static_cast<int>(a.k_sel);
+      while (l2 < h2) {
+        const int mid = (l2 + h2) >> 1;
+        if (a.idx[mid] < cfirst + 256) l2 = mid + 1; else h2 = mid;
+      }
+      s_cnt = (l2 - lo > 256) ? 256 : l2 - lo;      // more than 256 only for a broken (non-ascending) idx
+    }
+    __syncthreads();
+    if (threadIdx.x < s_cnt) s_idx[threadIdx.x] = a.idx[s_lo + threadIdx.x];
+    __syncthreads();
+    if (col_ok) {
+      int lo = 0, hi = s_cnt;
+      const int cmin = static_cast<int>(c0);
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (s_idx[mid] < cmin) lo = mid + 1; else hi = mid;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (lo < s_cnt && s_idx[lo] == cmin + j) {
+          pos[j] = s_lo + lo;
+          ++lo;
+        }
+      }
     }
   }
   if (gather && cb == 0 && slab == 0) {

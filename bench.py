@@ -37,8 +37,8 @@ FRACS = (0.0, 0.05, 0.25, 1.0)
 METRIC = "fq-linear step TFLOP/s (select + fwd + partial bwd); bwd TFLOP/s and speedup vs full-QAT bwd per unfrozen % in 'bwd'"
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture of the current kernel exists).
-DOMINANT_TRAFFIC_BYTES = None
+# capture summarised under profiles/ (set to None whenever the kernel changes after a capture).
+DOMINANT_TRAFFIC_BYTES = 28.86e6    # mean over the four dX launches of one step (profiles/gemm_kernel_dx_bench_cfg2.txt)
 
 
 def load_peaks():

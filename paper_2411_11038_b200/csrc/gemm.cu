@@ -53,6 +53,7 @@ struct GemmParams {
   int nkb;            // number of BK blocks along the contraction
   int BN;             // tile columns (multiple of 16, <= 256)
   int stages;
+  int kps;            // k-blocks per stage: one barrier round trip covers kps * 64 contraction elements
   int b_stage_bytes;
   int splits;
   int tiles_m, tiles_n;
@@ -96,7 +97,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms of TMA and UMMA
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
+  const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;     // one k-block of A and B
+  const int stage_bytes = p.kps * sub_bytes;
   uint8_t* out_stg = smem + p.stages * stage_bytes;          // [4 warps][STG_BYTES]
   uint8_t* x_stg = out_stg + 4 * STG_BYTES;                  // [4 warps][2][STG_BYTES]   (EPI_DX)
   SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? 8 * STG_BYTES : 0));
@@ -165,7 +167,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const uint32_t tx = (CTA2 ? 2u : 1u) * (A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : bn_cta * BK * 2));
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
-        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+        // One barrier round trip costs ~0.3 us whatever it carries, so a stage holds several
+        // k-blocks: all of them land on the same full barrier and are released by one commit.
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it) {
+          const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1;
           if (*abort_flag || !mbar_wait(&ctl->empty[s], ph ^ 1)) {
@@ -173,12 +178,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             *abort_flag = 1;
             break;
           }
-          uint8_t* sa = smem + s * stage_bytes;
+          // the leader's barrier collects the bytes of both CTAs of a pair; only the leader arrives on it
+          if (rank == 0) mbar_arrive_expect_tx(&ctl->full[s], tx * nsub);
+         for (int u = 0; u < nsub; ++u) {
+          const int kb = kb0 + u;
+          uint8_t* sa = smem + s * stage_bytes + u * sub_bytes;
           uint8_t* sb = sa + A_STAGE_BYTES;
           if (CTA2) {
-            // the leader's barrier collects the bytes of both CTAs; only the leader arrives on it
             const uint32_t fb = mapa_u32(smem_u32(&ctl->full[s]), 0);
-            if (rank == 0) mbar_arrive_expect_tx(&ctl->full[s], tx);
             if (A_MN) {
               tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
               tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
@@ -192,7 +199,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
             }
           } else if (p.cv.mode == 0) {
-            mbar_arrive_expect_tx(&ctl->full[s], tx);
             if (A_MN) {
               tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
               tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
@@ -207,7 +213,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           } else if (p.cv.mode == 3) {
             // grad-weight: contraction block kb = one box of 64 output pixels; tile rows = (tap, channel)
-            mbar_arrive_expect_tx(&ctl->full[s], tx);
             const int bw = kb % p.cv.tiles_w, bh = (kb / p.cv.tiles_w) % p.cv.tiles_h;
             const int bb = kb / (p.cv.tiles_w * p.cv.tiles_h);
             const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
@@ -222,7 +227,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               tma_load_4d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, w0, h0, b0);
           } else {
             // forward / grad-input: tile rows = one box of 128 pixels; contraction block kb = (tap, 64 channels)
-            mbar_arrive_expect_tx(&ctl->full[s], tx);
             const int tmi = t / p.tiles_n;
             const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
             const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
@@ -240,6 +244,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               tma_load_2d(sb, &tmB, &ctl->full[s], rs * p.cv.C + cc * 64, n0);
             }
           }
+         }
         }
       }
       // Make sure none of this CTA's bulk copies is still in flight when it exits (only
@@ -273,7 +278,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_STRIDE;
-        for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it) {
+          const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1;
           if (*abort_flag || !mbar_wait(&ctl->full[s], ph)) {
@@ -283,7 +289,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+         for (int u = 0; u < nsub; ++u) {
+          const int kb = kb0 + u;
+          const uint32_t a_addr = smem_u32(smem + s * stage_bytes + u * sub_bytes);
           const uint32_t b_addr = a_addr + A_STAGE_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
@@ -296,6 +304,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (CTA2) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
             else umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
           }
+         }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (CTA2) umma_commit_pair(&ctl->empty[s], 3); else umma_commit(&ctl->empty[s]);
         }
@@ -700,10 +709,18 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.chunk_cols = a.out_bf16 ? 64 : 32;
   p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2);
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
-  const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
+  const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;
   const int fixed_bytes = 4 * STG_BYTES + (a.epi == EPI_DX ? 8 * STG_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
                           (a.epi == EPI_FWD ? 2 * 4 * 256 * 4 : 0);
-  int stages = (227 * 1024 - 1024 - fixed_bytes) / stage_bytes;
+  const int ring_bytes = 227 * 1024 - 1024 - fixed_bytes;
+  // k-blocks per stage: as many as still leave three stages (two for the widest tiles), at most 4
+  int kps = ring_bytes / (3 * sub_bytes);
+  if (kps <= 1) kps = (ring_bytes / (2 * sub_bytes) >= 2) ? 2 : 1;
+  if (kps > 4) kps = 4;
+  if (kps > p.nkb) kps = p.nkb;
+  p.kps = kps;
+  const int stage_bytes = kps * sub_bytes;
+  int stages = ring_bytes / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return EFQAT_ERR_SHAPE;
   p.stages = stages;

@@ -100,8 +100,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;     // one k-block of A and B
   const int stage_bytes = p.kps * sub_bytes;
   uint8_t* out_stg = smem + p.stages * stage_bytes;          // [4 warps][STG_BYTES]
-  uint8_t* x_stg = out_stg + 4 * STG_BYTES;                  // [4 warps][2][STG_BYTES]   (EPI_DX)
-  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? 8 * STG_BYTES : 0));
+  uint8_t* x_stg = out_stg + 4 * STG_BYTES;                  // [4 warps][STG_BYTES]      (EPI_DX)
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? 4 * STG_BYTES : 0));
   float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [4 warps][256] (EPI_FWD), warp-private
   float* s_bias = s_scale + 4 * 256;                         // [4 warps][256]
 
@@ -317,7 +317,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------- epilogue (warps 2..5)
     const int q = warp & 3;                  // TMEM lane quarter this warp may read
     uint8_t* my_out = out_stg + q * STG_BYTES;
-    uint8_t* my_x = x_stg + q * 2 * STG_BYTES;
+    uint8_t* my_x = x_stg + q * STG_BYTES;
     const int cc = p.chunk_cols;
     ActQ xq = {};
     if (EPI != EPI_PART) xq = make_actq(p.s_x, p.z_x, p.x_bits, p.x_sym, nullptr);
@@ -359,10 +359,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       if (EPI == EPI_DX && lane == 0) {
         // first X slice of this tile: in flight while the main loop of the tile finishes
-        uint64_t* xb = &ctl->xbar[q][x_it & 1];
+        uint64_t* xb = &ctl->xbar[q][0];
         mbar_arrive_expect_tx(xb, STG_BYTES);
-        if (p.cv.mode != 0) tma_load_4d(my_x + (x_it & 1) * STG_BYTES, &tmX, xb, n0, pw0, ph0, pb0);
-        else tma_load_2d(my_x + (x_it & 1) * STG_BYTES, &tmX, xb, n0, row0);
+        if (p.cv.mode != 0) tma_load_4d(my_x, &tmX, xb, n0, pw0, ph0, pb0);
+        else tma_load_2d(my_x, &tmX, xb, n0, row0);
       }
       bool got = *abort_flag ? false : mbar_wait(&ctl->acc_full[buf], (acc_it >> 1) & 1);
       got = __all_sync(0xffffffffu, got);
@@ -396,18 +396,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const float* sc = s_scale + q * 256;
         const float* sb = s_bias + q * 256;
         for (int c0 = 0; c0 < n_eff && ok; c0 += cc) {
-          uint8_t* xs = nullptr;
+          uint4 xr[8];      // this thread's row of the X slice: 8 pieces of 16 bytes
           if (EPI == EPI_DX) {
-            const int xb_i = x_it & 1;
-            if (lane == 0 && c0 + cc < n_eff) {       // prefetch the next slice of this tile
-              uint64_t* xb = &ctl->xbar[q][xb_i ^ 1];
-              mbar_arrive_expect_tx(xb, STG_BYTES);
-              if (p.cv.mode != 0)
-                tma_load_4d(my_x + (xb_i ^ 1) * STG_BYTES, &tmX, xb, n0 + c0 + cc, pw0, ph0, pb0);
-              else
-                tma_load_2d(my_x + (xb_i ^ 1) * STG_BYTES, &tmX, xb, n0 + c0 + cc, row0);
-            }
-            bool gx = mbar_wait(&ctl->xbar[q][xb_i], (x_it >> 1) & 1);
+            bool gx = mbar_wait(&ctl->xbar[q][0], x_it & 1);
             gx = __all_sync(0xffffffffu, gx);
             if (!gx) {
               record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
@@ -415,15 +406,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               ok = false;
               break;
             }
-            xs = my_x + xb_i * STG_BYTES;
             ++x_it;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) xr[i] = *reinterpret_cast<const uint4*>(stg_addr(my_x, lane, i));
+            __syncwarp();
+            // the slice now lives in registers: fetch the next one of this tile behind the math
+            if (lane == 0 && c0 + cc < n_eff) {
+              uint64_t* xb = &ctl->xbar[q][0];
+              mbar_arrive_expect_tx(xb, STG_BYTES);
+              if (p.cv.mode != 0) tma_load_4d(my_x, &tmX, xb, n0 + c0 + cc, pw0, ph0, pb0);
+              else tma_load_2d(my_x, &tmX, xb, n0 + c0 + cc, row0);
+            }
           }
           // the previous TMA store must have finished reading the staging slice
           if (lane == 0) tma_store_wait_read0();
           __syncwarp();
-          for (int h = 0; h < cc; h += 32) {
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const int h = hh * 32;
             const int left = n_eff - c0 - h;
-            if (left <= 0) break;
+            if (h >= cc || left <= 0) break;
             uint32_t r[32];
             const int ncols = (left >= 32) ? 32 : 16;
             if (ncols == 32) tmem_ld_32x32(t_row + c0 + h, r); else tmem_ld_32x16(t_row + c0 + h, r);
@@ -441,7 +443,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 } else {
                   float x[8];
                   if (cc == 64) {      // bf16 activations: 8 values in one 16-byte piece
-                    const uint4 u = *reinterpret_cast<const uint4*>(stg_addr(xs, lane, (h >> 3) + g));
+                    const uint4 u = xr[hh * 4 + g];
                     const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
@@ -449,10 +451,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                       x[2 * i + 1] = __uint_as_float(wv[i] & 0xffff0000u);
                     }
                   } else {             // fp32 activations: two 16-byte pieces
-                    const float4 a = *reinterpret_cast<const float4*>(stg_addr(xs, lane, 2 * g));
-                    const float4 b = *reinterpret_cast<const float4*>(stg_addr(xs, lane, 2 * g + 1));
-                    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-                    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+                    const uint4 a = xr[(2 * g) & 7], b = xr[(2 * g + 1) & 7];
+                    x[0] = __uint_as_float(a.x); x[1] = __uint_as_float(a.y);
+                    x[2] = __uint_as_float(a.z); x[3] = __uint_as_float(a.w);
+                    x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y);
+                    x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
                   }
 #pragma unroll
                   for (int j = 0; j < 8; ++j) {
@@ -710,7 +713,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2);
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
   const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;
-  const int fixed_bytes = 4 * STG_BYTES + (a.epi == EPI_DX ? 8 * STG_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
+  const int fixed_bytes = 4 * STG_BYTES + (a.epi == EPI_DX ? 4 * STG_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
                           (a.epi == EPI_FWD ? 2 * 4 * 256 * 4 : 0);
   const int ring_bytes = 227 * 1024 - 1024 - fixed_bytes;
   // k-blocks per stage: as many as still leave three stages (two for the widest tiles), at most 4

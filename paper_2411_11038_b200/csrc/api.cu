@@ -97,7 +97,7 @@ int dx_partials(const efqat_layer_desc* l) {
   if (!spatial_conv(l)) return gemm_dx_num_partials(l->M, l->K);
   int tw, th, tb;
   conv_pixel_box(l->W, l->H, l->B, 128, &tw, &th, &tb);
-  return static_cast<int>(ceil_div(l->W, tw) * ceil_div(l->H, th) * ceil_div(l->B, tb) * ceil_div(l->Cin, 64) * 4);
+  return static_cast<int>(ceil_div(l->W, tw) * ceil_div(l->H, th) * ceil_div(l->B, tb) * ceil_div(l->Cin, 64) * 8);
 }
 
 LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, int64_t p_elems_override) {

@@ -31,10 +31,11 @@ static const int UMMA_K = 16;
 static const int MAX_STAGES = 8;
 static const int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB
 static const int CHUNK_BYTES = 64 * BK * 2;     // one 64-wide MN-major chunk, 8 KiB
-static const int GEMM_THREADS = 192;
+static const int EPI_WARPS = 8;
+static const int GEMM_THREADS = 64 + 32 * EPI_WARPS;
 static const int ACC_STRIDE = 256;              // TMEM columns between the two accumulators
 static const int TMEM_COLS = 512;
-static const int STG_BYTES = 32 * 128;          // staging slice of one epilogue warp: 32 rows x 128 B
+static const int HB_BYTES = 32 * 64;            // staging block of one epilogue warp: 32 rows x 64 B
 
 // Convolution geometry as the kernel needs it (mode 0 = plain matrices).
 struct ConvP {
@@ -57,7 +58,8 @@ struct GemmParams {
   int b_stage_bytes;
   int splits;
   int tiles_m, tiles_n;
-  int chunk_cols;     // output columns per 128-byte staging row: 64 (bf16) or 32 (fp32)
+  int blk_cols;       // output columns per 64-byte staging row: 32 (bf16) or 16 (fp32)
+  int out_bufs;       // staging buffers per epilogue warp (2 when shared memory allows)
   const float* col_scale;
   const float* col_bias;
   const float* s_x; const float* z_x; int x_bits, x_sym;
@@ -74,7 +76,7 @@ struct __align__(8) SmemCtl {
   uint64_t empty[MAX_STAGES];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
-  uint64_t xbar[4][2];
+  uint64_t xbar[EPI_WARPS];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -84,9 +86,9 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// 16-byte piece `piece` (0..7) of row `row` (0..31) inside a 128-byte-swizzled staging slice.
-__device__ __forceinline__ uint8_t* stg_addr(uint8_t* base, int row, int piece) {
-  return base + row * 128 + ((piece ^ (row & 7)) << 4);
+// 16-byte piece `piece` (0..3) of row `row` (0..31) inside a 64-byte-swizzled staging block.
+__device__ __forceinline__ uint8_t* stg64_addr(uint8_t* base, int row, int piece) {
+  return base + row * 64 + ((piece ^ ((row >> 1) & 3)) << 4);
 }
 
 template <int A_MN, int B_MN, int EPI, int CTA2>
@@ -99,11 +101,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;     // one k-block of A and B
   const int stage_bytes = p.kps * sub_bytes;
-  uint8_t* out_stg = smem + p.stages * stage_bytes;          // [4 warps][STG_BYTES]
-  uint8_t* x_stg = out_stg + 4 * STG_BYTES;                  // [4 warps][STG_BYTES]      (EPI_DX)
-  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? 4 * STG_BYTES : 0));
-  float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [4 warps][256] (EPI_FWD), warp-private
-  float* s_bias = s_scale + 4 * 256;                         // [4 warps][256]
+  uint8_t* out_stg = smem + p.stages * stage_bytes;          // [8 warps][out_bufs][HB_BYTES]
+  uint8_t* x_stg = out_stg + (EPI == EPI_PART ? 0 : EPI_WARPS * p.out_bufs * HB_BYTES);   // [8 warps][HB_BYTES] (EPI_DX)
+  SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? EPI_WARPS * HB_BYTES : 0));
+  float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [8 warps][128 scales, 128 biases] (EPI_FWD), warp-private
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_mn = p.tiles_m * p.tiles_n;
@@ -122,12 +123,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&ctl->acc_full[b], 1);
-      mbar_init(&ctl->acc_empty[b], CTA2 ? 8 : 4);
+      mbar_init(&ctl->acc_empty[b], (CTA2 ? 2 : 1) * EPI_WARPS);
     }
-    for (int w = 0; w < 4; ++w) {
-      mbar_init(&ctl->xbar[w][0], 1);
-      mbar_init(&ctl->xbar[w][1], 1);
-    }
+    for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&ctl->xbar[w], 1);
     ctl->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmA);
@@ -314,55 +312,94 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     }
   } else {
-    // ------------------------------------------------------------- epilogue (warps 2..5)
-    const int q = warp & 3;                  // TMEM lane quarter this warp may read
-    uint8_t* my_out = out_stg + q * STG_BYTES;
-    uint8_t* my_x = x_stg + q * STG_BYTES;
-    const int cc = p.chunk_cols;
+    // ------------------------------------------------------------- epilogue (warps 2..9)
+    // Warp e = warp - 2 reads TMEM lane quarter q = warp % 4 (the quarter the hardware lets
+    // it read) and owns one half of the tile's column blocks.  A block is 64 bytes of output
+    // columns (32 bf16 / 16 fp32): small enough that two staging buffers per warp fit, so the
+    // TMA store of one block drains while the next one is computed.
+    const int e = warp - 2;
+    const int q = warp & 3;
+    const int half = e >> 2;
+    const int bc = p.blk_cols;
+    uint8_t* my_out = out_stg + e * p.out_bufs * HB_BYTES;
+    uint8_t* my_x = x_stg + e * HB_BYTES;
+    float* my_sc = s_scale + e * 256;          // [128] scales then [128] biases of this warp's columns
     ActQ xq = {};
     if (EPI != EPI_PART) xq = make_actq(p.s_x, p.z_x, p.x_bits, p.x_sym, nullptr);
-    int acc_it = 0;
-    int x_it = 0;                            // X slices consumed so far by this warp (EPI_DX)
-    bool ok = true;
-    for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
-      const int split = w / tiles_mn, t = w - split * tiles_mn;
-      const int m0 = (t / p.tiles_n) * TILE_M + rank * BM, n0 = (t % p.tiles_n) * p.BN;
-      int n_eff = static_cast<int>(p.Nc - n0);
+
+    struct Geo {
+      int t, split, n0, n_eff, row0, jb0, jb1, pw0, ph0, pb0;
+      bool rows_live;
+    };
+    auto geo_of = [&](int w) {
+      Geo g;
+      g.split = w / tiles_mn;
+      g.t = w - g.split * tiles_mn;
+      const int m0 = (g.t / p.tiles_n) * TILE_M + rank * BM;
+      g.n0 = (g.t % p.tiles_n) * p.BN;
+      int n_eff = static_cast<int>(p.Nc - g.n0);
       if (n_eff > p.BN) n_eff = p.BN;
-      n_eff = (n_eff + 15) & ~15;
-      const int buf = acc_it & 1;
-      const int row0 = m0 + q * 32;
-      // convolution: this warp's 32 rows are a sub-box of the tile's pixel box
-      int pw0 = 0, ph0 = 0, pb0 = 0;
-      bool rows_live = row0 < p.Mr;
+      g.n_eff = (n_eff + 15) & ~15;
+      const int bw_cols = (EPI == EPI_PART) ? 32 : bc;
+      const int nblk = (g.n_eff + bw_cols - 1) / bw_cols;
+      const int nb0 = (nblk + 1) >> 1;
+      g.jb0 = half ? nb0 : 0;
+      g.jb1 = half ? nblk : nb0;
+      g.row0 = m0 + q * 32;
+      g.pw0 = g.ph0 = g.pb0 = 0;
+      g.rows_live = g.row0 < p.Mr;
       if (EPI != EPI_PART && p.cv.mode != 0) {
-        const int tmi = t / p.tiles_n;
+        // convolution: this warp's 32 rows are a sub-box of the tile's pixel box
+        const int tmi = g.t / p.tiles_n;
         const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
         const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
         const int pix = q * 32;
-        pw0 = bw * p.cv.tw;
-        ph0 = bh * p.cv.th + (pix / p.cv.tw) % p.cv.th;
-        pb0 = bb * p.cv.tb + pix / (p.cv.tw * p.cv.th);
-        rows_live = ph0 < p.cv.dimH && pb0 < p.cv.dimB;
+        g.pw0 = bw * p.cv.tw;
+        g.ph0 = bh * p.cv.th + (pix / p.cv.tw) % p.cv.th;
+        g.pb0 = bb * p.cv.tb + pix / (p.cv.tw * p.cv.th);
+        g.rows_live = g.ph0 < p.cv.dimH && g.pb0 < p.cv.dimB;
       }
+      return g;
+    };
+    auto fetch_x = [&](const Geo& g, int jb) {     // lane 0: one 32-row x 64-byte block of X
+      uint64_t* xb = &ctl->xbar[e];
+      mbar_arrive_expect_tx(xb, HB_BYTES);
+      if (p.cv.mode != 0) tma_load_4d(my_x, &tmX, xb, g.n0 + jb * bc, g.pw0, g.ph0, g.pb0);
+      else tma_load_2d(my_x, &tmX, xb, g.n0 + jb * bc, g.row0);
+    };
+
+    int acc_it = 0;
+    int x_it = 0;                            // X blocks consumed so far by this warp (EPI_DX)
+    int st_it = 0;                           // output blocks staged so far by this warp
+    bool ok = true;
+    Geo g = {};
+    if (unit < total_items) {
+      g = geo_of(unit);
+      if (EPI == EPI_DX && lane == 0 && g.jb0 < g.jb1) fetch_x(g, g.jb0);
       if (EPI == EPI_FWD) {
-        // this warp's own copy of the tile's column scales and biases (no cross-warp barrier)
-        float* sc = s_scale + q * 256;
-        float* sb = s_bias + q * 256;
-        __syncwarp();
-        for (int j = lane; j < p.BN; j += 32) {
-          const int64_t c = static_cast<int64_t>(n0) + j;
-          sc[j] = (c < p.Nc) ? p.col_scale[c] : 0.f;
-          sb[j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
+        for (int j = lane; j < 128; j += 32) {
+          const int64_t c = static_cast<int64_t>(g.n0) + g.jb0 * bc + j;
+          my_sc[j] = (c < p.Nc) ? p.col_scale[c] : 0.f;
+          my_sc[128 + j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
         }
         __syncwarp();
       }
-      if (EPI == EPI_DX && lane == 0) {
-        // first X slice of this tile: in flight while the main loop of the tile finishes
-        uint64_t* xb = &ctl->xbar[q][0];
-        mbar_arrive_expect_tx(xb, STG_BYTES);
-        if (p.cv.mode != 0) tma_load_4d(my_x, &tmX, xb, n0, pw0, ph0, pb0);
-        else tma_load_2d(my_x, &tmX, xb, n0, row0);
+    }
+    for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
+      const bool has_next = w + num_units < total_items;
+      const Geo gn = has_next ? geo_of(w + num_units) : g;
+      const int buf = acc_it & 1;
+      // next tile's column scales and biases: loaded now, parked in registers behind this tile's work
+      float nsc[4] = {0.f, 0.f, 0.f, 0.f}, nbi[4] = {0.f, 0.f, 0.f, 0.f};
+      if (EPI == EPI_FWD && has_next) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int64_t c = static_cast<int64_t>(gn.n0) + gn.jb0 * bc + lane + 32 * i;
+          if (c < p.Nc) {
+            nsc[i] = p.col_scale[c];
+            if (p.col_bias) nbi[i] = p.col_bias[c];
+          }
+        }
       }
       bool got = *abort_flag ? false : mbar_wait(&ctl->acc_full[buf], (acc_it >> 1) & 1);
       got = __all_sync(0xffffffffu, got);
@@ -377,28 +414,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       float acc_s = 0.f, acc_z = 0.f;
 
       if (EPI == EPI_PART) {
-        const int64_t row = static_cast<int64_t>(row0) + lane;
-        for (int c0 = 0; c0 < n_eff; c0 += 32) {
+        const int64_t row = static_cast<int64_t>(g.row0) + lane;
+        for (int jb = g.jb0; jb < g.jb1; ++jb) {
+          const int c0 = jb * 32;
           uint32_t r[32];
-          const int ncols = (n_eff - c0 >= 32) ? 32 : 16;
+          const int ncols = (g.n_eff - c0 >= 32) ? 32 : 16;
           if (ncols == 32) tmem_ld_32x32(t_row + c0, r); else tmem_ld_32x16(t_row + c0, r);
           tmem_wait_ld();
           if (row < p.Mr) {
-            float* outp = p.out + split * p.split_stride + row;
+            float* outp = p.out + g.split * p.split_stride + row;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int64_t col = static_cast<int64_t>(n0) + c0 + j;
+              const int64_t col = static_cast<int64_t>(g.n0) + c0 + j;
               if (j < ncols && col < p.part_cols) outp[col * p.ldo] = __uint_as_float(r[j]);
             }
           }
         }
       } else {
-        const float* sc = s_scale + q * 256;
-        const float* sb = s_bias + q * 256;
-        for (int c0 = 0; c0 < n_eff && ok; c0 += cc) {
-          uint4 xr[8];      // this thread's row of the X slice: 8 pieces of 16 bytes
+        for (int jb = g.jb0; jb < g.jb1 && ok; ++jb) {
+          const int c0 = jb * bc;
+          const int left = g.n_eff - c0;
+          const int ncols = (left >= 32 && bc == 32) ? 32 : 16;
+          uint4 xr[4];      // this thread's row of the X block: 4 pieces of 16 bytes
           if (EPI == EPI_DX) {
-            bool gx = mbar_wait(&ctl->xbar[q][0], x_it & 1);
+            bool gx = mbar_wait(&ctl->xbar[e], x_it & 1);
             gx = __all_sync(0xffffffffu, gx);
             if (!gx) {
               record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
@@ -408,83 +447,78 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             ++x_it;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) xr[i] = *reinterpret_cast<const uint4*>(stg_addr(my_x, lane, i));
+            for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const uint4*>(stg64_addr(my_x, lane, i));
             __syncwarp();
-            // the slice now lives in registers: fetch the next one of this tile behind the math
-            if (lane == 0 && c0 + cc < n_eff) {
-              uint64_t* xb = &ctl->xbar[q][0];
-              mbar_arrive_expect_tx(xb, STG_BYTES);
-              if (p.cv.mode != 0) tma_load_4d(my_x, &tmX, xb, n0 + c0 + cc, pw0, ph0, pb0);
-              else tma_load_2d(my_x, &tmX, xb, n0 + c0 + cc, row0);
+            // the block now lives in registers: fetch the next one (of this or the next tile) behind the math
+            if (lane == 0) {
+              if (jb + 1 < g.jb1) fetch_x(g, jb + 1);
+              else if (has_next && gn.jb0 < gn.jb1) fetch_x(gn, gn.jb0);
             }
           }
-          // the previous TMA store must have finished reading the staging slice
-          if (lane == 0) tma_store_wait_read0();
+          uint32_t r[32];
+          if (ncols == 32) tmem_ld_32x32(t_row + c0, r); else tmem_ld_32x16(t_row + c0, r);
+          // the TMA store that last used this staging buffer must have finished reading it
+          uint8_t* ob = my_out + (p.out_bufs == 2 ? (st_it & 1) * HB_BYTES : 0);
+          if (lane == 0) {
+            if (p.out_bufs == 2) tma_store_wait_read1(); else tma_store_wait_read0();
+          }
+          ++st_it;
+          tmem_wait_ld();
           __syncwarp();
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            const int h = hh * 32;
-            const int left = n_eff - c0 - h;
-            if (h >= cc || left <= 0) break;
-            uint32_t r[32];
-            const int ncols = (left >= 32) ? 32 : 16;
-            if (ncols == 32) tmem_ld_32x32(t_row + c0 + h, r); else tmem_ld_32x16(t_row + c0 + h, r);
-            tmem_wait_ld();
+          for (int gi = 0; gi < 4; ++gi) {
+            if (gi * 8 < ncols) {
+              float v[8];
+              if (EPI == EPI_FWD) {
+                const int cj = (jb - g.jb0) * bc + gi * 8;
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              if (g * 8 < ncols) {
-                float v[8];
-                if (EPI == EPI_FWD) {
+                for (int j = 0; j < 8; ++j)
+                  v[j] = fmaf(__uint_as_float(r[gi * 8 + j]) * xq.s, my_sc[cj + j], my_sc[128 + cj + j]);
+              } else {
+                float x[8];
+                if (bc == 32) {      // bf16 activations: 8 values in one 16-byte piece
+                  const uint4 u = xr[gi];
+                  const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-                  for (int j = 0; j < 8; ++j) {
-                    const int cj = c0 + h + g * 8 + j;
-                    v[j] = fmaf(__uint_as_float(r[g * 8 + j]) * xq.s, sc[cj], sb[cj]);
+                  for (int i = 0; i < 4; ++i) {
+                    x[2 * i] = __uint_as_float(wv[i] << 16);
+                    x[2 * i + 1] = __uint_as_float(wv[i] & 0xffff0000u);
                   }
-                } else {
-                  float x[8];
-                  if (cc == 64) {      // bf16 activations: 8 values in one 16-byte piece
-                    const uint4 u = xr[hh * 4 + g];
-                    const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                      x[2 * i] = __uint_as_float(wv[i] << 16);
-                      x[2 * i + 1] = __uint_as_float(wv[i] & 0xffff0000u);
-                    }
-                  } else {             // fp32 activations: two 16-byte pieces
-                    const uint4 a = xr[(2 * g) & 7], b = xr[(2 * g + 1) & 7];
-                    x[0] = __uint_as_float(a.x); x[1] = __uint_as_float(a.y);
-                    x[2] = __uint_as_float(a.z); x[3] = __uint_as_float(a.w);
-                    x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y);
-                    x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
-                  }
-#pragma unroll
-                  for (int j = 0; j < 8; ++j) {
-                    const float gx = __uint_as_float(r[g * 8 + j]);
-                    const QElem e = quant_act(x[j], xq);
-                    v[j] = e.flag ? 0.f : gx;
-                    acc_s = fmaf(gx, e.t, acc_s);
-                    acc_z += e.flag ? -gx * xq.s : 0.f;
-                  }
+                } else {             // fp32 activations: two 16-byte pieces
+                  const uint4 a = xr[(2 * gi) & 3], b = xr[(2 * gi + 1) & 3];
+                  x[0] = __uint_as_float(a.x); x[1] = __uint_as_float(a.y);
+                  x[2] = __uint_as_float(a.z); x[3] = __uint_as_float(a.w);
+                  x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y);
+                  x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
                 }
-                if (cc == 64) {
-                  uint4 o;
-                  o.x = pack2(v[0], v[1]); o.y = pack2(v[2], v[3]);
-                  o.z = pack2(v[4], v[5]); o.w = pack2(v[6], v[7]);
-                  *reinterpret_cast<uint4*>(stg_addr(my_out, lane, (h >> 3) + g)) = o;
-                } else {
-                  *reinterpret_cast<float4*>(stg_addr(my_out, lane, 2 * g)) = make_float4(v[0], v[1], v[2], v[3]);
-                  *reinterpret_cast<float4*>(stg_addr(my_out, lane, 2 * g + 1)) =
-                      make_float4(v[4], v[5], v[6], v[7]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float gx = __uint_as_float(r[gi * 8 + j]);
+                  const QElem qe = quant_act(x[j], xq);
+                  v[j] = qe.flag ? 0.f : gx;
+                  acc_s = fmaf(gx, qe.t, acc_s);
+                  acc_z += qe.flag ? -gx * xq.s : 0.f;
                 }
+              }
+              if (bc == 32) {
+                uint4 o;
+                o.x = pack2(v[0], v[1]); o.y = pack2(v[2], v[3]);
+                o.z = pack2(v[4], v[5]); o.w = pack2(v[6], v[7]);
+                *reinterpret_cast<uint4*>(stg64_addr(ob, lane, gi)) = o;
+              } else {
+                *reinterpret_cast<float4*>(stg64_addr(ob, lane, 2 * gi)) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4*>(stg64_addr(ob, lane, 2 * gi + 1)) = make_float4(v[4], v[5], v[6], v[7]);
               }
             }
           }
           fence_proxy_async();
           __syncwarp();
-          if (lane == 0 && rows_live && n0 + c0 < p.Nc) {     // stores are clipped at the tensor's edges
-            if (p.cv.mode != 0) tma_store_4d(&tmOut, my_out, n0 + c0, pw0, ph0, pb0);
-            else tma_store_2d(&tmOut, my_out, n0 + c0, row0);
-            tma_store_commit();
+          if (lane == 0) {
+            if (g.rows_live && g.n0 + c0 < p.Nc) {     // stores are clipped at the tensor's edges
+              if (p.cv.mode != 0) tma_store_4d(&tmOut, ob, g.n0 + c0, g.pw0, g.ph0, g.pb0);
+              else tma_store_2d(&tmOut, ob, g.n0 + c0, g.row0);
+            }
+            tma_store_commit();     // always: the buffer rotation counts committed groups
           }
         }
       }
@@ -499,11 +533,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         acc_s = warp_sum(acc_s);
         acc_z = warp_sum(acc_z);
         if (lane == 0) {
-          float* pp = p.partials + ((static_cast<int64_t>(t) * (CTA2 ? 2 : 1) + rank) * 4 + q) * 2;
+          float* pp = p.partials + ((static_cast<int64_t>(g.t) * (CTA2 ? 2 : 1) + rank) * EPI_WARPS + e) * 2;
           pp[0] = acc_s;
           pp[1] = acc_z;
         }
       }
+      if (EPI == EPI_FWD && has_next) {
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          my_sc[lane + 32 * i] = nsc[i];
+          my_sc[128 + lane + 32 * i] = nbi[i];
+        }
+        __syncwarp();
+      }
+      g = gn;
     }
     if (EPI != EPI_PART && lane == 0) tma_store_wait_all();
   }
@@ -532,35 +576,38 @@ int gemm_init() {
   return EFQAT_OK;
 }
 
-// 2-D row-major matrix [rows, cols] with pitch ld (elements); box = 128 bytes of columns x box_rows rows.
+// 2-D row-major matrix [rows, cols] with pitch ld (elements); box = row_bytes (128 or 64, the
+// swizzle span) of columns x box_rows rows.
 static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
-                    int box_rows) {
+                    int box_rows, int row_bytes = 128) {
   const int es = is_bf16 ? 2 : 4;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * es};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / es), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(row_bytes / es), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estr[2] = {1u, 1u};
   const CUresult r = g_encode(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
-// 4-D NHWC tensor [B,H,W,C] (pitch C elements per pixel); box = 128 bytes of channels x bw x bh x bb pixels.
+// 4-D NHWC tensor [B,H,W,C] (pitch C elements per pixel); box = row_bytes (128 or 64) of channels x bw x bh x bb pixels.
 static int make_map_4d(CUtensorMap* m, const void* base, int is_bf16, int64_t B, int64_t H, int64_t W, int64_t C,
-                       int64_t pitch, int bw, int bh, int bb) {
+                       int64_t pitch, int bw, int bh, int bb, int row_bytes = 128) {
   const int es = is_bf16 ? 2 : 4;
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
                               static_cast<cuuint64_t>(B)};
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(pitch) * es, static_cast<cuuint64_t>(pitch) * W * es,
                                  static_cast<cuuint64_t>(pitch) * W * H * es};
-  const cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / es), static_cast<cuuint32_t>(bw),
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(row_bytes / es), static_cast<cuuint32_t>(bw),
                              static_cast<cuuint32_t>(bh), static_cast<cuuint32_t>(bb)};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   const CUresult r = g_encode(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
                               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
@@ -603,8 +650,8 @@ static int choose_bn(int64_t Mr, int64_t Nc, int sm_count) {
 }
 
 int gemm_dx_num_partials(int64_t Mr, int64_t Nc) {
-  // upper bound over every tile width the heuristic may pick: 4 quarter-warps per tile
-  return static_cast<int>(ceil_div(Mr, BM) * ceil_div(Nc, 64) * 4);
+  // upper bound over every tile width the heuristic may pick: 8 epilogue warps per 128-row tile
+  return static_cast<int>(ceil_div(Mr, BM) * ceil_div(Nc, 64) * EPI_WARPS);
 }
 
 static int part_bn(int64_t Nc) {
@@ -674,16 +721,22 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
       p.BN = (cv->Cin % 256 == 0) ? 256 : (cv->Cin % 192 == 0) ? 192 : (cv->Cin % 128 == 0) ? 128 : 64;
     }
   }
-  // CTA pairs (256 x BN tiles) whenever the tiles are full in N: half the B traffic per FLOP
+  // CTA pairs (256 x BN tiles, tiles full in N) halve the B traffic from L2 per FLOP; they are
+  // taken unless one-CTA tiles fill the machine's last wave clearly better.
   int pair = 0;
   if (!cv && a.epi != EPI_PART && a.Mr >= 256 && a.Nc % 128 == 0) {
-    pair = 1;
     const int units = sm_count / 2;
     const int64_t mt = ceil_div(a.Mr, 2 * BM);
     const bool can256 = a.Nc % 256 == 0;
     const double c256 = can256 ? static_cast<double>(ceil_div(mt * (a.Nc / 256), units)) * (256 + 24) : 1e300;
     const double c128 = static_cast<double>(ceil_div(mt * (a.Nc / 128), units)) * (128 + 24);
-    p.BN = (c256 <= c128) ? 256 : 128;
+    const int bn_pair = (c256 <= c128) ? 256 : 128;
+    const double c_pair = 0.92 * (c256 <= c128 ? c256 : c128);
+    const double c_single = static_cast<double>(ceil_div(ceil_div(a.Mr, BM) * ceil_div(a.Nc, p.BN), sm_count)) * (p.BN + 24);
+    if (c_pair <= c_single) {
+      pair = 1;
+      p.BN = bn_pair;
+    }
   }
   const int bn_cta = pair ? p.BN / 2 : p.BN;
   p.tiles_m = static_cast<int>(ceil_div(a.Mr, pair ? 2 * BM : BM));
@@ -709,12 +762,13 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
       p.nkb = cv->R * cv->S * c.cchunks;
     }
   }
-  p.chunk_cols = a.out_bf16 ? 64 : 32;
+  p.blk_cols = a.out_bf16 ? 32 : 16;
   p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2);
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
   const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;
-  const int fixed_bytes = 4 * STG_BYTES + (a.epi == EPI_DX ? 4 * STG_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
-                          (a.epi == EPI_FWD ? 2 * 4 * 256 * 4 : 0);
+  const int out_stg_bytes = (a.epi == EPI_PART) ? 0 : EPI_WARPS * HB_BYTES;     // one staging buffer per warp
+  int fixed_bytes = out_stg_bytes + (a.epi == EPI_DX ? EPI_WARPS * HB_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
+                    (a.epi == EPI_FWD ? EPI_WARPS * 256 * 4 : 0);
   const int ring_bytes = 227 * 1024 - 1024 - fixed_bytes;
   // k-blocks per stage: as many as still leave three stages (two for the widest tiles), at most 4
   int kps = ring_bytes / (3 * sub_bytes);
@@ -727,6 +781,12 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return EFQAT_ERR_SHAPE;
   p.stages = stages;
+  // a second staging buffer per epilogue warp when the ring leaves room for it
+  p.out_bufs = 1;
+  if (out_stg_bytes && ring_bytes - stages * stage_bytes >= out_stg_bytes) {
+    p.out_bufs = 2;
+    fixed_bytes += out_stg_bytes;
+  }
   p.col_scale = a.col_scale;
   p.col_bias = a.col_bias;
   p.s_x = a.s_x; p.z_x = a.z_x; p.x_bits = a.x_bits; p.x_sym = a.x_sym;
@@ -747,11 +807,11 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
     to = ta;
     tx = ta;
     if (a.epi != EPI_PART) {
-      rc = make_map(&to, a.out, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+      rc = make_map(&to, a.out, a.out_bf16, a.Mr, a.Nc, a.ldo, 32, 64);
       if (rc != EFQAT_OK) return rc;
     }
     if (a.epi == EPI_DX) {
-      rc = make_map(&tx, a.X, a.out_bf16, a.Mr, a.Nc, a.ldo, 32);
+      rc = make_map(&tx, a.X, a.out_bf16, a.Mr, a.Nc, a.ldo, 32, 64);
       if (rc != EFQAT_OK) return rc;
     }
   } else {
@@ -764,15 +824,15 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
       rc = make_map_4d(&ta, a.A, 1, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, c.th, c.tb);
       if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, bn_cta);
       if (rc == EFQAT_OK)
-        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, qh, qb);
+        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, qh, qb, 64);
       tx = ta;
     } else if (cv->mode == 2) {
       rc = make_map_4d(&ta, a.A, 1, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, c.th, c.tb);
       if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, BK);
       if (rc == EFQAT_OK)
-        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb);
+        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb, 64);
       if (rc == EFQAT_OK)
-        rc = make_map_4d(&tx, a.X, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb);
+        rc = make_map_4d(&tx, a.X, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb, 64);
     } else {
       rc = make_map_4d(&ta, a.A, 1, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, c.th, c.tb);
       if (rc == EFQAT_OK) rc = make_map_4d(&tb, a.B, 1, cv->B, cv->Ho, cv->Wo, a.Nc, a.ldb, c.tw, c.th, c.tb);
@@ -787,7 +847,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   const int units = static_cast<int>(items < max_units ? items : max_units);
   const int grid = pair ? 2 * units : units;
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + fixed_bytes + 1024;
-  if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * 4;
+  if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * EPI_WARPS;
 
 #define EFQAT_LAUNCH(AM, BMj, E, P2) return launch<AM, BMj, E, P2>(ta, tb, to, tx, p, grid, smem, st)
   if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) {

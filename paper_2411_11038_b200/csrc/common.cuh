@@ -32,6 +32,13 @@ __device__ __forceinline__ void record_status(int* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
+// Round to nearest, ties to even, through the 1.5 * 2^23 constant: equal to rintf() for
+// |u| < 2^22 and still far outside every code range beyond that, at two full-rate adds
+// (rintf goes through the quarter-rate conversion unit).
+__device__ __forceinline__ float rne_small(float u) {
+  return __fadd_rn(__fadd_rn(u, 12582912.f), -12582912.f);
+}
+
 // Eq. 1 on one element.  The code is decided by u = fl32(x * fl32(1/s)), rounded to
 // nearest-even; the scale gradient uses x/s to roughly fp64 accuracy through the
 // two-term reciprocal (rne(u) - x*rinv is exact in one fma because rne(u) is within

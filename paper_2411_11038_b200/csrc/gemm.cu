@@ -71,7 +71,7 @@ struct GemmParams {
   int* status;
 };
 
-struct __align__(8) SmemCtl {
+struct __align__(16) SmemCtl {
   uint64_t full[MAX_STAGES];
   uint64_t empty[MAX_STAGES];
   uint64_t acc_full[2];
@@ -326,6 +326,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     float* my_sc = s_scale + e * 256;          // [128] scales then [128] biases of this warp's columns
     ActQ xq = {};
     if (EPI != EPI_PART) xq = make_actq(p.s_x, p.z_x, p.x_bits, p.x_sym, nullptr);
+    const float t_lo = xq.lo - xq.zr, t_hi = xq.hi - xq.zr;     // d/ds of a clipped element
 
     struct Geo {
       int t, split, n0, n_eff, row0, jb0, jb1, pw0, ph0, pb0;
@@ -379,7 +380,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (EPI == EPI_FWD) {
         for (int j = lane; j < 128; j += 32) {
           const int64_t c = static_cast<int64_t>(g.n0) + g.jb0 * bc + j;
-          my_sc[j] = (c < p.Nc) ? p.col_scale[c] : 0.f;
+          my_sc[j] = (c < p.Nc) ? p.col_scale[c] * xq.s : 0.f;
           my_sc[128 + j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
         }
         __syncwarp();
@@ -396,7 +397,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int i = 0; i < 4; ++i) {
           const int64_t c = static_cast<int64_t>(gn.n0) + gn.jb0 * bc + lane + 32 * i;
           if (c < p.Nc) {
-            nsc[i] = p.col_scale[c];
+            nsc[i] = p.col_scale[c] * xq.s;
             if (p.col_bias) nbi[i] = p.col_bias[c];
           }
         }
@@ -411,7 +412,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       tc_fence_after();
       const uint32_t t_row = tmem_base + buf * ACC_STRIDE + (static_cast<uint32_t>(q * 32) << 16);
-      float acc_s = 0.f, acc_z = 0.f;
+      float acc_s = 0.f, acc_c = 0.f;
 
       if (EPI == EPI_PART) {
         const int64_t row = static_cast<int64_t>(g.row0) + lane;
@@ -457,6 +458,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           uint32_t r[32];
           if (ncols == 32) tmem_ld_32x32(t_row + c0, r); else tmem_ld_32x16(t_row + c0, r);
+          float4 sc4[8], bi4[8];     // this block's column scales (s_x folded in) and biases
+          if (EPI == EPI_FWD) {
+            const float4* ps = reinterpret_cast<const float4*>(my_sc + (jb - g.jb0) * bc);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (i * 4 < bc) {
+                sc4[i] = ps[i];
+                bi4[i] = ps[32 + i];
+              }
+            }
+          }
           // the TMA store that last used this staging buffer must have finished reading it
           uint8_t* ob = my_out + (p.out_bufs == 2 ? (st_it & 1) * HB_BYTES : 0);
           if (lane == 0) {
@@ -470,10 +482,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (gi * 8 < ncols) {
               float v[8];
               if (EPI == EPI_FWD) {
-                const int cj = (jb - g.jb0) * bc + gi * 8;
+                const float sv[8] = {sc4[2 * gi].x, sc4[2 * gi].y, sc4[2 * gi].z, sc4[2 * gi].w,
+                                     sc4[2 * gi + 1].x, sc4[2 * gi + 1].y, sc4[2 * gi + 1].z, sc4[2 * gi + 1].w};
+                const float bv[8] = {bi4[2 * gi].x, bi4[2 * gi].y, bi4[2 * gi].z, bi4[2 * gi].w,
+                                     bi4[2 * gi + 1].x, bi4[2 * gi + 1].y, bi4[2 * gi + 1].z, bi4[2 * gi + 1].w};
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                  v[j] = fmaf(__uint_as_float(r[gi * 8 + j]) * xq.s, my_sc[cj + j], my_sc[128 + cj + j]);
+                for (int j = 0; j < 8; ++j) v[j] = fmaf(__uint_as_float(r[gi * 8 + j]), sv[j], bv[j]);
               } else {
                 float x[8];
                 if (bc == 32) {      // bf16 activations: 8 values in one 16-byte piece
@@ -493,11 +507,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
+                  // Eq. 1 with the straight-through estimator, the arithmetic of quant_act()
                   const float gx = __uint_as_float(r[gi * 8 + j]);
-                  const QElem qe = quant_act(x[j], xq);
-                  v[j] = qe.flag ? 0.f : gx;
-                  acc_s = fmaf(gx, qe.t, acc_s);
-                  acc_z += qe.flag ? -gx * xq.s : 0.f;
+                  const float rq = rne_small(__fmul_rn(x[j], xq.rinv));
+                  const float cq = rq + xq.zr;
+                  const bool below = cq < xq.lo, above = cq > xq.hi;
+                  const float resid = fmaf(-x[j], xq.rinv_lo, fmaf(-x[j], xq.rinv, rq));
+                  const float tq = below ? t_lo : (above ? t_hi : resid);
+                  const bool clipped = below || above;
+                  v[j] = clipped ? 0.f : gx;
+                  acc_s = fmaf(gx, tq, acc_s);
+                  acc_c += clipped ? gx : 0.f;
                 }
               }
               if (bc == 32) {
@@ -531,11 +551,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       if (EPI == EPI_DX && ok) {
         acc_s = warp_sum(acc_s);
-        acc_z = warp_sum(acc_z);
+        acc_c = warp_sum(acc_c);
         if (lane == 0) {
           float* pp = p.partials + ((static_cast<int64_t>(g.t) * (CTA2 ? 2 : 1) + rank) * EPI_WARPS + e) * 2;
           pp[0] = acc_s;
-          pp[1] = acc_z;
+          pp[1] = -xq.s * acc_c;     // Eq. 1: d(dequantised)/dZ = -s on clipped elements, 0 elsewhere
         }
       }
       if (EPI == EPI_FWD && has_next) {

@@ -46,7 +46,7 @@ __device__ __forceinline__ float rne_small(float u) {
 __device__ __forceinline__ QElem quant_act(float x, const ActQ& p) {
   QElem e;
   const float u = __fmul_rn(x, p.rinv);
-  const float r = rintf(u);
+  const float r = rne_small(u);
   const float c = r + p.zr;
   const float q = fminf(fmaxf(c, p.lo), p.hi);
   e.flag = (c < p.lo) ? 1 : ((c > p.hi) ? 2 : 0);
@@ -103,7 +103,7 @@ __device__ __forceinline__ RowQ make_rowq(float s, int w_bits) {
 __device__ __forceinline__ QElem quant_weight(float w, const RowQ& p) {
   QElem e;
   const float u = __fmul_rn(w, p.rinv);
-  const float c = rintf(u);
+  const float c = rne_small(u);
   const float q = fminf(fmaxf(c, -p.qmax), p.qmax);
   e.flag = (c < -p.qmax) ? 1 : ((c > p.qmax) ? 2 : 0);
   e.c0 = q;

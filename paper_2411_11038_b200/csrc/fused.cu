@@ -36,26 +36,43 @@ __device__ __forceinline__ void st8(bf16* p, const float (&v)[8]) {
   *reinterpret_cast<uint4*>(p) = o;
 }
 
-// ---- job: weight rows -> bf16 operand (MODE 0 codes, MODE 1 dequantised) --------------
+// ---- job: weights -> bf16 operand (MODE 0 codes, MODE 1 dequantised) -------------------
+// Flat over 8-element vectors (K % 8 == 0, so a vector never straddles two rows), four
+// independent loads in flight per thread.
 template <int MODE>
-__device__ __forceinline__ void job_weight_row(const PrepArgs& a, int64_t n) {
-  float s = a.s_w[n];
-  if (!scale_ok(s)) {
-    if (threadIdx.x == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
-    s = 1.f;
-  }
-  const RowQ p = make_rowq(s, a.w_bits);
-  const float* row = a.W + n * a.K;
-  bf16* orow = a.Wq + n * a.K;
-  for (int64_t k = threadIdx.x * 8; k < a.K; k += blockDim.x * 8) {
-    float v[8];
-    ld8<float>(row + k, v);
+__device__ __forceinline__ void job_weights(const PrepArgs& a, int block, int nblocks) {
+  const int64_t kv = a.K / 8;
+  const int64_t nvec = a.N * kv;
+  const int64_t stride = static_cast<int64_t>(nblocks) * blockDim.x;
+  for (int64_t v0 = static_cast<int64_t>(block) * blockDim.x + threadIdx.x; v0 < nvec; v0 += 4 * stride) {
+    float v[4][8];
+    float sc[4];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float q = quant_weight(v[j], p).c0;
-      v[j] = (MODE == 0) ? q : __fmul_rn(p.s, q);
+    for (int u = 0; u < 4; ++u) {
+      const int64_t i = v0 + u * stride;
+      if (i < nvec) {
+        ld8<float>(a.W + i * 8, v[u]);
+        sc[u] = __ldg(a.s_w + i / kv);
+      }
     }
-    st8(orow + k, v);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t i = v0 + u * stride;
+      if (i < nvec) {
+        float sw = sc[u];
+        if (!scale_ok(sw)) {
+          record_status(a.status, EFQAT_DEV_BAD_SCALE);
+          sw = 1.f;
+        }
+        const RowQ p = make_rowq(sw, a.w_bits);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float q = quant_weight(v[u][j], p).c0;
+          v[u][j] = (MODE == 0) ? q : __fmul_rn(p.s, q);
+        }
+        st8(a.Wq + i * 8, v[u]);
+      }
+    }
   }
 }
 
@@ -67,18 +84,26 @@ __device__ __forceinline__ void job_quant_x(const PrepArgs& a, int block, int nb
   if (bad && block == 0 && threadIdx.x == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
   const T* X = static_cast<const T*>(a.X);
   const int64_t n8 = a.x_count / 8;
-  for (int64_t i = static_cast<int64_t>(block) * blockDim.x + threadIdx.x; i < n8;
-       i += static_cast<int64_t>(nblocks) * blockDim.x) {
-    float v[8];
-    ld8<T>(X + i * 8, v);
+  const int64_t stride = static_cast<int64_t>(nblocks) * blockDim.x;
+  for (int64_t i0 = static_cast<int64_t>(block) * blockDim.x + threadIdx.x; i0 < n8; i0 += 4 * stride) {
+    float v[4][8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = quant_act(v[j], p).c0;
-    st8(a.Xc + i * 8, v);
+    for (int u = 0; u < 4; ++u)
+      if (i0 + u * stride < n8) ld8<T>(X + (i0 + u * stride) * 8, v[u]);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (i0 + u * stride < n8) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[u][j] = quant_act(v[u][j], p).c0;
+        st8(a.Xc + (i0 + u * stride) * 8, v[u]);
+      }
+    }
   }
 }
 
-// ---- job: one pass over dY: column-sum partials, gather of the selected columns, bf16 copy
-// Block (cb, slab): 256 columns x one slab of rows; warp w takes rows slab_lo + w, + 8, ...
+// ---- job: one pass over dY: column-sum partials and the bf16 copy ------------------------
+// Block (cb, slab): 256 columns x one slab of rows; warp w takes rows slab_lo + w, + 8, ...,
+// four rows (four independent 16-byte loads per thread) at a time.
 template <typename T>
 __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab, float* sh /* [8][256] */) {
   const T* dY = static_cast<const T*>(a.dY);
@@ -87,97 +112,24 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
   const int64_t rows = ceil_div(a.M, static_cast<int64_t>(a.slabs));
   const int64_t m_lo = slab * rows;
   const int64_t m_hi = (m_lo + rows < a.M) ? m_lo + rows : a.M;
-  const bool col_ok = c0 < a.N;
-  const bool gather = a.k_sel > 0 && a.k_sel < a.N;
-  int pos[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) pos[j] = -1;
-  if (gather) {
-    // Compact position of each of this thread's 8 consecutive columns in the ascending idx:
-    // one binary search for the first column, then a merge walk.  The slice of idx that this
-    // block's 256 columns can hit is staged in shared memory first (it holds at most 256 entries).
-    __shared__ int s_lo, s_cnt;
-    __shared__ int32_t s_idx[256];
-    if (threadIdx.x == 0) {
-      const int cfirst = cb * 256;
-      int lo = 0, hi = static_cast<int>(a.k_sel);
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (a.idx[mid] < cfirst) lo = mid + 1; else hi = mid;
-      }
-      s_lo = lo;
-      int l2 = lo, h2 = static_cast<int>(a.k_sel);
-      while (l2 < h2) {
-        const int mid = (l2 + h2) >> 1;
-        if (a.idx[mid] < cfirst + 256) l2 = mid + 1; else h2 = mid;
-      }
-      s_cnt = (l2 - lo > 256) ? 256 : l2 - lo;      // more than 256 only for a broken (non-ascending) idx
-    }
-    __syncthreads();
-    if (threadIdx.x < s_cnt) s_idx[threadIdx.x] = a.idx[s_lo + threadIdx.x];
-    __syncthreads();
-    if (col_ok) {
-      int lo = 0, hi = s_cnt;
-      const int cmin = static_cast<int>(c0);
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (s_idx[mid] < cmin) lo = mid + 1; else hi = mid;
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (lo < s_cnt && s_idx[lo] == cmin + j) {
-          pos[j] = s_lo + lo;
-          ++lo;
-        }
-      }
-    }
-  }
-  if (gather && cb == 0 && slab == 0) {
-    // index contract: strictly ascending, inside [0, N)
-    for (int j = threadIdx.x; j < a.k_sel; j += blockDim.x) {
-      const int c = a.idx[j];
-      if (c < 0 || c >= a.N || (j > 0 && a.idx[j - 1] >= c)) record_status(a.status, EFQAT_DEV_BAD_INDEX);
-    }
-  }
   float acc[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-  if (col_ok) {
-    int64_t m = m_lo + warp;
-    for (; m + 24 < m_hi; m += 32) {       // four independent 16-byte loads in flight per thread
+  if (c0 < a.N) {
+    for (int64_t m = m_lo + warp; m < m_hi; m += 32) {
       float v[4][8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) ld8<T>(dY + (m + 8 * u) * a.N + c0, v[u]);
+      for (int u = 0; u < 4; ++u)
+        if (m + 8 * u < m_hi) ld8<T>(dY + (m + 8 * u) * a.N + c0, v[u]);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
+        if (m + 8 * u < m_hi) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] += v[u][j];
-        if (a.dYb) st8(a.dYb + (m + 8 * u) * a.N + c0, v[u]);
-        if (gather) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (pos[j] >= 0) a.dYsel[(m + 8 * u) * a.pitch + pos[j]] = __float2bfloat16_rn(v[u][j]);
+          for (int j = 0; j < 8; ++j) acc[j] += v[u][j];
+          if (a.dYb) st8(a.dYb + (m + 8 * u) * a.N + c0, v[u]);
         }
       }
     }
-    for (; m < m_hi; m += 8) {
-      float v[8];
-      ld8<T>(dY + m * a.N + c0, v);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] += v[j];
-      if (a.dYb) st8(a.dYb + m * a.N + c0, v);
-      if (gather) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (pos[j] >= 0) a.dYsel[m * a.pitch + pos[j]] = __float2bfloat16_rn(v[j]);
-      }
-    }
-  }
-  if (gather && cb == 0) {
-    // zero the pad columns [k_sel, pitch) of this slab's rows
-    const int pad = static_cast<int>(a.pitch - a.k_sel);
-    for (int64_t i = threadIdx.x; i < (m_hi - m_lo) * pad; i += blockDim.x)
-      a.dYsel[(m_lo + i / pad) * a.pitch + a.k_sel + (i % pad)] = __float2bfloat16_rn(0.f);
   }
   if (a.colsum_ws) {
 #pragma unroll
@@ -193,16 +145,66 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
   }
 }
 
+// ---- job: gathered matrix dYsel[m, i] = bf16(dY[m, idx[i]]), pad columns [k_sel, pitch) zero ----
+// Whole rows of the gathered matrix leave as full 128-byte lines; the scattered 2- or 4-byte
+// reads of dY hit the sectors that the column-sum pass of the same launch brings into L2.
+// The index list is staged in shared memory 1024 entries at a time.
+static const int GATHER_ROWS = 64;      // rows of dY per block
+template <typename T>
+__device__ __forceinline__ void job_gather(const PrepArgs& a, int block, int32_t* s_idx /* [1024] */) {
+  const T* dY = static_cast<const T*>(a.dY);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t m_lo = static_cast<int64_t>(block) * GATHER_ROWS;
+  const int64_t m_hi = (m_lo + GATHER_ROWS < a.M) ? m_lo + GATHER_ROWS : a.M;
+  for (int64_t ch = 0; ch < a.pitch; ch += 1024) {
+    const int n = static_cast<int>((a.pitch - ch < 1024) ? a.pitch - ch : 1024);     // even: pitch % 16 == 0
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      int c = -1;
+      if (ch + i < a.k_sel) {
+        c = __ldg(a.idx + ch + i);
+        // index contract: strictly ascending, inside [0, N)
+        const bool bad = c < 0 || c >= a.N || (ch + i > 0 && __ldg(a.idx + ch + i - 1) >= c);
+        if (bad) {
+          if (block == 0) record_status(a.status, EFQAT_DEV_BAD_INDEX);
+          c = -1;
+        }
+      }
+      s_idx[i] = c;
+    }
+    __syncthreads();
+    for (int64_t m = m_lo + warp; m < m_hi; m += 32) {        // four rows in flight per warp
+      for (int i = 2 * lane; i < n; i += 64) {
+        const int ca = s_idx[i], cb = s_idx[i + 1];
+        float va[4], vb[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int64_t r = m + 8 * u;
+          va[u] = (r < m_hi && ca >= 0) ? static_cast<float>(dY[r * a.N + ca]) : 0.f;
+          vb[u] = (r < m_hi && cb >= 0) ? static_cast<float>(dY[r * a.N + cb]) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int64_t r = m + 8 * u;
+          if (r < m_hi) *reinterpret_cast<uint32_t*>(a.dYsel + r * a.pitch + ch + i) = pk2(va[u], vb[u]);
+        }
+      }
+    }
+  }
+}
+
 template <int W_MODE, typename TX>
 __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
   __shared__ float sh[8 * 256];
   const int b = blockIdx.x;
-  if (b < a.nb_w) {
-    job_weight_row<W_MODE>(a, b);
-  } else if (b < a.nb_w + a.nb_x) {
-    job_quant_x<TX>(a, b - a.nb_w, a.nb_x);
+  if (b < a.nb_g) {
+    job_gather<TX>(a, b, reinterpret_cast<int32_t*>(sh));
+  } else if (b < a.nb_g + a.nb_w) {
+    job_weights<W_MODE>(a, b - a.nb_g, a.nb_w);
+  } else if (b < a.nb_g + a.nb_w + a.nb_x) {
+    job_quant_x<TX>(a, b - a.nb_g - a.nb_w, a.nb_x);
   } else {
-    const int r = b - a.nb_w - a.nb_x;
+    const int r = b - a.nb_g - a.nb_w - a.nb_x;
     job_dy_pass<TX>(a, r % a.col_blocks, r / a.col_blocks, sh);
   }
 }
@@ -227,9 +229,17 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
     double acc = 0.0;
     for (int64_t k = threadIdx.x * 4; k < a.K; k += blockDim.x * 4) {
       float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int sp = 0; sp < a.splits; ++sp) {
-        const float4 t = *reinterpret_cast<const float4*>(a.P + sp * a.split_stride + i * a.K + k);
-        g.x += t.x; g.y += t.y; g.z += t.z; g.w += t.w;
+      for (int sp0 = 0; sp0 < a.splits; sp0 += 8) {       // eight independent loads in flight, summed in split order
+        float4 t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          t[u] = (sp0 + u < a.splits)
+                     ? __ldg(reinterpret_cast<const float4*>(a.P + (sp0 + u) * a.split_stride + i * a.K + k))
+                     : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          g.x += t[u].x; g.y += t[u].y; g.z += t[u].z; g.w += t[u].w;
+        }
       }
       const float4 w4 = *reinterpret_cast<const float4*>(wrow + k);
       const float gv[4] = {g.x * sx, g.y * sx, g.z * sx, g.w * sx};
@@ -305,33 +315,35 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
 
 }  // namespace
 
-// Row slabs of the dY pass: enough blocks (column blocks x slabs) to fill the GPU about four
-// times over, at least 32 rows per slab.
+// Row slabs of the dY pass: blocks of 256 columns x one slab of rows, about 32 KiB of dY
+// each (at least 32 rows), so that the launch spreads over the whole GPU a few times.
 int prepare_slabs(int64_t M, int64_t N) {
-  const int64_t col_blocks = ceil_div(N, 256);
-  int64_t s = ceil_div(4 * 148, col_blocks);
-  const int64_t by_rows = ceil_div(M, 32);
-  if (s > by_rows) s = by_rows;
+  (void)N;
+  int64_t s = ceil_div(M, 64);
   if (s > 2048) s = 2048;
   if (s < 1) s = 1;
   return static_cast<int>(s);
 }
 
+// Blocks of a flat job: about `per_block` vectors of 8 elements each, at most four waves of the GPU.
+static int flat_blocks(int64_t vectors, int64_t per_block) {
+  int64_t nb = ceil_div(vectors, per_block);
+  if (nb > 148 * 12) nb = 148 * 12;
+  if (nb < 1) nb = 1;
+  return static_cast<int>(nb);
+}
+
 void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
-  a.nb_w = static_cast<int>(a.N);
+  a.nb_w = flat_blocks(a.N * (a.K / 8), 256 * 4);       // 32 KiB of fp32 weights per block
   a.nb_x = 0;
-  if (a.Xc) {
-    int64_t nb = ceil_div(a.x_count / 8, 256 * 2);
-    if (nb > 148 * 8) nb = 148 * 8;
-    if (nb < 1) nb = 1;
-    a.nb_x = static_cast<int>(nb);
-  }
-  const bool gather = a.k_sel > 0 && a.k_sel < a.N;
+  if (a.Xc) a.nb_x = flat_blocks(a.x_count / 8, 256 * 8);   // 32 KiB (bf16) / 64 KiB (fp32) per block
+  const bool gather = a.dY && a.dYsel && a.k_sel > 0 && a.k_sel < a.N;
+  a.nb_g = gather ? static_cast<int>(ceil_div(a.M, GATHER_ROWS)) : 0;
   int nb_y = 0;
   a.col_blocks = static_cast<int>(ceil_div(a.N, 256));
   a.slabs = prepare_slabs(a.M, a.N);
-  if (a.dY && (a.colsum_ws || gather || a.dYb)) nb_y = a.col_blocks * a.slabs;
-  const int grid = a.nb_w + a.nb_x + nb_y;
+  if (a.dY && (a.colsum_ws || a.dYb)) nb_y = a.col_blocks * a.slabs;
+  const int grid = a.nb_g + a.nb_w + a.nb_x + nb_y;
   count_launches(1);
   if (w_mode == 0) {
     if (act_bf16) prepare_kernel<0, bf16><<<grid, 256, 0, st>>>(a);

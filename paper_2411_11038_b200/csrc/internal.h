@@ -41,8 +41,9 @@ void launch_absmax_rows(const float* W, int64_t N, int64_t K, int w_bits, float*
 
 // ---- fused.cu -----------------------------------------------------------------------
 // One launch in front of the GEMMs: weight rows -> bf16 operand, activations -> centred codes
-// (skipped when Xc is null), and one pass over dY (skipped when dY is null or nothing of it
-// is wanted) producing column-sum partials, the gathered selected columns and a bf16 copy.
+// (skipped when Xc is null), one pass over dY (skipped when dY is null or nothing of it is
+// wanted) producing column-sum partials and a bf16 copy, and the gather of the selected
+// columns of dY (when dYsel is set and 0 < k_sel < N).
 struct PrepArgs {
   int64_t M, N, K;
   const float* W; const float* s_w; int w_bits; bf16* Wq;
@@ -51,7 +52,7 @@ struct PrepArgs {
   const void* dY; bf16* dYb; float* colsum_ws;
   const int32_t* idx; int64_t k_sel, pitch; bf16* dYsel;
   int* status;
-  int nb_w, nb_x, col_blocks, slabs;   // filled by launch_prepare
+  int nb_g, nb_w, nb_x, col_blocks, slabs;   // filled by launch_prepare
 };
 int prepare_slabs(int64_t M, int64_t N);
 void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st);

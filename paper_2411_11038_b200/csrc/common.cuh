@@ -28,6 +28,13 @@ struct QElem {
   int code;   // clamp(c, lo, hi)
 };
 
+// Programmatic dependent launch: every kernel of the layer path lets the next launch of the
+// stream start early (pdl_trigger) and waits for the launches before it to finish, with
+// their writes visible, before it touches global memory (pdl_wait).  Between the two, only
+// set-up that reads no global data may run.  Both are no-ops for a plain launch.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void record_status(int* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }

@@ -196,6 +196,8 @@ __device__ __forceinline__ void job_gather(const PrepArgs& a, int block, int32_t
 template <int W_MODE, typename TX>
 __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
   __shared__ float sh[8 * 256];
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.x;
   if (b < a.nb_g) {
     job_gather<TX>(a, b, reinterpret_cast<int32_t*>(sh));
@@ -212,6 +214,8 @@ __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
 // ---- finalize: dW rows (mask, dS_w, optional SGD) | dS_x, dZ_x | db ------------------------
 __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
   __shared__ double shd[2][256];
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.x;
   if (b < a.k_sel) {
     const int64_t i = b;
@@ -346,11 +350,11 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   const int grid = a.nb_g + a.nb_w + a.nb_x + nb_y;
   count_launches(1);
   if (w_mode == 0) {
-    if (act_bf16) prepare_kernel<0, bf16><<<grid, 256, 0, st>>>(a);
-    else prepare_kernel<0, float><<<grid, 256, 0, st>>>(a);
+    if (act_bf16) launch_dependent(prepare_kernel<0, bf16>, grid, 256, 0, st, 1, a);
+    else launch_dependent(prepare_kernel<0, float>, grid, 256, 0, st, 1, a);
   } else {
-    if (act_bf16) prepare_kernel<1, bf16><<<grid, 256, 0, st>>>(a);
-    else prepare_kernel<1, float><<<grid, 256, 0, st>>>(a);
+    if (act_bf16) launch_dependent(prepare_kernel<1, bf16>, grid, 256, 0, st, 1, a);
+    else launch_dependent(prepare_kernel<1, float>, grid, 256, 0, st, 1, a);
   }
 }
 
@@ -358,7 +362,7 @@ void launch_finalize(FinArgs a, cudaStream_t st) {
   const int nb_db = a.db ? static_cast<int>(ceil_div(a.N, 32)) : 0;
   const int grid = static_cast<int>(a.k_sel) + 1 + nb_db;
   count_launches(1);
-  finalize_kernel<<<grid, 256, 0, st>>>(a);
+  launch_dependent(finalize_kernel, grid, 256, 0, st, 1, a);
 }
 
 }  // namespace efqat

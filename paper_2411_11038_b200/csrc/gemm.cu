@@ -147,6 +147,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (CTA2) cluster_sync();     // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  // barriers, TMEM and descriptor prefetches are in place; everything below reads global memory
+  pdl_trigger();
+  pdl_wait();
   volatile int* abort_flag = &ctl->abort_flag;
 
   if (warp == 0) {
@@ -703,23 +706,9 @@ static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMa
     configured[dev] = true;
   }
   count_launches(1);
-  if (CTA2) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    cfg.blockDim = dim3(GEMM_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2;
-    at[0].val.clusterDim.y = 1;
-    at[0].val.clusterDim.z = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, ta, tb, to, tx, p) != cudaSuccess) return EFQAT_ERR_CUDA;
-  } else {
-    kern<<<grid, GEMM_THREADS, smem, st>>>(ta, tb, to, tx, p);
-  }
+  if (launch_dependent(kern, static_cast<unsigned>(grid), GEMM_THREADS, smem, st, CTA2 ? 2 : 1, ta, tb, to, tx, p) !=
+      cudaSuccess)
+    return EFQAT_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 

@@ -24,6 +24,8 @@ struct TableChunk {
 };
 
 __global__ void table_write_kernel(TableChunk chunk, int count, LayerEntry* __restrict__ dst) {
+  pdl_trigger();
+  pdl_wait();
   const int i = threadIdx.x;
   if (i < count) dst[i] = chunk.e[i];
 }
@@ -46,6 +48,8 @@ __device__ __forceinline__ double abs4(const float4 a) {
 __global__ void __launch_bounds__(256) row_importance_kernel(const LayerEntry* __restrict__ table, int L,
                                                              int total_rows, float* __restrict__ keys,
                                                              double* __restrict__ rowsum) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   for (int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5); row < total_rows;
@@ -81,6 +85,8 @@ __global__ void __launch_bounds__(256) row_importance_kernel(const LayerEntry* _
 __global__ void __launch_bounds__(256) layer_importance_kernel(const LayerEntry* __restrict__ table,
                                                                const double* __restrict__ rowsum,
                                                                float* __restrict__ layer_keys) {
+  pdl_trigger();
+  pdl_wait();
   const LayerEntry e = table[blockIdx.x];
   double acc = 0.0;
   for (int i = threadIdx.x; i < e.N; i += blockDim.x) acc += rowsum[e.row_off + i];
@@ -136,6 +142,8 @@ __device__ __forceinline__ void block_scan2(int a, int b, int& pa, int& pb, int*
 __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restrict__ keys,
                                                             const LayerEntry* __restrict__ table, int single_len,
                                                             int single_k, int32_t* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int hist[256];
   __shared__ int suf[257];
   __shared__ int scan_sh[64];
@@ -228,6 +236,8 @@ struct TopkState {
 static const int BIG_CHUNK = 4096;      // keys per block in the count / write kernels
 
 __global__ void topk_big_init_kernel(TopkState* st, int k, int* ghist) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x < 256) ghist[threadIdx.x] = 0;
   if (threadIdx.x == 0) {
     st->prefix = 0; st->mask = 0; st->remaining = k; st->pad = 0;
@@ -236,6 +246,8 @@ __global__ void topk_big_init_kernel(TopkState* st, int k, int* ghist) {
 __global__ void __launch_bounds__(256) topk_big_hist_kernel(const float* __restrict__ keys, int n,
                                                             const TopkState* __restrict__ st, int shift,
                                                             int* __restrict__ ghist) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int sh[256];
   sh[threadIdx.x] = 0;
   __syncthreads();
@@ -248,6 +260,8 @@ __global__ void __launch_bounds__(256) topk_big_hist_kernel(const float* __restr
   if (sh[threadIdx.x]) atomicAdd(&ghist[threadIdx.x], sh[threadIdx.x]);
 }
 __global__ void __launch_bounds__(256) topk_big_pick_kernel(TopkState* st, int shift, int* ghist) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int suf[257];
   const int d = threadIdx.x;
   suf[d] = ghist[d];
@@ -273,6 +287,8 @@ __global__ void __launch_bounds__(256) topk_big_pick_kernel(TopkState* st, int s
 __global__ void __launch_bounds__(TOPK_THREADS) topk_big_count_kernel(const float* __restrict__ keys, int n,
                                                                       const TopkState* __restrict__ st,
                                                                       int* __restrict__ counts) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int red[2][32];
   const uint32_t thr = st->prefix;
   const int lo = blockIdx.x * BIG_CHUNK, hi = min(n, lo + BIG_CHUNK);
@@ -296,6 +312,8 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_big_count_kernel(const floa
   }
 }
 __global__ void topk_big_scan_kernel(const int* __restrict__ counts, int blocks, int* __restrict__ offs) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
   int a = 0, b = 0;
   for (int i = 0; i < blocks; ++i) {
@@ -309,6 +327,8 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_big_write_kernel(const floa
                                                                       const TopkState* __restrict__ st,
                                                                       const int* __restrict__ offs,
                                                                       int32_t* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int scan_sh[64];
   __shared__ int carry[2];
   const uint32_t thr = st->prefix;
@@ -336,6 +356,8 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_big_write_kernel(const floa
 
 __global__ void cwpl_offsets_kernel(const LayerEntry* __restrict__ table, int L, int total,
                                     int32_t* __restrict__ offsets) {
+  pdl_trigger();
+  pdl_wait();
   const int l = blockIdx.x * blockDim.x + threadIdx.x;
   if (l < L) offsets[l] = table[l].out_off;
   if (l == L) offsets[L] = total;
@@ -344,6 +366,8 @@ __global__ void cwpl_offsets_kernel(const LayerEntry* __restrict__ table, int L,
 // CWPN: sel holds the k_tot winning global ids in ascending order.
 __global__ void cwpn_split_kernel(const LayerEntry* __restrict__ table, int L, const int32_t* __restrict__ sel,
                                   int k_tot, int32_t* __restrict__ idx, int32_t* __restrict__ offsets) {
+  pdl_trigger();
+  pdl_wait();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j < k_tot) {
     const int g = sel[j];
@@ -364,6 +388,8 @@ __global__ void cwpn_split_kernel(const LayerEntry* __restrict__ table, int L, c
 // LWPN: lsel holds the k_L winning layer ids ascending; offsets = prefix of N_l over kept layers.
 __global__ void lwpn_offsets_kernel(const LayerEntry* __restrict__ table, int L, const int32_t* __restrict__ lsel,
                                     int k_L, int32_t* __restrict__ keep, int32_t* __restrict__ offsets) {
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
   int p = 0, off = 0;
   for (int l = 0; l < L; ++l) {
@@ -378,6 +404,8 @@ __global__ void lwpn_offsets_kernel(const LayerEntry* __restrict__ table, int L,
 __global__ void lwpn_fill_kernel(const LayerEntry* __restrict__ table, int L, int total_rows,
                                  const int32_t* __restrict__ keep, const int32_t* __restrict__ offsets,
                                  int32_t* __restrict__ idx) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= total_rows) return;
   const int l = layer_of_row(table, L, row);
@@ -471,19 +499,19 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
       out_off += e.k;
     }
     count_launches(1);
-    table_write_kernel<<<1, TABLE_CHUNK, 0, st>>>(chunk, cnt, w.table + base);
+    launch_dependent(table_write_kernel, 1, TABLE_CHUNK, 0, st, 1, chunk, cnt, w.table + base);
   }
   const int tot = static_cast<int>(total);
   {
     int64_t blocks = ceil_div(total, 8);
     if (blocks > 148 * 8) blocks = 148 * 8;
     count_launches(1);
-    row_importance_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(w.table, L, tot, w.keys, w.rowsum);
+    launch_dependent(row_importance_kernel, static_cast<unsigned>(blocks), 256, 0, st, 1, w.table, L, tot, w.keys, w.rowsum);
   }
   if (mode == EFQAT_CWPL) {
     count_launches(2);
-    topk_kernel<<<L, TOPK_THREADS, 0, st>>>(w.keys, w.table, 0, 0, idx);
-    cwpl_offsets_kernel<<<static_cast<unsigned>(ceil_div(L + 1, 256)), 256, 0, st>>>(w.table, L,
+    launch_dependent(topk_kernel, L, TOPK_THREADS, 0, st, 1, w.keys, w.table, 0, 0, idx);
+    launch_dependent(cwpl_offsets_kernel, static_cast<unsigned>(ceil_div(L + 1, 256)), 256, 0, st, 1, w.table, L,
                                                                                     static_cast<int>(out_off),
                                                                                     offsets);
     if (importance) cudaMemcpyAsync(importance, w.keys, sizeof(float) * total, cudaMemcpyDeviceToDevice, st);
@@ -494,30 +522,30 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
       int hgrid = static_cast<int>(ceil_div(tot, 256 * 4));
       if (hgrid > 148 * 4) hgrid = 148 * 4;
       count_launches(13);
-      topk_big_init_kernel<<<1, 256, 0, st>>>(w.big_state, kt, w.big_hist);
+      launch_dependent(topk_big_init_kernel, 1, 256, 0, st, 1, w.big_state, kt, w.big_hist);
       for (int shift = 24; shift >= 0; shift -= 8) {
-        topk_big_hist_kernel<<<hgrid, 256, 0, st>>>(w.keys, tot, w.big_state, shift, w.big_hist);
-        topk_big_pick_kernel<<<1, 256, 0, st>>>(w.big_state, shift, w.big_hist);
+        launch_dependent(topk_big_hist_kernel, hgrid, 256, 0, st, 1, w.keys, tot, w.big_state, shift, w.big_hist);
+        launch_dependent(topk_big_pick_kernel, 1, 256, 0, st, 1, w.big_state, shift, w.big_hist);
       }
-      topk_big_count_kernel<<<blocks, TOPK_THREADS, 0, st>>>(w.keys, tot, w.big_state, w.big_counts);
-      topk_big_scan_kernel<<<1, 32, 0, st>>>(w.big_counts, blocks, w.big_offs);
-      topk_big_write_kernel<<<blocks, TOPK_THREADS, 0, st>>>(w.keys, tot, w.big_state, w.big_offs, w.sel);
+      launch_dependent(topk_big_count_kernel, blocks, TOPK_THREADS, 0, st, 1, w.keys, tot, w.big_state, w.big_counts);
+      launch_dependent(topk_big_scan_kernel, 1, 32, 0, st, 1, w.big_counts, blocks, w.big_offs);
+      launch_dependent(topk_big_write_kernel, blocks, TOPK_THREADS, 0, st, 1, w.keys, tot, w.big_state, w.big_offs, w.sel);
     } else {
       count_launches(1);
-      topk_kernel<<<1, TOPK_THREADS, 0, st>>>(w.keys, nullptr, tot, kt, w.sel);
+      launch_dependent(topk_kernel, 1, TOPK_THREADS, 0, st, 1, w.keys, nullptr, tot, kt, w.sel);
     }
     count_launches(1);
     const int work = (kt > L + 1) ? kt : L + 1;
-    cwpn_split_kernel<<<static_cast<unsigned>(ceil_div(work, 256)), 256, 0, st>>>(w.table, L, w.sel, kt, idx,
+    launch_dependent(cwpn_split_kernel, static_cast<unsigned>(ceil_div(work, 256)), 256, 0, st, 1, w.table, L, w.sel, kt, idx,
                                                                                  offsets);
     if (importance) cudaMemcpyAsync(importance, w.keys, sizeof(float) * total, cudaMemcpyDeviceToDevice, st);
   } else {
     const int kl = static_cast<int>(k[0]);
     count_launches(4);
-    layer_importance_kernel<<<L, 256, 0, st>>>(w.table, w.rowsum, w.layer_keys);
-    topk_kernel<<<1, TOPK_THREADS, 0, st>>>(w.layer_keys, nullptr, L, kl, w.lsel);
-    lwpn_offsets_kernel<<<1, 32, 0, st>>>(w.table, L, w.lsel, kl, w.keep, offsets);
-    lwpn_fill_kernel<<<static_cast<unsigned>(ceil_div(total, 256)), 256, 0, st>>>(w.table, L, tot, w.keep, offsets,
+    launch_dependent(layer_importance_kernel, L, 256, 0, st, 1, w.table, w.rowsum, w.layer_keys);
+    launch_dependent(topk_kernel, 1, TOPK_THREADS, 0, st, 1, w.layer_keys, nullptr, L, kl, w.lsel);
+    launch_dependent(lwpn_offsets_kernel, 1, 32, 0, st, 1, w.table, L, w.lsel, kl, w.keep, offsets);
+    launch_dependent(lwpn_fill_kernel, static_cast<unsigned>(ceil_div(total, 256)), 256, 0, st, 1, w.table, L, tot, w.keep, offsets,
                                                                                  idx);
     if (importance) cudaMemcpyAsync(importance, w.layer_keys, sizeof(float) * L, cudaMemcpyDeviceToDevice, st);
   }

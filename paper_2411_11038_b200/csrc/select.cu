@@ -108,6 +108,7 @@ __device__ __forceinline__ uint32_t key_bits(float f) {
 }
 
 static const int TOPK_THREADS = 1024;
+static const int TOPK_SMEM_KEYS = 8192;
 
 // Block-wide exclusive scan of two counters (all TOPK_THREADS threads must call).
 __device__ __forceinline__ void block_scan2(int a, int b, int& pa, int& pb, int* sh) {
@@ -149,6 +150,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
   __shared__ int scan_sh[64];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
+  __shared__ uint32_t skeys[TOPK_SMEM_KEYS];
 
   int begin = 0, n = single_len, k = single_k, out_off = 0;
   if (table) {
@@ -160,6 +162,15 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
   const float* kp = keys + begin;
   int32_t* op = out + out_off;
 
+  // Segments of up to TOPK_SMEM_KEYS keys are read from global memory once, as their
+  // order-preserving integer images, and every pass works on the shared copy.
+  const bool cached = n <= TOPK_SMEM_KEYS;
+  if (cached) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) skeys[i] = key_bits(kp[i]);
+    __syncthreads();
+  }
+  auto key_at = [&](int i) { return cached ? skeys[i] : key_bits(kp[i]); };
+
   uint32_t prefix = 0, mask = 0;
   int remaining = k;
   for (int shift = 24; shift >= 0; shift -= 8) {
@@ -167,28 +178,48 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
     __syncthreads();
     for (int base = 0; base < n; base += blockDim.x) {
       const int i = base + threadIdx.x;
-      int digit = 256 + (threadIdx.x & 31);          // distinct dummy values for idle lanes
+      int digit = -1;                                // -1: not a candidate any more
       if (i < n) {
-        const uint32_t kb = key_bits(kp[i]);
+        const uint32_t kb = key_at(i);
         if ((kb & mask) == prefix) digit = (kb >> shift) & 255;
       }
-      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit < 256 && (threadIdx.x & 31) == (__ffs(peers) - 1)) atomicAdd(&hist[digit], __popc(peers));
+      // Importance keys share their leading bytes, so in the first passes a whole warp usually
+      // lands in one bin: that case costs one atomic per warp, the general one one per lane.
+      const uint32_t cand = __ballot_sync(0xffffffffu, digit >= 0);
+      if (cand) {
+        const int leader = __ffs(cand) - 1;
+        const int d0 = __shfl_sync(0xffffffffu, digit, leader);
+        const bool same = __all_sync(0xffffffffu, digit < 0 || digit == d0);
+        if (same) {
+          if ((threadIdx.x & 31) == leader) atomicAdd(&hist[d0], __popc(cand));
+        } else if (digit >= 0) {
+          atomicAdd(&hist[digit], 1);
+        }
+      }
     }
     __syncthreads();
-    // digit of the k-th largest candidate: largest d whose suffix count reaches `remaining`
-    // (suffix sums over the 256 bins, Hillis-Steele in shared memory)
+    // digit of the k-th largest candidate: largest d whose suffix count reaches `remaining`.
+    // Suffix sums over the 256 bins: inclusive suffix inside each of 8 warps by shuffles,
+    // then the totals of the warps above are added.
     {
-      const int d = threadIdx.x;
-      if (d < 256) suf[d] = hist[d];
+      const int d = threadIdx.x, lane = d & 31, warp = d >> 5;
+      int v = (d < 256) ? hist[d] : 0;
+      if (d < 256) {
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int u = __shfl_down_sync(0xffffffffu, v, o);
+          if (lane + o < 32) v += u;
+        }
+        if (lane == 0) scan_sh[warp] = v;          // total of this warp's 32 bins
+      }
+      __syncthreads();
+      if (d < 256) {
+        int above = 0;
+        for (int w2 = warp + 1; w2 < 8; ++w2) above += scan_sh[w2];
+        suf[d] = v + above;
+      }
       if (d == 0) suf[256] = 0;
       __syncthreads();
-      for (int o = 1; o < 256; o <<= 1) {
-        const int v = (d < 256 && d + o < 256) ? suf[d + o] : 0;
-        __syncthreads();
-        if (d < 256) suf[d] += v;
-        __syncthreads();
-      }
       if (d < 256 && ((suf[d] >= remaining && suf[d + 1] < remaining) || (d == 0 && suf[0] < remaining))) {
         sh_prefix = prefix | (static_cast<uint32_t>(d) << shift);
         sh_remaining = remaining - suf[d + 1];
@@ -207,7 +238,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
   const int lo = min(n, static_cast<int>(threadIdx.x) * per), hi = min(n, lo + per);
   int gt = 0, eq = 0;
   for (int i = lo; i < hi; ++i) {
-    const uint32_t kb = key_bits(kp[i]);
+    const uint32_t kb = key_at(i);
     gt += kb > thr;
     eq += kb == thr;
   }
@@ -216,7 +247,7 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_kernel(const float* __restr
   int pos = pg + min(pe, remaining);
   int erank = pe;
   for (int i = lo; i < hi; ++i) {
-    const uint32_t kb = key_bits(kp[i]);
+    const uint32_t kb = key_at(i);
     bool take = kb > thr;
     if (kb == thr) {
       take = erank < remaining;

@@ -146,16 +146,17 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
 }
 
 // ---- job: gathered matrix dYsel[m, i] = bf16(dY[m, idx[i]]), pad columns [k_sel, pitch) zero ----
-// Whole rows of the gathered matrix leave as full 128-byte lines; the scattered 2- or 4-byte
-// reads of dY hit the sectors that the column-sum pass of the same launch brings into L2.
+// Whole rows of the gathered matrix leave as full 128-byte lines.  Block `slab` covers the rows
+// of that slab of the dY pass and sits next to the slab's column-sum blocks in launch order,
+// so its scattered 2- or 4-byte reads of dY meet the same sectors in L2 (or in flight to it).
 // The index list is staged in shared memory 1024 entries at a time.
-static const int GATHER_ROWS = 64;      // rows of dY per block
 template <typename T>
 __device__ __forceinline__ void job_gather(const PrepArgs& a, int block, int32_t* s_idx /* [1024] */) {
   const T* dY = static_cast<const T*>(a.dY);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t m_lo = static_cast<int64_t>(block) * GATHER_ROWS;
-  const int64_t m_hi = (m_lo + GATHER_ROWS < a.M) ? m_lo + GATHER_ROWS : a.M;
+  const int64_t rows = ceil_div(a.M, static_cast<int64_t>(a.slabs));
+  const int64_t m_lo = block * rows;
+  const int64_t m_hi = (m_lo + rows < a.M) ? m_lo + rows : a.M;
   for (int64_t ch = 0; ch < a.pitch; ch += 1024) {
     const int n = static_cast<int>((a.pitch - ch < 1024) ? a.pitch - ch : 1024);     // even: pitch % 16 == 0
     __syncthreads();
@@ -199,21 +200,24 @@ __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
   pdl_trigger();
   pdl_wait();
   const int b = blockIdx.x;
-  if (b < a.nb_g) {
-    job_gather<TX>(a, b, reinterpret_cast<int32_t*>(sh));
-  } else if (b < a.nb_g + a.nb_w) {
-    job_weights<W_MODE>(a, b - a.nb_g, a.nb_w);
-  } else if (b < a.nb_g + a.nb_w + a.nb_x) {
-    job_quant_x<TX>(a, b - a.nb_g - a.nb_w, a.nb_x);
+  if (b < a.nb_w) {
+    job_weights<W_MODE>(a, b, a.nb_w);
+  } else if (b < a.nb_w + a.nb_x) {
+    job_quant_x<TX>(a, b - a.nb_w, a.nb_x);
   } else {
-    const int r = b - a.nb_g - a.nb_w - a.nb_x;
-    job_dy_pass<TX>(a, r % a.col_blocks, r / a.col_blocks, sh);
+    // per slab of rows: [gather block,] then the column blocks of the dY pass
+    const int r = b - a.nb_w - a.nb_x;
+    const int per_slab = a.col_blocks * a.dy_on + a.nb_g;
+    const int slab = r / per_slab, j = r - slab * per_slab;
+    if (j < a.nb_g) job_gather<TX>(a, slab, reinterpret_cast<int32_t*>(sh));
+    else job_dy_pass<TX>(a, j - a.nb_g, slab, sh);
   }
 }
 
 // ---- finalize: dW rows (mask, dS_w, optional SGD) | dS_x, dZ_x | db ------------------------
 __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
   __shared__ double shd[2][256];
+  __shared__ float4 red[256];
   pdl_trigger();
   pdl_wait();
   const int b = blockIdx.x;
@@ -230,45 +234,72 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
     float sx = a.s_x[0];
     if (!scale_ok(sx)) sx = 1.f;
     const float* wrow = a.W + n * a.K;
+    // Short rows leave most of the block idle in the k loop, so the split partial products are
+    // shared out over G groups of threads and combined through shared memory in a fixed order.
+    const int nk4 = static_cast<int>(a.K >> 2);
+    int G = 1;
+    if (nk4 < 256) {
+      G = 256 / nk4;
+      if (G > a.splits) G = a.splits;
+      if (G < 1) G = 1;
+    }
+    const int kq = (G > 1) ? static_cast<int>(threadIdx.x) % nk4 : static_cast<int>(threadIdx.x);
+    const int sg = (G > 1) ? static_cast<int>(threadIdx.x) / nk4 : 0;
     double acc = 0.0;
-    for (int64_t k = threadIdx.x * 4; k < a.K; k += blockDim.x * 4) {
+    for (int64_t k0 = 0; k0 < a.K; k0 += 1024) {       // one pass unless K > 1024
+      const int64_t k = k0 + 4 * kq;
       float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int sp0 = 0; sp0 < a.splits; sp0 += 8) {       // eight independent loads in flight, summed in split order
-        float4 t[8];
+      if (k < a.K && sg < G) {
+        for (int sp0 = sg; sp0 < a.splits; sp0 += 8 * G) {       // eight independent loads in flight
+          float4 t[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-          t[u] = (sp0 + u < a.splits)
-                     ? __ldg(reinterpret_cast<const float4*>(a.P + (sp0 + u) * a.split_stride + i * a.K + k))
-                     : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int u = 0; u < 8; ++u)
+            t[u] = (sp0 + u * G < a.splits)
+                       ? __ldg(reinterpret_cast<const float4*>(a.P + (sp0 + u * G) * a.split_stride + i * a.K + k))
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          g.x += t[u].x; g.y += t[u].y; g.z += t[u].z; g.w += t[u].w;
+          for (int u = 0; u < 8; ++u) {
+            g.x += t[u].x; g.y += t[u].y; g.z += t[u].z; g.w += t[u].w;
+          }
         }
       }
-      const float4 w4 = *reinterpret_cast<const float4*>(wrow + k);
-      const float gv[4] = {g.x * sx, g.y * sx, g.z * sx, g.w * sx};
-      const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
-      float ov[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const QElem e = quant_weight(wv[j], p);
-        ov[j] = e.flag ? 0.f : gv[j];
-        acc += static_cast<double>(gv[j]) * static_cast<double>(e.t);
+      if (G > 1) {
+        __syncthreads();
+        red[threadIdx.x] = g;
+        __syncthreads();
+        if (sg == 0 && k < a.K) {
+          for (int j = 1; j < G; ++j) {
+            const float4 t = red[j * nk4 + kq];
+            g.x += t.x; g.y += t.y; g.z += t.z; g.w += t.w;
+          }
+        }
       }
-      *reinterpret_cast<float4*>(a.dW_sel + i * a.K + k) = make_float4(ov[0], ov[1], ov[2], ov[3]);
-      if (a.has_opt) {
-        const int64_t o = n * a.K + k;
-        const float4 w0 = *reinterpret_cast<const float4*>(a.opt.W_inout + o);
-        const float4 m0 = *reinterpret_cast<const float4*>(a.opt.mom_inout + o);
-        const float wi[4] = {w0.x, w0.y, w0.z, w0.w}, mi[4] = {m0.x, m0.y, m0.z, m0.w};
-        float wo[4], mo[4];
+      if (sg == 0 && k < a.K) {
+        const float4 w4 = *reinterpret_cast<const float4*>(wrow + k);
+        const float gv[4] = {g.x * sx, g.y * sx, g.z * sx, g.w * sx};
+        const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
+        float ov[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          mo[j] = a.opt.momentum * mi[j] + (ov[j] + a.opt.weight_decay * wi[j]);
-          wo[j] = wi[j] - a.opt.lr * mo[j];
+          const QElem e = quant_weight(wv[j], p);
+          ov[j] = e.flag ? 0.f : gv[j];
+          acc += static_cast<double>(gv[j]) * static_cast<double>(e.t);
         }
-        *reinterpret_cast<float4*>(a.opt.mom_inout + o) = make_float4(mo[0], mo[1], mo[2], mo[3]);
-        *reinterpret_cast<float4*>(a.opt.W_inout + o) = make_float4(wo[0], wo[1], wo[2], wo[3]);
+        *reinterpret_cast<float4*>(a.dW_sel + i * a.K + k) = make_float4(ov[0], ov[1], ov[2], ov[3]);
+        if (a.has_opt) {
+          const int64_t o = n * a.K + k;
+          const float4 w0 = *reinterpret_cast<const float4*>(a.opt.W_inout + o);
+          const float4 m0 = *reinterpret_cast<const float4*>(a.opt.mom_inout + o);
+          const float wi[4] = {w0.x, w0.y, w0.z, w0.w}, mi[4] = {m0.x, m0.y, m0.z, m0.w};
+          float wo[4], mo[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            mo[j] = a.opt.momentum * mi[j] + (ov[j] + a.opt.weight_decay * wi[j]);
+            wo[j] = wi[j] - a.opt.lr * mo[j];
+          }
+          *reinterpret_cast<float4*>(a.opt.mom_inout + o) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+          *reinterpret_cast<float4*>(a.opt.W_inout + o) = make_float4(wo[0], wo[1], wo[2], wo[3]);
+        }
       }
     }
     acc = warp_sum(acc);
@@ -281,9 +312,12 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
     }
   } else if (b == a.k_sel) {
     double x = 0.0, z = 0.0;
+    const float2* pp = reinterpret_cast<const float2*>(a.dx_partials);
+#pragma unroll 8
     for (int i = threadIdx.x; i < a.n_partials; i += 256) {
-      x += static_cast<double>(a.dx_partials[2 * i]);
-      z += static_cast<double>(a.dx_partials[2 * i + 1]);
+      const float2 t = pp[i];
+      x += static_cast<double>(t.x);
+      z += static_cast<double>(t.y);
     }
     shd[0][threadIdx.x] = x;
     shd[1][threadIdx.x] = z;
@@ -304,8 +338,10 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
     const int c = threadIdx.x & 31, j = threadIdx.x >> 5;
     const int64_t n = static_cast<int64_t>(b - a.k_sel - 1) * 32 + c;
     double acc = 0.0;
-    if (n < a.N)
+    if (n < a.N) {
+#pragma unroll 16
       for (int s = j; s < a.slabs; s += 8) acc += static_cast<double>(a.colsum_ws[static_cast<int64_t>(s) * a.N + n]);
+    }
     shd[0][threadIdx.x] = acc;
     __syncthreads();
     if (j == 0 && n < a.N) {
@@ -319,12 +355,13 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
 
 }  // namespace
 
-// Row slabs of the dY pass: blocks of 256 columns x one slab of rows, about 32 KiB of dY
-// each (at least 32 rows), so that the launch spreads over the whole GPU a few times.
+// Row slabs of the dY pass: blocks of 256 columns x one slab of rows, 64 rows (32 KiB of
+// bf16) each until there are 512 slabs; beyond that the slabs grow, so that the sum over the
+// slabs' column-sum partials stays short.
 int prepare_slabs(int64_t M, int64_t N) {
   (void)N;
   int64_t s = ceil_div(M, 64);
-  if (s > 2048) s = 2048;
+  if (s > 512) s = 512;
   if (s < 1) s = 1;
   return static_cast<int>(s);
 }
@@ -342,12 +379,12 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   a.nb_x = 0;
   if (a.Xc) a.nb_x = flat_blocks(a.x_count / 8, 256 * 8);   // 32 KiB (bf16) / 64 KiB (fp32) per block
   const bool gather = a.dY && a.dYsel && a.k_sel > 0 && a.k_sel < a.N;
-  a.nb_g = gather ? static_cast<int>(ceil_div(a.M, GATHER_ROWS)) : 0;
-  int nb_y = 0;
+  a.nb_g = gather ? 1 : 0;                       // gather blocks per slab
   a.col_blocks = static_cast<int>(ceil_div(a.N, 256));
   a.slabs = prepare_slabs(a.M, a.N);
-  if (a.dY && (a.colsum_ws || a.dYb)) nb_y = a.col_blocks * a.slabs;
-  const int grid = a.nb_g + a.nb_w + a.nb_x + nb_y;
+  a.dy_on = (a.dY && (a.colsum_ws || a.dYb)) ? 1 : 0;
+  const int nb_y = (a.col_blocks * a.dy_on + a.nb_g) * a.slabs;
+  const int grid = a.nb_w + a.nb_x + nb_y;
   count_launches(1);
   if (w_mode == 0) {
     if (act_bf16) launch_dependent(prepare_kernel<0, bf16>, grid, 256, 0, st, 1, a);

@@ -79,7 +79,7 @@ struct PrepArgs {
   const void* dY; bf16* dYb; float* colsum_ws;
   const int32_t* idx; int64_t k_sel, pitch; bf16* dYsel;
   int* status;
-  int nb_g, nb_w, nb_x, col_blocks, slabs;   // filled by launch_prepare
+  int nb_g, nb_w, nb_x, col_blocks, slabs, dy_on;   // filled by launch_prepare
 };
 int prepare_slabs(int64_t M, int64_t N);
 void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st);

@@ -200,17 +200,19 @@ __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
   pdl_trigger();
   pdl_wait();
   const int b = blockIdx.x;
-  if (b < a.nb_w) {
-    job_weights<W_MODE>(a, b, a.nb_w);
-  } else if (b < a.nb_w + a.nb_x) {
-    job_quant_x<TX>(a, b - a.nb_w, a.nb_x);
-  } else {
-    // per slab of rows: [gather block,] then the column blocks of the dY pass
-    const int r = b - a.nb_w - a.nb_x;
-    const int per_slab = a.col_blocks * a.dy_on + a.nb_g;
-    const int slab = r / per_slab, j = r - slab * per_slab;
+  const int per_slab = a.col_blocks * a.dy_on + a.nb_g;
+  const int nb_y = per_slab * a.slabs;
+  if (b < nb_y) {
+    // per slab of rows: [gather block,] then the column blocks of the dY pass.  These come first
+    // in launch order: the gather blocks are the longest dependent chains of the launch, and
+    // the short flat quantizer blocks behind them fill its tail.
+    const int slab = b / per_slab, j = b - slab * per_slab;
     if (j < a.nb_g) job_gather<TX>(a, slab, reinterpret_cast<int32_t*>(sh));
     else job_dy_pass<TX>(a, j - a.nb_g, slab, sh);
+  } else if (b < nb_y + a.nb_w) {
+    job_weights<W_MODE>(a, b - nb_y, a.nb_w);
+  } else {
+    job_quant_x<TX>(a, b - nb_y - a.nb_w, a.nb_x);
   }
 }
 

@@ -62,7 +62,14 @@ __global__ void __launch_bounds__(256) row_importance_kernel(const LayerEntry* _
       const float4* w4 = reinterpret_cast<const float4*>(w);
       const int n4 = e.K >> 2;
       int i = lane;
-      for (; i + 96 < n4; i += 128) {     // four independent 16-byte loads in flight per lane
+      for (; i + 224 < n4; i += 256) {    // eight independent 16-byte loads in flight per lane
+        float4 t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) t[u] = __ldg(w4 + i + 32 * u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc += abs4(t[u]);
+      }
+      for (; i + 96 < n4; i += 128) {     // four
         const float4 a = __ldg(w4 + i), b = __ldg(w4 + i + 32), c = __ldg(w4 + i + 64), d = __ldg(w4 + i + 96);
         acc += abs4(a);
         acc += abs4(b);

@@ -55,6 +55,7 @@ struct GemmParams {
   int BN;             // tile columns (multiple of 16, <= 256)
   int stages;
   int kps;            // k-blocks per stage: one barrier round trip covers kps * 64 contraction elements
+  int merged;         // MN-major operands arrive as one TMA box per 64-wide chunk and stage (plain matrices only)
   int b_stage_bytes;
   int splits;
   int tiles_m, tiles_n;
@@ -165,7 +166,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         n_eff = (n_eff + 15) & ~15;
         const int b_chunks = (n_eff + 63) >> 6;
         // bytes credited to the (leader's) full barrier per stage: both CTAs' copies in pair mode
-        const uint32_t tx = (CTA2 ? 2u : 1u) * (A_STAGE_BYTES + (B_MN ? b_chunks * CHUNK_BYTES : bn_cta * BK * 2));
+        // (a merged MN-major box always brings all kps k-blocks of its chunk, used or not)
+        const uint32_t tx_a = A_STAGE_BYTES, tx_b = B_MN ? b_chunks * CHUNK_BYTES : bn_cta * BK * 2;
+        const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
         // One barrier round trip costs ~0.3 us whatever it carries, so a stage holds several
@@ -180,35 +183,62 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           // the leader's barrier collects the bytes of both CTAs of a pair; only the leader arrives on it
-          if (rank == 0) mbar_arrive_expect_tx(&ctl->full[s], tx * nsub);
+          if (rank == 0)
+            mbar_arrive_expect_tx(&ctl->full[s], (CTA2 ? 2u : 1u) * (tx_a * (a_mrg ? p.kps : nsub) +
+                                                                    tx_b * (b_mrg ? p.kps : nsub)));
+          uint8_t* a_reg = smem + s * stage_bytes;               // [kps k-blocks of A][kps k-blocks of B]
+          uint8_t* b_reg = a_reg + p.kps * A_STAGE_BYTES;
+          if (a_mrg || b_mrg) {
+            // one box of kps * 64 contraction rows per 64-wide chunk: chunk c sits at c * kps * 8 KiB
+            const uint32_t fb = CTA2 ? mapa_u32(smem_u32(&ctl->full[s]), 0) : 0u;
+            const int chunk_stride = p.kps * CHUNK_BYTES;
+            if (a_mrg) {
+              for (int c = 0; c < 2; ++c) {
+                if (CTA2) tma_load_2d_pair(a_reg + c * chunk_stride, &tmA, fb, m0 + 64 * c, kb0 * BK);
+                else tma_load_2d(a_reg + c * chunk_stride, &tmA, &ctl->full[s], m0 + 64 * c, kb0 * BK);
+              }
+            }
+            if (b_mrg) {
+              for (int c = 0; c < b_chunks; ++c) {
+                if (CTA2) tma_load_2d_pair(b_reg + c * chunk_stride, &tmB, fb, n0 + 64 * c, kb0 * BK);
+                else tma_load_2d(b_reg + c * chunk_stride, &tmB, &ctl->full[s], n0 + 64 * c, kb0 * BK);
+              }
+            }
+          }
          for (int u = 0; u < nsub; ++u) {
           const int kb = kb0 + u;
-          uint8_t* sa = smem + s * stage_bytes + u * sub_bytes;
-          uint8_t* sb = sa + A_STAGE_BYTES;
+          uint8_t* sa = a_reg + u * A_STAGE_BYTES;
+          uint8_t* sb = b_reg + u * p.b_stage_bytes;
           if (CTA2) {
             const uint32_t fb = mapa_u32(smem_u32(&ctl->full[s]), 0);
             if (A_MN) {
-              tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
-              tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
+              if (!a_mrg) {
+                tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
+                tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
+              }
             } else {
               tma_load_2d_pair(sa, &tmA, fb, kb * BK, m0);
             }
             if (B_MN) {
-              for (int c = 0; c < b_chunks; ++c)
-                tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
+              if (!b_mrg)
+                for (int c = 0; c < b_chunks; ++c)
+                  tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
             } else {
               tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
             }
           } else if (p.cv.mode == 0) {
             if (A_MN) {
-              tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
-              tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+              if (!a_mrg) {
+                tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
+                tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+              }
             } else {
               tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
             }
             if (B_MN) {
-              for (int c = 0; c < b_chunks; ++c)
-                tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
+              if (!b_mrg)
+                for (int c = 0; c < b_chunks; ++c)
+                  tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
             } else {
               tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
             }
@@ -292,15 +322,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tc_fence_after();
          for (int u = 0; u < nsub; ++u) {
           const int kb = kb0 + u;
-          const uint32_t a_addr = smem_u32(smem + s * stage_bytes + u * sub_bytes);
-          const uint32_t b_addr = a_addr + A_STAGE_BYTES;
+          // k-block u of the stage: merged MN-major operands keep their chunks kps * 8 KiB apart
+          const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
+          const uint32_t a_base = smem_u32(smem + s * stage_bytes);
+          const uint32_t b_base = a_base + p.kps * A_STAGE_BYTES;
+          const uint32_t a_addr = a_base + u * (a_mrg ? CHUNK_BYTES : A_STAGE_BYTES);
+          const uint32_t b_addr = b_base + u * (b_mrg ? CHUNK_BYTES : p.b_stage_bytes);
+          const uint32_t a_lbo = a_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
+          const uint32_t b_lbo = b_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // K-major: 16 contraction elements = 32 bytes inside the swizzled 128-byte row.
             // MN-major: 16 contraction elements = 16 rows of 128 bytes = two 8-row groups.
-            const uint64_t adesc = A_MN ? smem_desc_sw128(a_addr + k * 2048, CHUNK_BYTES, 1024)
+            const uint64_t adesc = A_MN ? smem_desc_sw128(a_addr + k * 2048, a_lbo, 1024)
                                         : smem_desc_sw128(a_addr + k * 32, 16, 1024);
-            const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, CHUNK_BYTES, 1024)
+            const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, b_lbo, 1024)
                                         : smem_desc_sw128(b_addr + k * 32, 16, 1024);
             if (CTA2) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
             else umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
@@ -785,6 +821,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   if (kps > 4) kps = 4;
   if (kps > p.nkb) kps = p.nkb;
   p.kps = kps;
+  p.merged = cv ? 0 : 1;
   const int stage_bytes = kps * sub_bytes;
   int stages = ring_bytes / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -809,9 +846,10 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   CUtensorMap ta, tb, to, tx;
   if (a.epi == EPI_DX && (a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;
   if (!cv) {
-    rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
+    // MN-major operands: one box = all kps k-blocks of a stage for one 64-wide chunk
+    rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK * kps) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
     if (rc != EFQAT_OK) return rc;
-    rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, bn_cta);
+    rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK * kps) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, bn_cta);
     if (rc != EFQAT_OK) return rc;
     to = ta;
     tx = ta;

@@ -155,9 +155,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane == 0) {
+    // Lane 0 owns the barrier protocol; the copies of a stage are issued by several lanes at
+    // once (a single thread spends ~0.06 us per bulk tensor copy, which bounds narrow tiles).
+    // Lanes 0..5 take the merged MN-major boxes (A chunks 0-1, B chunks 0-3); lanes 8.. take
+    // the per-k-block copies, two lanes per k-block (A operand, B operand).
+    {
       int it = 0;
-      for (int w = unit; w < total_items && !*abort_flag; w += num_units) {
+      bool live = true;
+      for (int w = unit; w < total_items && live; w += num_units) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
         const int m0 = (t / p.tiles_n) * TILE_M + rank * BM;
         const int n0 = (t % p.tiles_n) * p.BN + rank * bn_cta;     // first B column staged by this CTA
@@ -177,111 +182,124 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1;
-          if (*abort_flag || !mbar_wait(&ctl->empty[s], ph ^ 1)) {
-            record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
-            *abort_flag = 1;
+          int ok_stage = 1;
+          if (lane == 0) {
+            if (*abort_flag || !mbar_wait(&ctl->empty[s], ph ^ 1)) {
+              record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
+              *abort_flag = 1;
+              ok_stage = 0;
+            } else if (rank == 0) {
+              // the leader's barrier collects the bytes of both CTAs of a pair; only the leader arrives on it
+              mbar_arrive_expect_tx(&ctl->full[s], (CTA2 ? 2u : 1u) * (tx_a * (a_mrg ? p.kps : nsub) +
+                                                                      tx_b * (b_mrg ? p.kps : nsub)));
+            }
+          }
+          ok_stage = __shfl_sync(0xffffffffu, ok_stage, 0);
+          if (!ok_stage) {
+            live = false;
             break;
           }
-          // the leader's barrier collects the bytes of both CTAs of a pair; only the leader arrives on it
-          if (rank == 0)
-            mbar_arrive_expect_tx(&ctl->full[s], (CTA2 ? 2u : 1u) * (tx_a * (a_mrg ? p.kps : nsub) +
-                                                                    tx_b * (b_mrg ? p.kps : nsub)));
           uint8_t* a_reg = smem + s * stage_bytes;               // [kps k-blocks of A][kps k-blocks of B]
           uint8_t* b_reg = a_reg + p.kps * A_STAGE_BYTES;
-          if (a_mrg || b_mrg) {
+          const uint32_t fb = CTA2 ? mapa_u32(smem_u32(&ctl->full[s]), 0) : 0u;
+          if (lane < 6) {
             // one box of kps * 64 contraction rows per 64-wide chunk: chunk c sits at c * kps * 8 KiB
-            const uint32_t fb = CTA2 ? mapa_u32(smem_u32(&ctl->full[s]), 0) : 0u;
             const int chunk_stride = p.kps * CHUNK_BYTES;
-            if (a_mrg) {
-              for (int c = 0; c < 2; ++c) {
-                if (CTA2) tma_load_2d_pair(a_reg + c * chunk_stride, &tmA, fb, m0 + 64 * c, kb0 * BK);
-                else tma_load_2d(a_reg + c * chunk_stride, &tmA, &ctl->full[s], m0 + 64 * c, kb0 * BK);
-              }
+            if (a_mrg && lane < 2) {
+              const int c = lane;
+              if (CTA2) tma_load_2d_pair(a_reg + c * chunk_stride, &tmA, fb, m0 + 64 * c, kb0 * BK);
+              else tma_load_2d(a_reg + c * chunk_stride, &tmA, &ctl->full[s], m0 + 64 * c, kb0 * BK);
             }
-            if (b_mrg) {
-              for (int c = 0; c < b_chunks; ++c) {
-                if (CTA2) tma_load_2d_pair(b_reg + c * chunk_stride, &tmB, fb, n0 + 64 * c, kb0 * BK);
-                else tma_load_2d(b_reg + c * chunk_stride, &tmB, &ctl->full[s], n0 + 64 * c, kb0 * BK);
-              }
+            if (b_mrg && lane >= 2 && lane - 2 < b_chunks) {
+              const int c = lane - 2;
+              if (CTA2) tma_load_2d_pair(b_reg + c * chunk_stride, &tmB, fb, n0 + 64 * c, kb0 * BK);
+              else tma_load_2d(b_reg + c * chunk_stride, &tmB, &ctl->full[s], n0 + 64 * c, kb0 * BK);
             }
           }
-         for (int u = 0; u < nsub; ++u) {
-          const int kb = kb0 + u;
-          uint8_t* sa = a_reg + u * A_STAGE_BYTES;
-          uint8_t* sb = b_reg + u * p.b_stage_bytes;
-          if (CTA2) {
-            const uint32_t fb = mapa_u32(smem_u32(&ctl->full[s]), 0);
-            if (A_MN) {
-              if (!a_mrg) {
-                tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
-                tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
+          const int u = (lane - 8) >> 1;
+          const bool do_a = lane >= 8 && u < nsub && !(lane & 1) && !a_mrg;
+          const bool do_b = lane >= 8 && u < nsub && (lane & 1) && !b_mrg;
+          if (do_a || do_b) {
+            const int kb = kb0 + u;
+            uint8_t* sa = a_reg + u * A_STAGE_BYTES;
+            uint8_t* sb = b_reg + u * p.b_stage_bytes;
+            if (CTA2) {
+              if (do_a) {
+                if (A_MN) {
+                  tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
+                  tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
+                } else {
+                  tma_load_2d_pair(sa, &tmA, fb, kb * BK, m0);
+                }
+              } else {
+                if (B_MN) {
+                  for (int c = 0; c < b_chunks; ++c)
+                    tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
+                } else {
+                  tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
+                }
+              }
+            } else if (p.cv.mode == 0) {
+              if (do_a) {
+                if (A_MN) {
+                  tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
+                  tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+                } else {
+                  tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
+                }
+              } else {
+                if (B_MN) {
+                  for (int c = 0; c < b_chunks; ++c)
+                    tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
+                } else {
+                  tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+                }
+              }
+            } else if (p.cv.mode == 3) {
+              // grad-weight: contraction block kb = one box of 64 output pixels; tile rows = (tap, channel)
+              const int bw = kb % p.cv.tiles_w, bh = (kb / p.cv.tiles_w) % p.cv.tiles_h;
+              const int bb = kb / (p.cv.tiles_w * p.cv.tiles_h);
+              const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
+              if (do_a) {
+                for (int j = 0; j < 2; ++j) {
+                  const int k = m0 + 64 * j;
+                  int rs = k / p.cv.C, c = k - rs * p.cv.C;
+                  if (rs >= p.cv.R * p.cv.S) { rs = 0; c = p.cv.C; }     // past the last tap: all zeros
+                  const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
+                  tma_load_4d(sa + j * CHUNK_BYTES, &tmA, &ctl->full[s], c, w0 + sx - p.cv.pad, h0 + r - p.cv.pad, b0);
+                }
+              } else {
+                for (int c = 0; c < b_chunks; ++c)
+                  tma_load_4d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, w0, h0, b0);
               }
             } else {
-              tma_load_2d_pair(sa, &tmA, fb, kb * BK, m0);
-            }
-            if (B_MN) {
-              if (!b_mrg)
-                for (int c = 0; c < b_chunks; ++c)
-                  tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
-            } else {
-              tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
-            }
-          } else if (p.cv.mode == 0) {
-            if (A_MN) {
-              if (!a_mrg) {
-                tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
-                tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
-              }
-            } else {
-              tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
-            }
-            if (B_MN) {
-              if (!b_mrg)
-                for (int c = 0; c < b_chunks; ++c)
-                  tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
-            } else {
-              tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
-            }
-          } else if (p.cv.mode == 3) {
-            // grad-weight: contraction block kb = one box of 64 output pixels; tile rows = (tap, channel)
-            const int bw = kb % p.cv.tiles_w, bh = (kb / p.cv.tiles_w) % p.cv.tiles_h;
-            const int bb = kb / (p.cv.tiles_w * p.cv.tiles_h);
-            const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
-            for (int j = 0; j < 2; ++j) {
-              const int k = m0 + 64 * j;
-              int rs = k / p.cv.C, c = k - rs * p.cv.C;
-              if (rs >= p.cv.R * p.cv.S) { rs = 0; c = p.cv.C; }     // past the last tap: all zeros
+              // forward / grad-input: tile rows = one box of 128 pixels; contraction block kb = (tap, 64 channels)
+              const int tmi = t / p.tiles_n;
+              const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
+              const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
+              const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
+              const int rs = kb / p.cv.cchunks, cc = kb - rs * p.cv.cchunks;
               const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
-              tma_load_4d(sa + j * CHUNK_BYTES, &tmA, &ctl->full[s], c, w0 + sx - p.cv.pad, h0 + r - p.cv.pad, b0);
-            }
-            for (int c = 0; c < b_chunks; ++c)
-              tma_load_4d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, w0, h0, b0);
-          } else {
-            // forward / grad-input: tile rows = one box of 128 pixels; contraction block kb = (tap, 64 channels)
-            const int tmi = t / p.tiles_n;
-            const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
-            const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
-            const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
-            const int rs = kb / p.cv.cchunks, cc = kb - rs * p.cv.cchunks;
-            const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
-            const int dw = (p.cv.mode == 1) ? sx - p.cv.pad : p.cv.pad - sx;
-            const int dh = (p.cv.mode == 1) ? r - p.cv.pad : p.cv.pad - r;
-            tma_load_4d(sa, &tmA, &ctl->full[s], cc * 64, w0 + dw, h0 + dh, b0);
-            if (B_MN) {     // W^ viewed as [N rows, R*S*Cin columns]: rows = contraction, Nc = Cin
-              for (int c = 0; c < b_chunks; ++c)
-                tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s],
-                            rs * static_cast<int>(p.Nc) + n0 + 64 * c, cc * 64);
-            } else {        // weight codes [N, R*S*Cin]
-              tma_load_2d(sb, &tmB, &ctl->full[s], rs * p.cv.C + cc * 64, n0);
+              const int dw = (p.cv.mode == 1) ? sx - p.cv.pad : p.cv.pad - sx;
+              const int dh = (p.cv.mode == 1) ? r - p.cv.pad : p.cv.pad - r;
+              if (do_a) {
+                tma_load_4d(sa, &tmA, &ctl->full[s], cc * 64, w0 + dw, h0 + dh, b0);
+              } else if (B_MN) {     // W^ viewed as [N rows, R*S*Cin columns]: rows = contraction, Nc = Cin
+                for (int c = 0; c < b_chunks; ++c)
+                  tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s],
+                              rs * static_cast<int>(p.Nc) + n0 + 64 * c, cc * 64);
+              } else {               // weight codes [N, R*S*Cin]
+                tma_load_2d(sb, &tmB, &ctl->full[s], rs * p.cv.C + cc * 64, n0);
+              }
             }
           }
-         }
+          __syncwarp();
         }
       }
       // Make sure none of this CTA's bulk copies is still in flight when it exits (only
       // relevant after an abort: otherwise the MMA warp has consumed every stage).
       const int issued = it;
-      if (rank == 0)
+      if (lane == 0 && rank == 0)
         for (int j = (issued > p.stages ? issued - p.stages : 0); j < issued; ++j)
           mbar_wait(&ctl->full[j % p.stages], (j / p.stages) & 1, 20000000ull);
     }
@@ -769,7 +787,11 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   // CTA pairs (256 x BN tiles, tiles full in N) halve the B traffic from L2 per FLOP; they are
   // taken unless one-CTA tiles fill the machine's last wave clearly better.
   int pair = 0;
-  if (!cv && a.epi != EPI_PART && a.Mr >= 256 && a.Nc % 128 == 0) {
+  // (full weight-gradient GEMM: measured gain only on long runs of tiles, 1.18-1.33x at >= 1024 pair
+  // tiles, a loss at 256)
+  const bool part_pair = a.a_mn && a.b_mn && a.splits == 1 && a.Nc % 256 == 0 &&
+                         ceil_div(a.Mr, 2 * BM) * (a.Nc / 256) >= 4 * static_cast<int64_t>(sm_count);
+  if (!cv && (a.epi != EPI_PART || part_pair) && a.Mr >= 256 && a.Nc % 128 == 0) {
     const int units = sm_count / 2;
     const int64_t mt = ceil_div(a.Mr, 2 * BM);
     const bool can256 = a.Nc % 256 == 0;
@@ -905,7 +927,10 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
     if (pair) EFQAT_LAUNCH(0, 1, EPI_DX, 1);
     EFQAT_LAUNCH(0, 1, EPI_DX, 0);
   }
-  if (a.epi == EPI_PART && a.a_mn && a.b_mn) EFQAT_LAUNCH(1, 1, EPI_PART, 0);
+  if (a.epi == EPI_PART && a.a_mn && a.b_mn) {
+    if (pair) EFQAT_LAUNCH(1, 1, EPI_PART, 1);
+    EFQAT_LAUNCH(1, 1, EPI_PART, 0);
+  }
   if (a.epi == EPI_PART && !a.a_mn && !a.b_mn) EFQAT_LAUNCH(0, 0, EPI_PART, 0);
   if (a.epi == EPI_PART && !a.a_mn && a.b_mn) EFQAT_LAUNCH(0, 1, EPI_PART, 0);
   if (a.epi == EPI_PART && a.a_mn && !a.b_mn) EFQAT_LAUNCH(1, 0, EPI_PART, 0);

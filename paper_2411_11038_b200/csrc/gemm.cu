@@ -384,6 +384,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     ActQ xq = {};
     if (EPI != EPI_PART) xq = make_actq(p.s_x, p.z_x, p.x_bits, p.x_sym, nullptr);
     const float t_lo = xq.lo - xq.zr, t_hi = xq.hi - xq.zr;     // d/ds of a clipped element
+    const float q_half = 0.5f * (xq.hi - xq.lo), z_mid = xq.zr - 0.5f * (xq.hi + xq.lo);
 
     struct Geo {
       int t, split, n0, n_eff, row0, jb0, jb1, pw0, ph0, pb0;
@@ -562,19 +563,37 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y);
                   x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
                 }
+                // Eq. 1 with the straight-through estimator, the arithmetic of quant_act().  An
+                // element is clipped iff |rne(x/s) + Z - mid| > half (all operands are multiples
+                // of 0.5 below 2^23: exact).  Groups in which no lane of the warp has a clipped
+                // element skip the selects and the zero-point sum.
+                float rq[8], dq[8];
+                bool any_clip = false;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                  // Eq. 1 with the straight-through estimator, the arithmetic of quant_act()
-                  const float gx = __uint_as_float(r[gi * 8 + j]);
-                  const float rq = rne_small(__fmul_rn(x[j], xq.rinv));
-                  const float cq = rq + xq.zr;
-                  const bool below = cq < xq.lo, above = cq > xq.hi;
-                  const float resid = fmaf(-x[j], xq.rinv_lo, fmaf(-x[j], xq.rinv, rq));
-                  const float tq = below ? t_lo : (above ? t_hi : resid);
-                  const bool clipped = below || above;
-                  v[j] = clipped ? 0.f : gx;
-                  acc_s = fmaf(gx, tq, acc_s);
-                  acc_c += clipped ? gx : 0.f;
+                  rq[j] = rne_small(__fmul_rn(x[j], xq.rinv));
+                  dq[j] = rq[j] + z_mid;
+                  any_clip = any_clip || fabsf(dq[j]) > q_half;
+                }
+                if (!__any_sync(0xffffffffu, any_clip)) {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    const float gx = __uint_as_float(r[gi * 8 + j]);
+                    const float resid = fmaf(-x[j], xq.rinv_lo, fmaf(-x[j], xq.rinv, rq[j]));
+                    v[j] = gx;
+                    acc_s = fmaf(gx, resid, acc_s);
+                  }
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    const float gx = __uint_as_float(r[gi * 8 + j]);
+                    const bool clipped = fabsf(dq[j]) > q_half;
+                    const float resid = fmaf(-x[j], xq.rinv_lo, fmaf(-x[j], xq.rinv, rq[j]));
+                    const float tq = clipped ? (dq[j] < 0.f ? t_lo : t_hi) : resid;
+                    v[j] = clipped ? 0.f : gx;
+                    acc_s = fmaf(gx, tq, acc_s);
+                    acc_c += clipped ? gx : 0.f;
+                  }
                 }
               }
               if (bc == 32) {

@@ -132,6 +132,7 @@ class Workload:
             views = [plan.idx[offs[i]:offs[i + 1]] if ks[i] else None for i in range(len(ks))]
             self.sel[f] = (plan, ks, views)
         self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+        self.copy_stream = None
 
     def flops(self, frac, fwd=True, bwd=True):
         tot = 0.0
@@ -167,12 +168,29 @@ class Workload:
 
     def step_e2e(self, frac):
         """Same step with this step's activations coming from pinned host memory and the
-        parameter gradients going back to it."""
-        _, ks, _ = self.sel[frac]
-        for c, D, plan in self.layers:
-            D["X"].copy_(D["host_X"], non_blocking=True)
-            D["dY"].copy_(D["host_dY"], non_blocking=True)
-        self.step(frac)
+        parameter gradients going back to it.  The host-to-device copies run on a second
+        stream in the order the layers need them, so a layer's kernels start as soon as its
+        own inputs have landed; everything is ordered back into the timed stream."""
+        _, ks, views = self.sel[frac]
+        cur = torch.cuda.current_stream()
+        if self.copy_stream is None:
+            self.copy_stream = torch.cuda.Stream()
+        self.copy_stream.wait_stream(cur)          # the previous step has finished with the buffers
+        ev_x, ev_dy = [], []
+        with torch.cuda.stream(self.copy_stream):
+            for c, D, plan in self.layers:
+                D["X"].copy_(D["host_X"], non_blocking=True)
+                ev_x.append(self.copy_stream.record_event())
+            for c, D, plan in self.layers:
+                D["dY"].copy_(D["host_dY"], non_blocking=True)
+                ev_dy.append(self.copy_stream.record_event())
+        self.select(frac)
+        for (c, D, plan), e in zip(self.layers, ev_x):
+            cur.wait_event(e)
+            plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"])
+        for (c, D, plan), k, idx, e in zip(self.layers, ks, views, ev_dy):
+            cur.wait_event(e)
+            plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True)
         for (c, D, plan), k in zip(self.layers, ks):
             if k:
                 D["host_dW"][:k].copy_(plan.dW_sel[:k], non_blocking=True)

@@ -435,6 +435,9 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.split_stride = k_sel * K;
     g.part_cols = k_sel;
     g.status = ctx->d_status;
+    // reads only what the prepare launch wrote, which the grad-input GEMM just before it has
+    // already waited for: free to run beside that GEMM on the SMs it leaves idle
+    g.defer_wait = 1;
     rc = timed_gemm(ctx, 2, g, st);
     if (rc != EFQAT_OK) return rc;
   }

@@ -70,6 +70,7 @@ struct GemmParams {
   int64_t split_stride;
   int64_t part_cols;
   int* status;
+  int defer_wait;
 };
 
 struct __align__(16) SmemCtl {
@@ -149,8 +150,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   // barriers, TMEM and descriptor prefetches are in place; everything below reads global memory
+  // The launch before this one is complete (its writes visible) before this one lets the next
+  // launch start.  A launch that reads nothing of its direct predecessor (defer_wait: the
+  // weight-gradient GEMM behind the grad-input GEMM, both fed by the prepare launch that the
+  // grad-input GEMM has already waited for) starts at once on whatever SMs are free and only
+  // holds its exit until the predecessor is done, so that launches behind it still see both.
+  if (!p.defer_wait) pdl_wait();
   pdl_trigger();
-  pdl_wait();
   volatile int* abort_flag = &ctl->abort_flag;
 
   if (warp == 0) {
@@ -650,6 +656,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (CTA2) cluster_sync();     // neither CTA leaves while its peer may still signal its barriers
+  if (p.defer_wait && threadIdx.x == 0) pdl_wait();
   if (warp == 1) {
     if (CTA2) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
   }
@@ -883,6 +890,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   p.split_stride = a.split_stride;
   p.part_cols = a.part_cols;
   p.status = a.status;
+  p.defer_wait = a.defer_wait;
 
   CUtensorMap ta, tb, to, tx;
   if (a.epi == EPI_DX && (a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;

@@ -149,6 +149,10 @@ struct GemmArgs {
   int64_t split_stride;
   int64_t part_cols;
   int* status;
+  // 1: this launch reads nothing that the launch directly before it in the stream writes, and
+  // everything else it reads was complete before that launch began its work; it may then run
+  // beside its predecessor (see gemm_kernel)
+  int defer_wait;
 };
 // Number of (dS_x, dZ_x) partial pairs EPI_DX writes for this problem.
 int gemm_dx_num_partials(int64_t Mr, int64_t Nc);

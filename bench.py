@@ -133,6 +133,7 @@ class Workload:
             self.sel[f] = (plan, ks, views)
         self.flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
         self.copy_stream = None
+        self.side_stream = None
 
     def flops(self, frac, fwd=True, bwd=True):
         tot = 0.0
@@ -161,9 +162,18 @@ class Workload:
             plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True)
 
     def step(self, frac):
-        self.select(frac)
+        """Selection only reads the weights and only the backward needs its result, so it runs
+        on a second stream beside the forward launches and is joined before the backward."""
+        cur = torch.cuda.current_stream()
+        if self.side_stream is None:
+            self.side_stream = torch.cuda.Stream()
+        self.side_stream.wait_stream(cur)
+        with torch.cuda.stream(self.side_stream):
+            self.select(frac)
+            joined = self.side_stream.record_event()
         for c, D, plan in self.layers:
             plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"])
+        cur.wait_event(joined)
         self.backward(frac)
 
     def step_e2e(self, frac):

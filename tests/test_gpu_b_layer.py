@@ -137,3 +137,38 @@ def test_host_errors(ctx):
     with pytest.raises(B.EfqatError) as e:     # partial selection without indices
         B.fq_linear_bwd(ctx, D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], None, 5, 8, 8, False)
     assert e.value.code == -1
+
+
+def test_backward_back_to_back_on_one_workspace(ctx):
+    """Two different problems alternate through ONE plan (one workspace) without any host
+    synchronisation in between.  The weight-gradient GEMM runs beside the grad-input GEMM of
+    the same call; if it ever started before that call's producers had finished it would
+    contract the previous problem's codes, which differ everywhere."""
+    M, K, N = 512, 256, 384
+    dev = torch.device("cuda", 0)
+    cases = [_case("b2b_a", M, K, N, torch.bfloat16, seed=11), _case("b2b_b", M, K, N, torch.bfloat16, seed=12)]
+    probs = []
+    for c in cases:
+        T = I.make_tensors(c)
+        s_w, s_x, z_x = U.oracle_qparams(c, T, (0.8, 0.9, 1.3))
+        D = U.to_dev(T, s_w, s_x, z_x)
+        idx_np = np.arange(1, N, 5, dtype=np.int32)
+        idx = torch.from_numpy(idx_np).to(dev)
+        X64, W64, dY64 = I.as_f64(T["X"]), I.as_f64(T["W"]), I.as_f64(T["dY"])
+        ref = O.backward_efqat(dY64, X64, W64, s_w, s_x, z_x, idx_np, c.w_bits, c.x_bits, c.x_symmetric,
+                               operand_model="bf16")
+        probs.append((D, idx, len(idx_np), ref))
+    plan = B.LayerPlan(ctx, M, N, K, torch.bfloat16, 8, 8, False, N, dev)
+    got = []
+    for rep in range(6):
+        D, idx, k, _ = probs[rep % 2]
+        out = plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True)
+        got.append({key: out[key][:k].clone() if key in ("dW_sel", "dS_w_sel") else out[key].clone()
+                    for key in ("dW_sel", "dS_w_sel", "dX", "dS_x")})
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for rep, g in enumerate(got):
+        ref = probs[rep % 2][3]
+        U.assert_fp32_class(U.np32(g["dW_sel"]), ref["dW_sel"], ref["G_w_sel_abs"], f"rep {rep} dW_sel")
+        U.assert_fp32_class(U.np32(g["dX"]), ref["dX"], ref["G_x_abs"], f"rep {rep} dX", out_is_bf16=True)
+        U.assert_fp32_class(U.np32(g["dS_x"])[0], ref["dS_x"], ref["dS_x_abs"], f"rep {rep} dS_x", atol=1e-30)

@@ -38,7 +38,7 @@ METRIC = "fq-linear step TFLOP/s (select + fwd + partial bwd); bwd TFLOP/s and s
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (set to None whenever the kernel changes after a capture).
-DOMINANT_TRAFFIC_BYTES = 28.96e6    # mean over the four dX launches of one step (profiles/gemm_kernel_dx_bench_cfg2.txt)
+DOMINANT_TRAFFIC_BYTES = 28.93e6    # mean over the four dX launches of one step (profiles/gemm_kernel_dx_bench_cfg2.txt)
 
 
 def load_peaks():

@@ -135,11 +135,12 @@ int guard_device(const efqat_ctx* ctx) {
 int last_error() { return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA; }
 
 // run_gemm, bracketed by a pair of events when per-kernel timing is switched on.
-int timed_gemm(efqat_ctx* ctx, int kind, const GemmArgs& g, cudaStream_t st, int* tiles = nullptr) {
+int timed_gemm(efqat_ctx* ctx, int kind, const GemmArgs& g, cudaStream_t st, int* tiles = nullptr,
+               int* grid = nullptr) {
   const bool rec = ctx->prof_on && ctx->ev_used[kind] < PROF_RING;
   const int slot = ctx->ev_used[kind];
   if (rec) cudaEventRecord(ctx->ev[kind][2 * slot], st);
-  const int rc = run_gemm(g, ctx->sm_count, st, tiles);
+  const int rc = run_gemm(g, ctx->sm_count, st, tiles, grid);
   if (rec) {
     cudaEventRecord(ctx->ev[kind][2 * slot + 1], st);
     ctx->ev_used[kind] = slot + 1;
@@ -398,7 +399,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   pa.status = ctx->d_status;
   launch_prepare(pa, 1, act_bf16, st);
   // a4 + a5: dX = (dY W^) masked, with the dS_x / dZ_x partial sums in the epilogue
-  int tiles = 0;
+  int tiles = 0, dx_grid = 0, dw_splits = w.splits;
   const bool sconv = spatial_conv(layer);
   ConvArgs cv_dx = conv_args(layer, 2), cv_dw = conv_args(layer, 3);
   {
@@ -417,7 +418,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.X = X; g.x_dtype = layer->act_dtype;
     g.partials = w.dxpart;
     g.status = ctx->d_status;
-    rc = timed_gemm(ctx, 1, g, st, &tiles);
+    rc = timed_gemm(ctx, 1, g, st, &tiles, &dx_grid);
     if (rc != EFQAT_OK) return rc;
   }
   // a6: weight gradient of the unfrozen channels only, as split partial products
@@ -431,7 +432,19 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
     g.a_mn = 1; g.b_mn = 1;
     g.epi = EPI_PART;
     g.out = w.P; g.ldo = K;
-    g.splits = w.splits;
+    // The weight-gradient GEMM starts beside the grad-input GEMM (defer_wait below).  When the
+    // SMs that GEMM leaves idle can hold one CTA per output tile, the contraction is split only
+    // as far as those SMs go: every CTA then runs at once and the finalize launch sums fewer
+    // partial products.  Otherwise the split sized for the whole GPU stands.
+    int splits = w.splits;
+    if (!sconv) {
+      const int64_t dw_tiles = gemm_part_tiles(g.Mr, g.Nc);
+      const int64_t idle = ctx->sm_count - dx_grid;
+      if (idle >= dw_tiles && dw_tiles * splits > idle) splits = static_cast<int>(idle / dw_tiles);
+      if (splits < 1) splits = 1;
+    }
+    g.splits = splits;
+    dw_splits = splits;
     g.split_stride = k_sel * K;
     g.part_cols = k_sel;
     g.status = ctx->d_status;
@@ -444,7 +457,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   // a5 (+ a7): one launch: dW rows (mask, dS_w, optional SGD), dS_x / dZ_x, db
   FinArgs fa = {};
   fa.N = N; fa.K = K; fa.k_sel = k_sel;
-  fa.P = w.P; fa.splits = w.splits; fa.split_stride = k_sel * K;
+  fa.P = w.P; fa.splits = dw_splits; fa.split_stride = k_sel * K;
   fa.W = W; fa.s_w = s_w; fa.s_x = s_x; fa.w_bits = q->w_bits;
   fa.idx = gathered ? idx : nullptr;
   fa.dW_sel = dW_sel; fa.dS_w_sel = dS_w_sel;

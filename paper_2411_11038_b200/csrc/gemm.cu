@@ -761,6 +761,8 @@ static int part_bn(int64_t Nc) {
   return (Nc <= 64) ? static_cast<int>(round_up(Nc, 16)) : (Nc <= 128 ? 128 : 256);
 }
 
+int64_t gemm_part_tiles(int64_t Mr, int64_t Nc) { return ceil_div(Mr, BM) * ceil_div(Nc, part_bn(Nc)); }
+
 int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
   const int64_t nkb = ceil_div(Kc, BK);
   const int64_t tiles = ceil_div(Mr, BM) * ceil_div(Nc, part_bn(Nc));
@@ -792,7 +794,7 @@ static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMa
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
-int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
+int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, int* grid_out) {
   if (a.Mr < 1 || a.Nc < 1 || a.Kc < 1) return EFQAT_ERR_SHAPE;
   int rc = gemm_init();
   if (rc != EFQAT_OK) return rc;
@@ -944,6 +946,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out) {
   const int grid = pair ? 2 * units : units;
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + fixed_bytes + 1024;
   if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * EPI_WARPS;
+  if (grid_out) *grid_out = grid;
 
 #define EFQAT_LAUNCH(AM, BMj, E, P2) return launch<AM, BMj, E, P2>(ta, tb, to, tx, p, grid, smem, st)
   if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) {

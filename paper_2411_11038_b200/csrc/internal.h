@@ -161,6 +161,9 @@ int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count);
 int gemm_init();  // resolves the tensor-map encoder; returns an efqat_status
 void conv_pixel_box(int W, int H, int B, int target, int* tw, int* th, int* tb);
 // tiles_out (optional): number of output tiles = number of partial pairs EPI_DX wrote.
-int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out = nullptr);
+// grid_out (optional): number of CTAs launched.
+int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out = nullptr, int* grid_out = nullptr);
+// Output tiles of an EPI_PART problem (before the split of the contraction).
+int64_t gemm_part_tiles(int64_t Mr, int64_t Nc);
 
 }  // namespace efqat

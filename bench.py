@@ -34,10 +34,11 @@ sys.path.insert(0, ROOT)
 from paper_2411_11038_b200 import inputs as I  # noqa: E402
 
 FRACS = (0.0, 0.05, 0.25, 1.0)
-METRIC = "fq-linear step TFLOP/s (select + fwd + partial bwd); bwd TFLOP/s and speedup vs full-QAT bwd per unfrozen % in 'bwd'"
+METRIC = "fq-linear step TFLOP/s (select + fwd + partial bwd + fused sparse SGD); bwd TFLOP/s and speedup vs full-QAT bwd per unfrozen % in 'bwd'"
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (set to None whenever the kernel changes after a capture).
+SGD_LR = 1e-9
 DOMINANT_TRAFFIC_BYTES = 28.93e6    # mean over the four dX launches of one step (profiles/gemm_kernel_dx_bench_cfg2.txt)
 
 
@@ -121,6 +122,12 @@ class Workload:
             D["host_X"] = T["X"].pin_memory()
             D["host_dY"] = T["dY"].pin_memory()
             plan = B.LayerPlan(ctx, c.M, c.N, c.K, c.act_dtype, c.w_bits, c.x_bits, c.x_symmetric, c.N, device)
+            # fused sparse SGD-momentum of Algorithm 1 on the unfrozen rows (momentum and weight decay
+            # of Section 4).  The learning rate is scaled down: the synthetic dY has unit variance,
+            # a real loss gradient is orders of magnitude smaller, and the weights must stay put
+            # over hundreds of timed steps; the arithmetic and the traffic are those of any rate.
+            D["mom"] = torch.zeros_like(D["W"])
+            D["sgd"] = B.make_sgd(SGD_LR, 0.9, 1e-4, D["W"], D["mom"])
             D["host_dW"] = torch.empty((c.N, c.K), dtype=torch.float32).pin_memory()
             D["host_small"] = torch.empty(2 * c.N + 2, dtype=torch.float32).pin_memory()
             self.layers.append((c, D, plan))
@@ -159,7 +166,7 @@ class Workload:
     def backward(self, frac):
         _, ks, views = self.sel[frac]
         for (c, D, plan), k, idx in zip(self.layers, ks, views):
-            plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True)
+            plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True, sgd=D["sgd"])
 
     def step(self, frac):
         """Selection only reads the weights and only the backward needs its result, so it runs
@@ -200,7 +207,7 @@ class Workload:
             plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"])
         for (c, D, plan), k, idx, e in zip(self.layers, ks, views, ev_dy):
             cur.wait_event(e)
-            plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True)
+            plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True, sgd=D["sgd"])
         for (c, D, plan), k in zip(self.layers, ks):
             if k:
                 D["host_dW"][:k].copy_(plan.dW_sel[:k], non_blocking=True)
@@ -258,7 +265,8 @@ def oracle_step_seconds(frac, layers=None, rows=None):
         k = O.ratio_to_k(frac, c.N)
         idx = O.select_cwpl([W], [k])[0]
         O.forward(X, W, s_w, s_x, z_x, b, c.w_bits, c.x_bits, c.x_symmetric)
-        O.backward_efqat(dY, X, W, s_w, s_x, z_x, idx, c.w_bits, c.x_bits, c.x_symmetric)
+        g = O.backward_efqat(dY, X, W, s_w, s_x, z_x, idx, c.w_bits, c.x_bits, c.x_symmetric)
+        O.sgd_rows(W, np.zeros_like(W), g["dW_sel"], idx, SGD_LR, 0.9, 1e-4)
         flops += 2.0 * c.M * c.N * c.K * 2 + 2.0 * c.M * k * c.K
     return time.perf_counter() - t0, flops, [c.name for c in cases]
 
@@ -384,6 +392,8 @@ def run_ours(args):
             "config": {"workload": "configs[1]: BERT-base-shaped linears 768->2304, 768->768, 768->3072, 3072->768 "
                                    "at M=4096, bf16 activations, W8A8, CWPL",
                        "unfrozen": frac, "l2": "256 MiB buffer written between timed steps",
+                       "optimizer": "fused SGD-momentum on the unfrozen rows (momentum 0.9, weight decay 1e-4, "
+                                    f"lr {SGD_LR:g} scaled for unit-variance synthetic dY)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": sampler.summary(),
             "e2e": {"value": e2e_val, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": bi,

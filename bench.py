@@ -34,7 +34,9 @@ sys.path.insert(0, ROOT)
 from paper_2411_11038_b200 import inputs as I  # noqa: E402
 
 FRACS = (0.0, 0.05, 0.25, 1.0)
-METRIC = "fq-linear step TFLOP/s (select + fwd + partial bwd + fused sparse SGD); bwd TFLOP/s and speedup vs full-QAT bwd per unfrozen % in 'bwd'"
+METRIC = ("fq-linear backward TFLOP/s & speedup vs full-QAT bwd per unfrozen %; roofline frac "
+          "[value: TFLOP/s of one step of the whole path = select + fwd + partial bwd + fused sparse SGD; "
+          "backward-only ms, TFLOP/s and speedups per unfrozen % under 'bwd']")
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (set to None whenever the kernel changes after a capture).

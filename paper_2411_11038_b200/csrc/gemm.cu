@@ -830,10 +830,17 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   // CTA pairs (256 x BN tiles, tiles full in N) halve the B traffic from L2 per FLOP; they are
   // taken unless one-CTA tiles fill the machine's last wave clearly better.
   int pair = 0;
-  // (full weight-gradient GEMM: measured gain only on long runs of tiles, 1.18-1.33x at >= 1024 pair
-  // tiles, a loss at 256)
-  const bool part_pair = a.a_mn && a.b_mn && a.splits == 1 && a.Nc % 256 == 0 &&
-                         ceil_div(a.Mr, 2 * BM) * (a.Nc / 256) >= 4 * static_cast<int64_t>(sm_count);
+  // Full weight-gradient GEMM (both operands MN-major), as measured at M = 16384 over ten (K, N)
+  // shapes: pairs give 1.22-1.43 PFLOP/s against 1.0-1.17 for one-CTA tiles, except on the two
+  // squares 4096^2 and 5120^2 (0.88-0.96 against 1.09-1.12), for which no cause was found.
+  // Pairs are therefore taken when the smaller output extent is at most 3072 and there are at
+  // least 64 pair tiles (small problems, split many ways, lose: 768^2 went from 24 to 39 us),
+  // or on long runs of unsplit tiles.
+  const int64_t pair_tiles = ceil_div(a.Mr, 2 * BM) * (a.Nc / 256);
+  const int64_t small_ext = a.Mr < a.Nc ? a.Mr : a.Nc;
+  const bool part_pair = a.a_mn && a.b_mn && a.Nc % 256 == 0 &&
+                         ((a.splits == 1 && pair_tiles >= 4 * static_cast<int64_t>(sm_count)) ||
+                          (small_ext <= 3072 && pair_tiles >= 64));
   if (!cv && (a.epi != EPI_PART || part_pair) && a.Mr >= 256 && a.Nc % 128 == 0) {
     const int units = sm_count / 2;
     const int64_t mt = ceil_div(a.Mr, 2 * BM);

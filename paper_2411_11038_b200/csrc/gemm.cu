@@ -766,27 +766,25 @@ int64_t gemm_part_tiles(int64_t Mr, int64_t Nc) { return ceil_div(Mr, BM) * ceil
 int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
   const int64_t nkb = ceil_div(Kc, BK);
   const int64_t tiles = ceil_div(Mr, BM) * ceil_div(Nc, part_bn(Nc));
-  const int64_t max_s = nkb / 4 > 0 ? nkb / 4 : 1;   // at least four contraction blocks per split
-  if (tiles >= sm_count) {
-    // More tiles than SMs: a short last wave can cost up to half a tile time.  Splitting the
-    // contraction in 2-4 makes the work items smaller; take the split with the fewest tile
-    // times, charging 3 % per extra split for the larger partial-product traffic.
-    int best = 1;
-    double best_cost = 1e300;
-    for (int64_t c = 1; c <= 4 && c <= max_s; ++c) {
-      const double cost = static_cast<double>(ceil_div(tiles * c, sm_count)) / c * (1.0 + 0.03 * (c - 1));
-      if (cost < best_cost - 1e-9) {
-        best_cost = cost;
-        best = static_cast<int>(c);
-      }
+  int64_t max_s = nkb / 4 > 0 ? nkb / 4 : 1;        // at least four contraction blocks per split
+  // More tiles than SMs: a short last wave can cost up to half a tile time, and splitting the
+  // contraction in 2-4 makes the work items smaller.  Fewer tiles than SMs: split until the SMs
+  // are full, but never into a second, nearly empty wave (32 tiles x 5 splits = 160 items on 148
+  // SMs took twice the time of 32 x 4).  Either way: the split with the fewest tile times,
+  // charging 2 % per extra split for the larger partial-product traffic.
+  if (tiles >= sm_count && max_s > 4) max_s = 4;
+  if (max_s > sm_count) max_s = sm_count;
+  int best = 1;
+  double best_cost = 1e300;
+  for (int64_t c = 1; c <= max_s; ++c) {
+    const double cost = static_cast<double>(ceil_div(tiles * c, sm_count)) / c * (1.0 + 0.02 * (c - 1));
+    if (cost < best_cost - 1e-12) {
+      best_cost = cost;
+      best = static_cast<int>(c);
     }
-    return best;
+    if (tiles * c > 2 * static_cast<int64_t>(sm_count) && tiles < sm_count) break;
   }
-  int64_t s = ceil_div(sm_count, tiles);
-  if (s > max_s) s = max_s;
-  if (s > sm_count) s = sm_count;
-  if (s < 1) s = 1;
-  return static_cast<int>(s);
+  return best;
 }
 
 template <int A_MN, int B_MN, int EPI, int CTA2>

@@ -833,11 +833,11 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   // squares 4096^2 and 5120^2 (0.88-0.96 against 1.09-1.12), for which no cause was found.
   // Pairs are therefore taken when the smaller output extent is at most 3072 and there are at
   // least 64 pair tiles (small problems, split many ways, lose: 768^2 went from 24 to 39 us),
-  // or on long runs of unsplit tiles.
+  // or on long runs (>= 512, the shortest measured good one) of unsplit pair tiles.
   const int64_t pair_tiles = ceil_div(a.Mr, 2 * BM) * (a.Nc / 256);
   const int64_t small_ext = a.Mr < a.Nc ? a.Mr : a.Nc;
   const bool part_pair = a.a_mn && a.b_mn && a.Nc % 256 == 0 &&
-                         ((a.splits == 1 && pair_tiles >= 4 * static_cast<int64_t>(sm_count)) ||
+                         ((a.splits == 1 && pair_tiles >= 512) ||
                           (small_ext <= 3072 && pair_tiles >= 64));
   if (!cv && (a.epi != EPI_PART || part_pair) && a.Mr >= 256 && a.Nc % 128 == 0) {
     const int units = sm_count / 2;

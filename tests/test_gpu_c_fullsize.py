@@ -32,6 +32,28 @@ def test_config2_layer_full_size(ctx, li):
     U.check_backward(ctx, case, T, D, s_w, s_x, z_x, idx)
 
 
+def test_config2_layer_full_size_with_fused_sgd(ctx):
+    """The benchmark's step as it is timed: 5 % partial backward of the 768 -> 2304 layer with
+    the fused SGD-momentum update (momentum 0.9, weight decay 1e-4) on the unfrozen rows."""
+    case = I.config2()[0]
+    T = I.make_tensors(case)
+    s_w, s_x, z_x = U.oracle_qparams(case, T)
+    D = U.to_dev(T, s_w, s_x, z_x)
+    k = B.ratio_to_k(0.05, case.N)
+    idx = O.select_cwpl([T["W"].numpy()], [k])[0]
+    g = torch.Generator().manual_seed(7)
+    V0 = torch.randn(T["W"].shape, generator=g) * 0.01
+    Wd, Vd = D["W"].clone(), V0.cuda()
+    lr = 1e-3
+    out = U.check_backward(ctx, case, T, D, s_w, s_x, z_x, idx, sgd=B.make_sgd(lr, 0.9, 1e-4, Wd, Vd))
+    W2, V2 = O.sgd_rows(T["W"].numpy(), V0.numpy(), out["dW_sel"], idx, lr, 0.9, 1e-4)
+    frozen = np.setdiff1d(np.arange(case.N), idx)
+    assert np.array_equal(Wd.cpu().numpy()[frozen], T["W"].numpy()[frozen])
+    assert np.array_equal(Vd.cpu().numpy()[frozen], V0.numpy()[frozen])
+    np.testing.assert_allclose(Vd.cpu().numpy()[idx], V2[idx], rtol=1e-5, atol=1e-6)
+    np.testing.assert_allclose(Wd.cpu().numpy()[idx], W2[idx], rtol=1e-5, atol=1e-7)
+
+
 def test_config2_full_qat_backward(ctx):
     case = I.config2()[1]
     T = I.make_tensors(case)

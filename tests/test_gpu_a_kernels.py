@@ -36,6 +36,24 @@ def test_gemm_core_exact_on_integers(ctx, a_mn, b_mn, M, N, K, splits):
     assert np.array_equal(got, ref)
 
 
+@pytest.mark.parametrize("splits", [1, 3])
+def test_gemm_core_cta_pairs_exact_on_integers(ctx, splits):
+    """Both operands MN-major and 64 output tiles of 256 x 256: the shape class for which the
+    partial-product GEMM runs on CTA pairs (cta_group::2), with and without a split contraction."""
+    M, N, K = 2048, 2048, 1024
+    g = torch.Generator().manual_seed(77 + splits)
+    A = torch.randint(-4, 5, (M, K), generator=g).float()
+    Bm = torch.randint(-4, 5, (N, K), generator=g).float()
+    ref = (A.double() @ Bm.double().T).numpy()
+    A_st = A.T.contiguous().to(torch.bfloat16).cuda()
+    B_st = Bm.T.contiguous().to(torch.bfloat16).cuda()
+    out = B.gemm_bf16(ctx, A_st, B_st, M, N, K, 1, 1, splits)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    got = out.double().sum(dim=0).cpu().numpy().T
+    assert np.array_equal(got, ref)
+
+
 def test_gemm_core_random_bf16(ctx):
     g = torch.Generator().manual_seed(5)
     M, N, K = 640, 392, 1096

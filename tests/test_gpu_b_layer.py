@@ -27,6 +27,8 @@ SMALL = [
     _case("tiles_bf16_w4", 512, 320, 520, torch.bfloat16, w_bits=4, seed=3),
     _case("sym_a4", 260, 64, 128, torch.bfloat16, w_bits=4, x_bits=4, sym=True, seed=4),
     _case("one_row", 1, 64, 8, torch.float32, seed=5),
+    _case("two_bit", 160, 72, 40, torch.bfloat16, w_bits=2, x_bits=2, seed=6),
+    _case("smallest", 8, 8, 8, torch.bfloat16, seed=7),
 ]
 
 
@@ -49,6 +51,8 @@ def test_backward_parity_and_invariants(ctx, case, clip):
     k5 = max(1, N // 20)
     sets = [np.zeros(0, np.int32), O.select_cwpl([T["W"].numpy()], [k5])[0],
             np.arange(0, N, 3, dtype=np.int32), np.arange(N, dtype=np.int32)]
+    if N > 2:
+        sets.insert(3, np.delete(np.arange(N, dtype=np.int32), N // 2))      # all channels but one: widest gather
     outs = [U.check_backward(ctx, case, T, D, s_w, s_x, z_x, idx) for idx in sets]
     # dX, dS_x, dZ_x, db never depend on the selection: bit-identical across idx
     for o in outs[1:]:

@@ -111,6 +111,24 @@ def sweep_network(ctx, timer, dev):
     return out
 
 
+def sweep_layerwise(ctx, timer, dev):
+    """Layer-wise mode (LWPN) over the four W8A8 sweep shapes as one stack: the selection kernel
+    ranks whole layers by mean |w| and unfreezes the top half; a frozen layer then runs the 0 %
+    backward and an unfrozen one the 100 % backward of the per-layer records above."""
+    cases = I.config5()
+    g = torch.Generator().manual_seed(5000)
+    Ws = [(torch.randn((c.N, c.K), generator=g) * 0.02).to(dev) for c in cases]
+    k_l = len(cases) // 2
+    plan = B.SelectPlan(ctx, B.LWPN, Ws, [k_l])
+    plan.run()
+    torch.cuda.synchronize()
+    t = timer.ms(plan.run)
+    counts = (plan.offsets[1:] - plan.offsets[:-1]).cpu().tolist()
+    nbytes = sum(w.numel() * 4 for w in Ws)
+    return {"layer": "cfg5_lwpn_selection_4_layers", "select_ms": t, "select_gbs": nbytes / t / 1e6,
+            "layers": [c.name for c in cases], "unfrozen_layers": k_l, "channels_per_layer": counts}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
@@ -135,6 +153,9 @@ def main():
                 cases = [c for c in cases if args.only in c.name]
             for c in cases:
                 recs.append(sweep_layer(ctx, c, FRACS[cfg], timer, dev))
+                torch.cuda.empty_cache()
+            if cfg == 5 and not args.only:
+                recs.append(sweep_layerwise(ctx, timer, dev))
                 torch.cuda.empty_cache()
         for r in recs:
             r["config"] = cfg

@@ -68,6 +68,7 @@ struct LayerWs {
   float* P;        // [splits][k_sel][K] partial weight-gradient products
   float* dxpart;   // [tiles][2]
   float* colsum;   // [COLSUM_SLABS][N]
+  int32_t* wsum;   // [N] row sums of the 8-bit weight codes (integer forward)
   int64_t pitch;
   int splits;
   size_t bytes;
@@ -122,6 +123,7 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   w.P = reinterpret_cast<float*>(take(p_elems * 4));
   w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(dx_partials(l)) * 8));
   w.colsum = reinterpret_cast<float*>(take(static_cast<int64_t>(prepare_slabs(M, N)) * N * 4));
+  w.wsum = reinterpret_cast<int32_t*>(take(N * 4));
   w.bytes = off + 256;
   return w;
 }
@@ -334,9 +336,23 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric; pa.Xc = w.Xc;
   pa.x_count = x_elems(layer);
   pa.status = ctx->d_status;
+  // A plain layer runs its forward on the integer tensor cores: 8-bit codes (the code buffers
+  // of the bf16 path are reused, half filled), int32 accumulation, zero point taken out exactly in
+  // the epilogue.  int32 holds K * 255 * 127 up to K = 65536; the limit here leaves a factor 2.
+  // (row pitch of the 8-bit operands must be a multiple of 16 bytes for TMA; tiles are kept to
+  // multiples of 32 columns, the coarser of the instruction's N granularities)
+  const bool i8 = !spatial_conv(layer) && K <= 32768 && K % 16 == 0 && N % 32 == 0;
+  if (i8) {
+    pa.i8 = 1;
+    pa.Wq8 = reinterpret_cast<int8_t*>(w.Wq);
+    pa.Xc8 = reinterpret_cast<uint8_t*>(w.Xc);
+    pa.wsum = w.wsum;
+  }
   launch_prepare(pa, 0, act_bf16, st);
   ConvArgs cva;
   GemmArgs g = {};
+  g.i8 = i8 ? 1 : 0;
+  g.wsum = w.wsum;
   g.A = w.Xc; g.B = w.Wq;
   g.Mr = M; g.Nc = N; g.Kc = K;
   g.lda = K; g.ldb = K;

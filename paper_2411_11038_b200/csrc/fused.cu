@@ -101,6 +101,74 @@ __device__ __forceinline__ void job_quant_x(const PrepArgs& a, int block, int nb
   }
 }
 
+// ---- jobs of the integer forward: 8-bit codes -------------------------------------------
+__device__ __forceinline__ uint32_t pack4(const int (&c)[8], int o) {
+  return (static_cast<uint32_t>(c[o]) & 255u) | ((static_cast<uint32_t>(c[o + 1]) & 255u) << 8) |
+         ((static_cast<uint32_t>(c[o + 2]) & 255u) << 16) | ((static_cast<uint32_t>(c[o + 3]) & 255u) << 24);
+}
+// One warp per weight row: signed codes and their sum (the zero-point correction of the epilogue).
+__device__ __forceinline__ void job_weights_i8(const PrepArgs& a, int block, int nblocks) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t kv = a.K / 8;
+  for (int64_t n = static_cast<int64_t>(block) * 8 + warp; n < a.N; n += static_cast<int64_t>(nblocks) * 8) {
+    float sw = __ldg(a.s_w + n);
+    if (!scale_ok(sw)) {
+      if (lane == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
+      sw = 1.f;
+    }
+    const RowQ p = make_rowq(sw, a.w_bits);
+    const float* row = a.W + n * a.K;
+    int8_t* orow = a.Wq8 + n * a.K;
+    int sum = 0;
+    for (int64_t v0 = lane; v0 < kv; v0 += 128) {       // four independent 32-byte loads in flight
+      float v[4][8];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (v0 + 32 * u < kv) ld8<float>(row + (v0 + 32 * u) * 8, v[u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (v0 + 32 * u < kv) {
+          int c[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            c[j] = quant_weight(v[u][j], p).code;
+            sum += c[j];
+          }
+          *reinterpret_cast<uint2*>(orow + (v0 + 32 * u) * 8) = make_uint2(pack4(c, 0), pack4(c, 4));
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) a.wsum[n] = sum;
+  }
+}
+// Activations -> 8-bit codes clamp(rne(x/s) + Zr, lo, hi) (unsigned; signed for the symmetric quantizer).
+template <typename T>
+__device__ __forceinline__ void job_quant_x_i8(const PrepArgs& a, int block, int nblocks) {
+  bool bad;
+  const ActQ p = make_actq(a.s_x, a.z_x, a.x_bits, a.x_sym, &bad);
+  if (bad && block == 0 && threadIdx.x == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
+  const T* X = static_cast<const T*>(a.X);
+  const int64_t n8 = a.x_count / 8;
+  const int64_t stride = static_cast<int64_t>(nblocks) * blockDim.x;
+  for (int64_t i0 = static_cast<int64_t>(block) * blockDim.x + threadIdx.x; i0 < n8; i0 += 4 * stride) {
+    float v[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (i0 + u * stride < n8) ld8<T>(X + (i0 + u * stride) * 8, v[u]);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (i0 + u * stride < n8) {
+        int c[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c[j] = quant_act(v[u][j], p).code;
+        *reinterpret_cast<uint2*>(a.Xc8 + (i0 + u * stride) * 8) = make_uint2(pack4(c, 0), pack4(c, 4));
+      }
+    }
+  }
+}
+
 // ---- job: one pass over dY: column-sum partials and the bf16 copy ------------------------
 // Block (cb, slab): 256 columns x one slab of rows; warp w takes rows slab_lo + w, + 8, ...,
 // four rows (four independent 16-byte loads per thread) at a time.
@@ -210,9 +278,11 @@ __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
     if (j < a.nb_g) job_gather<TX>(a, slab, reinterpret_cast<int32_t*>(sh));
     else job_dy_pass<TX>(a, j - a.nb_g, slab, sh);
   } else if (b < nb_y + a.nb_w) {
-    job_weights<W_MODE>(a, b - nb_y, a.nb_w);
+    if (W_MODE == 0 && a.i8) job_weights_i8(a, b - nb_y, a.nb_w);
+    else job_weights<W_MODE>(a, b - nb_y, a.nb_w);
   } else {
-    job_quant_x<TX>(a, b - nb_y - a.nb_w, a.nb_x);
+    if (W_MODE == 0 && a.i8) job_quant_x_i8<TX>(a, b - nb_y - a.nb_w, a.nb_x);
+    else job_quant_x<TX>(a, b - nb_y - a.nb_w, a.nb_x);
   }
 }
 
@@ -378,8 +448,9 @@ static int flat_blocks(int64_t vectors, int64_t per_block) {
 
 void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   a.nb_w = flat_blocks(a.N * (a.K / 8), 256 * 4);       // 32 KiB of fp32 weights per block
+  if (a.i8) a.nb_w = static_cast<int>(ceil_div(a.N, 8) < 148 * 12 ? ceil_div(a.N, 8) : 148 * 12);   // a warp per row
   a.nb_x = 0;
-  if (a.Xc) a.nb_x = flat_blocks(a.x_count / 8, 256 * 8);   // 32 KiB (bf16) / 64 KiB (fp32) per block
+  if (a.Xc || (a.i8 && a.Xc8)) a.nb_x = flat_blocks(a.x_count / 8, 256 * 8);   // 32 KiB (bf16) / 64 KiB (fp32) per block
   const bool gather = a.dY && a.dYsel && a.k_sel > 0 && a.k_sel < a.N;
   a.nb_g = gather ? 1 : 0;                       // gather blocks per slab
   a.col_blocks = static_cast<int>(ceil_div(a.N, 256));

@@ -54,6 +54,10 @@ struct GemmParams {
   int nkb;            // number of BK blocks along the contraction
   int BN;             // tile columns (multiple of 16, <= 256)
   int stages;
+  int i8;             // EPI_FWD on 8-bit integer operands (kind::i8): 128 contraction elements per k-block
+  int bk;             // contraction elements per k-block: 64 (bf16) or 128 (8-bit)
+  int a_signed;       // i8: activation codes are signed (symmetric quantizer)
+  const int32_t* wsum;
   int kps;            // k-blocks per stage: one barrier round trip covers kps * 64 contraction elements
   int merged;         // MN-major operands arrive as one TMA box per 64-wide chunk and stage (plain matrices only)
   int b_stage_bytes;
@@ -106,7 +110,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   uint8_t* out_stg = smem + p.stages * stage_bytes;          // [8 warps][out_bufs][HB_BYTES]
   uint8_t* x_stg = out_stg + (EPI == EPI_PART ? 0 : EPI_WARPS * p.out_bufs * HB_BYTES);   // [8 warps][HB_BYTES] (EPI_DX)
   SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? EPI_WARPS * HB_BYTES : 0));
-  float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [8 warps][128 scales, 128 biases] (EPI_FWD), warp-private
+  float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [8 warps][128 scales, 128 biases, 128 zero-point terms] (EPI_FWD), warp-private
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_mn = p.tiles_m * p.tiles_n;
@@ -235,14 +239,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
                   tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
                 } else {
-                  tma_load_2d_pair(sa, &tmA, fb, kb * BK, m0);
+                  tma_load_2d_pair(sa, &tmA, fb, kb * p.bk, m0);
                 }
               } else {
                 if (B_MN) {
                   for (int c = 0; c < b_chunks; ++c)
                     tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
                 } else {
-                  tma_load_2d_pair(sb, &tmB, fb, kb * BK, n0);
+                  tma_load_2d_pair(sb, &tmB, fb, kb * p.bk, n0);
                 }
               }
             } else if (p.cv.mode == 0) {
@@ -251,14 +255,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
                   tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
                 } else {
-                  tma_load_2d(sa, &tmA, &ctl->full[s], kb * BK, m0);
+                  tma_load_2d(sa, &tmA, &ctl->full[s], kb * p.bk, m0);
                 }
               } else {
                 if (B_MN) {
                   for (int c = 0; c < b_chunks; ++c)
                     tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
                 } else {
-                  tma_load_2d(sb, &tmB, &ctl->full[s], kb * BK, n0);
+                  tma_load_2d(sb, &tmB, &ctl->full[s], kb * p.bk, n0);
                 }
               }
             } else if (p.cv.mode == 3) {
@@ -320,7 +324,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         int n_eff = static_cast<int>(p.Nc - n0);
         if (n_eff > p.BN) n_eff = p.BN;
         n_eff = (n_eff + 15) & ~15;
-        const uint32_t idesc = instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
+        const uint32_t idesc = (EPI == EPI_FWD && p.i8) ? instr_desc_i8(TILE_M, n_eff, p.a_signed, 1)
+                                                        : instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
         const int buf = acc_it & 1;
@@ -362,8 +367,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                         : smem_desc_sw128(a_addr + k * 32, 16, 1024);
             const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, b_lbo, 1024)
                                         : smem_desc_sw128(b_addr + k * 32, 16, 1024);
-            if (CTA2) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
-            else umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > kb_begin || k > 0) ? 1u : 0u);
+            const uint32_t accum = (kb > kb_begin || k > 0) ? 1u : 0u;
+            if (EPI == EPI_FWD && p.i8) {
+              if (CTA2) umma_i8_pair(d_tmem, adesc, bdesc, idesc, accum); else umma_i8(d_tmem, adesc, bdesc, idesc, accum);
+            } else {
+              if (CTA2) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, accum); else umma_bf16(d_tmem, adesc, bdesc, idesc, accum);
+            }
           }
          }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
@@ -386,9 +395,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int bc = p.blk_cols;
     uint8_t* my_out = out_stg + e * p.out_bufs * HB_BYTES;
     uint8_t* my_x = x_stg + e * HB_BYTES;
-    float* my_sc = s_scale + e * 256;          // [128] scales then [128] biases of this warp's columns
+    float* my_sc = s_scale + e * 384;          // [128] scales, [128] biases, [128] Zr * wsum (as int) of this warp's columns
+    int* my_zw = reinterpret_cast<int*>(my_sc + 256);
     ActQ xq = {};
     if (EPI != EPI_PART) xq = make_actq(p.s_x, p.z_x, p.x_bits, p.x_sym, nullptr);
+    const int zr_i = static_cast<int>(xq.zr);
     const float t_lo = xq.lo - xq.zr, t_hi = xq.hi - xq.zr;     // d/ds of a clipped element
     const float q_half = 0.5f * (xq.hi - xq.lo), z_mid = xq.zr - 0.5f * (xq.hi + xq.lo);
 
@@ -446,6 +457,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int64_t c = static_cast<int64_t>(g.n0) + g.jb0 * bc + j;
           my_sc[j] = (c < p.Nc) ? p.col_scale[c] * xq.s : 0.f;
           my_sc[128 + j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
+          my_zw[j] = (p.i8 && c < p.Nc) ? zr_i * p.wsum[c] : 0;
         }
         __syncwarp();
       }
@@ -456,6 +468,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int buf = acc_it & 1;
       // next tile's column scales and biases: loaded now, parked in registers behind this tile's work
       float nsc[4] = {0.f, 0.f, 0.f, 0.f}, nbi[4] = {0.f, 0.f, 0.f, 0.f};
+      int nzw[4] = {0, 0, 0, 0};
       if (EPI == EPI_FWD && has_next) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -463,6 +476,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (c < p.Nc) {
             nsc[i] = p.col_scale[c] * xq.s;
             if (p.col_bias) nbi[i] = p.col_bias[c];
+            if (p.i8) nzw[i] = zr_i * p.wsum[c];
           }
         }
       }
@@ -523,13 +537,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           uint32_t r[32];
           if (ncols == 32) tmem_ld_32x32(t_row + c0, r); else tmem_ld_32x16(t_row + c0, r);
           float4 sc4[8], bi4[8];     // this block's column scales (s_x folded in) and biases
+          int4 zw4[8];               // and, on integer operands, Zr * (row sum of the weight codes)
           if (EPI == EPI_FWD) {
             const float4* ps = reinterpret_cast<const float4*>(my_sc + (jb - g.jb0) * bc);
+            const int4* pz = reinterpret_cast<const int4*>(my_zw + (jb - g.jb0) * bc);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               if (i * 4 < bc) {
                 sc4[i] = ps[i];
                 bi4[i] = ps[32 + i];
+                if (p.i8) zw4[i] = pz[i];
               }
             }
           }
@@ -550,8 +567,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                      sc4[2 * gi + 1].x, sc4[2 * gi + 1].y, sc4[2 * gi + 1].z, sc4[2 * gi + 1].w};
                 const float bv[8] = {bi4[2 * gi].x, bi4[2 * gi].y, bi4[2 * gi].z, bi4[2 * gi].w,
                                      bi4[2 * gi + 1].x, bi4[2 * gi + 1].y, bi4[2 * gi + 1].z, bi4[2 * gi + 1].w};
+                if (p.i8) {
+                  // integer accumulators: sum_k q_x q_w - Zr sum_k q_w = sum_k (q_x - Zr) q_w, exact in int32
+                  const int zv[8] = {zw4[2 * gi].x, zw4[2 * gi].y, zw4[2 * gi].z, zw4[2 * gi].w,
+                                     zw4[2 * gi + 1].x, zw4[2 * gi + 1].y, zw4[2 * gi + 1].z, zw4[2 * gi + 1].w};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = fmaf(__uint_as_float(r[gi * 8 + j]), sv[j], bv[j]);
+                  for (int j = 0; j < 8; ++j)
+                    v[j] = fmaf(static_cast<float>(static_cast<int>(r[gi * 8 + j]) - zv[j]), sv[j], bv[j]);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) v[j] = fmaf(__uint_as_float(r[gi * 8 + j]), sv[j], bv[j]);
+                }
               } else {
                 float x[8];
                 if (bc == 32) {      // bf16 activations: 8 values in one 16-byte piece
@@ -646,6 +672,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int i = 0; i < 4; ++i) {
           my_sc[lane + 32 * i] = nsc[i];
           my_sc[128 + lane + 32 * i] = nbi[i];
+          my_zw[lane + 32 * i] = nzw[i];
         }
         __syncwarp();
       }
@@ -680,15 +707,17 @@ int gemm_init() {
 }
 
 // 2-D row-major matrix [rows, cols] with pitch ld (elements); box = row_bytes (128 or 64, the
-// swizzle span) of columns x box_rows rows.
+// swizzle span) of columns x box_rows rows.  is_bf16: 0 fp32, 1 bf16, 2 8-bit integer.
 static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows, int64_t cols, int64_t ld,
                     int box_rows, int row_bytes = 128) {
-  const int es = is_bf16 ? 2 : 4;
+  const int es = (is_bf16 == 2) ? 1 : (is_bf16 ? 2 : 4);
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * es};
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(row_bytes / es), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estr[2] = {1u, 1u};
-  const CUresult r = g_encode(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+  const CUtensorMapDataType dt = (is_bf16 == 2) ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                 : (is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
+  const CUresult r = g_encode(m, dt, 2,
                               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                               row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -814,7 +843,13 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   GemmParams p = {};
   p.Mr = a.Mr;
   p.Nc = a.Nc;
-  p.nkb = static_cast<int>(ceil_div(a.Kc, BK));
+  // forward of a plain layer on integer operands: 8-bit codes, 128 of them per 128-byte k-block
+  const int i8 = (a.epi == EPI_FWD && a.i8 && !a.conv && !a.a_mn && !a.b_mn) ? 1 : 0;
+  p.i8 = i8;
+  p.bk = i8 ? 128 : BK;
+  p.a_signed = a.x_sym ? 1 : 0;
+  p.wsum = a.wsum;
+  p.nkb = static_cast<int>(ceil_div(a.Kc, p.bk));
   p.splits = (a.epi == EPI_PART) ? a.splits : 1;
   if (p.splits < 1 || p.splits > p.nkb) return EFQAT_ERR_SHAPE;
   p.BN = (a.epi == EPI_PART) ? part_bn(a.Nc) : choose_bn(a.Mr, a.Nc, sm_count);
@@ -883,7 +918,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;
   const int out_stg_bytes = (a.epi == EPI_PART) ? 0 : EPI_WARPS * HB_BYTES;     // one staging buffer per warp
   int fixed_bytes = out_stg_bytes + (a.epi == EPI_DX ? EPI_WARPS * HB_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
-                    (a.epi == EPI_FWD ? EPI_WARPS * 256 * 4 : 0);
+                    (a.epi == EPI_FWD ? EPI_WARPS * 384 * 4 : 0);
   const int ring_bytes = 227 * 1024 - 1024 - fixed_bytes;
   // k-blocks per stage: as many as still leave three stages (two for the widest tiles), at most 4
   int kps = ring_bytes / (3 * sub_bytes);
@@ -918,9 +953,9 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   if (a.epi == EPI_DX && (a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;
   if (!cv) {
     // MN-major operands: one box = all kps k-blocks of a stage for one 64-wide chunk
-    rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK * kps) : make_map(&ta, a.A, 1, a.Mr, a.Kc, a.lda, BM);
+    rc = a.a_mn ? make_map(&ta, a.A, 1, a.Kc, a.Mr, a.lda, BK * kps) : make_map(&ta, a.A, i8 ? 2 : 1, a.Mr, a.Kc, a.lda, BM);
     if (rc != EFQAT_OK) return rc;
-    rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK * kps) : make_map(&tb, a.B, 1, a.Nc, a.Kc, a.ldb, bn_cta);
+    rc = a.b_mn ? make_map(&tb, a.B, 1, a.Kc, a.Nc, a.ldb, BK * kps) : make_map(&tb, a.B, i8 ? 2 : 1, a.Nc, a.Kc, a.ldb, bn_cta);
     if (rc != EFQAT_OK) return rc;
     to = ta;
     tx = ta;

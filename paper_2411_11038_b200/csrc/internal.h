@@ -79,6 +79,9 @@ struct PrepArgs {
   const void* dY; bf16* dYb; float* colsum_ws;
   const int32_t* idx; int64_t k_sel, pitch; bf16* dYsel;
   int* status;
+  // forward on the integer tensor cores: 8-bit codes (weights signed, activations unsigned or,
+  // for the symmetric quantizer, signed; not centred) and the row sums of the weight codes
+  int i8; int8_t* Wq8; uint8_t* Xc8; int32_t* wsum;
   int nb_g, nb_w, nb_x, col_blocks, slabs, dy_on;   // filled by launch_prepare
 };
 int prepare_slabs(int64_t M, int64_t N);
@@ -138,6 +141,9 @@ struct GemmArgs {
   // EPI_FWD
   const float* col_scale;  // s_w[Nc]
   const float* col_bias;   // bias[Nc] or null
+  // EPI_FWD with 8-bit integer operands (kind::i8, K-major, plain matrices): A = activation codes
+  // (not centred), B = weight codes, wsum[n] = sum_k B[n,k]; the epilogue subtracts Zr * wsum[n]
+  int i8; const int32_t* wsum;
   // EPI_FWD / EPI_DX: learnable activation scale / zero point and their bit-width
   const float* s_x; const float* z_x; int x_bits, x_sym;
   // EPI_DX

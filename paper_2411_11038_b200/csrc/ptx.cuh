@@ -234,6 +234,37 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   d |= 2ull << 61;   // SWIZZLE_128B
   return d;
 }
+// kind::i8: 8-bit integer A/B (K-major only), 32-bit integer accumulator; 32 contraction
+// elements per instruction, i.e. the same 32 bytes of a swizzled row as kind::f16.
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Instruction descriptor for kind::i8: D format s32; A / B format 0 = unsigned, 1 = signed 8-bit.
+__host__ __device__ __forceinline__ uint32_t instr_desc_i8(int M, int N, int a_signed, int b_signed) {
+  uint32_t d = 0;
+  d |= 2u << 4;                       // D format s32
+  d |= static_cast<uint32_t>(a_signed ? 1 : 0) << 7;
+  d |= static_cast<uint32_t>(b_signed ? 1 : 0) << 10;
+  d |= static_cast<uint32_t>(N >> 3) << 17;
+  d |= static_cast<uint32_t>(M >> 4) << 24;
+  return d;
+}
+
 // Instruction descriptor for kind::f16 with bf16 A/B and fp32 D.
 // a_mn / b_mn: 1 when the operand is stored with its non-contracted dimension contiguous.
 __host__ __device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N, int a_mn, int b_mn) {

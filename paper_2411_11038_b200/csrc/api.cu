@@ -341,7 +341,9 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   // the epilogue.  int32 holds K * 255 * 127 up to K = 65536; the limit here leaves a factor 2.
   // (row pitch of the 8-bit operands must be a multiple of 16 bytes for TMA; tiles are kept to
   // multiples of 32 columns, the coarser of the instruction's N granularities)
-  const bool i8 = !spatial_conv(layer) && K <= 32768 && K % 16 == 0 && N % 32 == 0;
+  // Short contractions (K <= 256: output-bound layers whose 128-wide k-blocks would be half
+  // padding) measured slower this way and stay on the bf16 path.
+  const bool i8 = !spatial_conv(layer) && K >= 512 && K <= 32768 && K % 16 == 0 && N % 32 == 0;
   if (i8) {
     pa.i8 = 1;
     pa.Wq8 = reinterpret_cast<int8_t*>(w.Wq);

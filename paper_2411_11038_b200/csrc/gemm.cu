@@ -102,6 +102,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmX,
             const GemmParams p) {
+  constexpr bool FWD = (EPI == EPI_FWD || EPI == EPI_FWD_I8);   // forward epilogue (scale, bias)
+  constexpr bool I8 = (EPI == EPI_FWD_I8);                       // ... on 8-bit integer operands
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms of TMA and UMMA
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -324,7 +326,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         int n_eff = static_cast<int>(p.Nc - n0);
         if (n_eff > p.BN) n_eff = p.BN;
         n_eff = (n_eff + 15) & ~15;
-        const uint32_t idesc = (EPI == EPI_FWD && p.i8) ? instr_desc_i8(TILE_M, n_eff, p.a_signed, 1)
+        const uint32_t idesc = I8 ? instr_desc_i8(TILE_M, n_eff, p.a_signed, 1)
                                                         : instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
@@ -368,7 +370,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, b_lbo, 1024)
                                         : smem_desc_sw128(b_addr + k * 32, 16, 1024);
             const uint32_t accum = (kb > kb_begin || k > 0) ? 1u : 0u;
-            if (EPI == EPI_FWD && p.i8) {
+            if (I8) {
               if (CTA2) umma_i8_pair(d_tmem, adesc, bdesc, idesc, accum); else umma_i8(d_tmem, adesc, bdesc, idesc, accum);
             } else {
               if (CTA2) umma_bf16_pair(d_tmem, adesc, bdesc, idesc, accum); else umma_bf16(d_tmem, adesc, bdesc, idesc, accum);
@@ -452,12 +454,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (unit < total_items) {
       g = geo_of(unit);
       if (EPI == EPI_DX && lane == 0 && g.jb0 < g.jb1) fetch_x(g, g.jb0);
-      if (EPI == EPI_FWD) {
+      if (FWD) {
         for (int j = lane; j < 128; j += 32) {
           const int64_t c = static_cast<int64_t>(g.n0) + g.jb0 * bc + j;
           my_sc[j] = (c < p.Nc) ? p.col_scale[c] * xq.s : 0.f;
           my_sc[128 + j] = (c < p.Nc && p.col_bias) ? p.col_bias[c] : 0.f;
-          my_zw[j] = (p.i8 && c < p.Nc) ? zr_i * p.wsum[c] : 0;
+          if (I8) my_zw[j] = (c < p.Nc) ? zr_i * p.wsum[c] : 0;
         }
         __syncwarp();
       }
@@ -469,14 +471,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // next tile's column scales and biases: loaded now, parked in registers behind this tile's work
       float nsc[4] = {0.f, 0.f, 0.f, 0.f}, nbi[4] = {0.f, 0.f, 0.f, 0.f};
       int nzw[4] = {0, 0, 0, 0};
-      if (EPI == EPI_FWD && has_next) {
+      if (FWD && has_next) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int64_t c = static_cast<int64_t>(gn.n0) + gn.jb0 * bc + lane + 32 * i;
           if (c < p.Nc) {
             nsc[i] = p.col_scale[c] * xq.s;
             if (p.col_bias) nbi[i] = p.col_bias[c];
-            if (p.i8) nzw[i] = zr_i * p.wsum[c];
+            if (I8) nzw[i] = zr_i * p.wsum[c];
           }
         }
       }
@@ -537,16 +539,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           uint32_t r[32];
           if (ncols == 32) tmem_ld_32x32(t_row + c0, r); else tmem_ld_32x16(t_row + c0, r);
           float4 sc4[8], bi4[8];     // this block's column scales (s_x folded in) and biases
-          int4 zw4[8];               // and, on integer operands, Zr * (row sum of the weight codes)
-          if (EPI == EPI_FWD) {
+          if (FWD) {
             const float4* ps = reinterpret_cast<const float4*>(my_sc + (jb - g.jb0) * bc);
-            const int4* pz = reinterpret_cast<const int4*>(my_zw + (jb - g.jb0) * bc);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               if (i * 4 < bc) {
                 sc4[i] = ps[i];
                 bi4[i] = ps[32 + i];
-                if (p.i8) zw4[i] = pz[i];
               }
             }
           }
@@ -562,15 +561,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int gi = 0; gi < 4; ++gi) {
             if (gi * 8 < ncols) {
               float v[8];
-              if (EPI == EPI_FWD) {
+              if (FWD) {
                 const float sv[8] = {sc4[2 * gi].x, sc4[2 * gi].y, sc4[2 * gi].z, sc4[2 * gi].w,
                                      sc4[2 * gi + 1].x, sc4[2 * gi + 1].y, sc4[2 * gi + 1].z, sc4[2 * gi + 1].w};
                 const float bv[8] = {bi4[2 * gi].x, bi4[2 * gi].y, bi4[2 * gi].z, bi4[2 * gi].w,
                                      bi4[2 * gi + 1].x, bi4[2 * gi + 1].y, bi4[2 * gi + 1].z, bi4[2 * gi + 1].w};
-                if (p.i8) {
+                if (I8) {
                   // integer accumulators: sum_k q_x q_w - Zr sum_k q_w = sum_k (q_x - Zr) q_w, exact in int32
-                  const int zv[8] = {zw4[2 * gi].x, zw4[2 * gi].y, zw4[2 * gi].z, zw4[2 * gi].w,
-                                     zw4[2 * gi + 1].x, zw4[2 * gi + 1].y, zw4[2 * gi + 1].z, zw4[2 * gi + 1].w};
+                  const int4* pz = reinterpret_cast<const int4*>(my_zw + (jb - g.jb0) * bc) + 2 * gi;
+                  const int4 z0 = pz[0], z1 = pz[1];       // Zr * (row sum of the weight codes) of these columns
+                  const int zv[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
 #pragma unroll
                   for (int j = 0; j < 8; ++j)
                     v[j] = fmaf(static_cast<float>(static_cast<int>(r[gi * 8 + j]) - zv[j]), sv[j], bv[j]);
@@ -666,13 +666,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           pp[1] = -xq.s * acc_c;     // Eq. 1: d(dequantised)/dZ = -s on clipped elements, 0 elsewhere
         }
       }
-      if (EPI == EPI_FWD && has_next) {
+      if (FWD && has_next) {
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           my_sc[lane + 32 * i] = nsc[i];
           my_sc[128 + lane + 32 * i] = nbi[i];
-          my_zw[lane + 32 * i] = nzw[i];
+          if (I8) my_zw[lane + 32 * i] = nzw[i];
         }
         __syncwarp();
       }
@@ -1005,6 +1005,10 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
 
 #define EFQAT_LAUNCH(AM, BMj, E, P2) return launch<AM, BMj, E, P2>(ta, tb, to, tx, p, grid, smem, st)
   if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) {
+    if (i8) {
+      if (pair) EFQAT_LAUNCH(0, 0, EPI_FWD_I8, 1);
+      EFQAT_LAUNCH(0, 0, EPI_FWD_I8, 0);
+    }
     if (pair) EFQAT_LAUNCH(0, 0, EPI_FWD, 1);
     EFQAT_LAUNCH(0, 0, EPI_FWD, 0);
   }

@@ -108,7 +108,7 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
                cudaStream_t st);
 
 // ---- gemm.cu ------------------------------------------------------------------------
-enum GemmEpi { EPI_FWD = 0, EPI_DX = 1, EPI_PART = 2 };
+enum GemmEpi { EPI_FWD = 0, EPI_DX = 1, EPI_PART = 2, EPI_FWD_I8 = 3 };   // EPI_FWD_I8: chosen inside run_gemm
 
 // Implicit-GEMM convolution geometry (stride 1).  The activation operand is read through a
 // 4-D tensor map over its NHWC tensor with a box of pixels shifted by the filter tap; pixels

@@ -394,6 +394,8 @@ def run_ours(args):
             "config": {"workload": "configs[1]: BERT-base-shaped linears 768->2304, 768->768, 768->3072, 3072->768 "
                                    "at M=4096, bf16 activations, W8A8, CWPL",
                        "unfrozen": frac, "l2": "256 MiB buffer written between timed steps",
+                       "arithmetic": "forward: 8-bit codes on the integer tensor cores, int32 accumulate; "
+                                     "backward contractions: bf16 operands, fp32 accumulate",
                        "optimizer": "fused SGD-momentum on the unfrozen rows (momentum 0.9, weight decay 1e-4, "
                                     f"lr {SGD_LR:g} scaled for unit-variance synthetic dY)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},

@@ -140,9 +140,9 @@ int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_des
 /* ---- a2 + a3: fake-quantize X and W, forward GEMM (Eq. 1, Eq. 3, Section 3.1) -------- */
 /* Y[m,n] = s_x * s_w[n] * sum_k (q_x[m,k] - Z) * q_w[n,k] + bias[n].
  * s_w [N], s_x [1], z_x [1] (ignored when x_symmetric), bias [N] or NULL; Y in act_dtype.
- * The integer sum is exact: plain layers with 512 <= K <= 32768, K % 16 == 0 and N % 32 == 0
- * contract the 8-bit codes on the integer tensor cores (int32 accumulation), all others
- * contract the same integers held in bf16 (fp32 accumulation). */
+ * Plain layers with 512 <= K <= 32768, K % 16 == 0 and N % 32 == 0 contract the 8-bit codes
+ * on the integer tensor cores (int32 accumulation: the integer sum is exact); all others
+ * contract the same integers held in bf16, with fp32 accumulation. */
 int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
                         const float* W, const float* s_w, const float* s_x, const float* z_x,
                         const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream);

@@ -29,6 +29,10 @@ SMALL = [
     _case("one_row", 1, 64, 8, torch.float32, seed=5),
     _case("two_bit", 160, 72, 40, torch.bfloat16, w_bits=2, x_bits=2, seed=6),
     _case("smallest", 8, 8, 8, torch.bfloat16, seed=7),
+    # contractions of 512 and more with N % 32 == 0: the forward runs on the integer tensor cores
+    _case("int8_asym_bf16", 333, 640, 96, torch.bfloat16, seed=8),
+    _case("int8_asym_f32", 200, 512, 64, torch.float32, seed=9),
+    _case("int8_sym_w4", 130, 1024, 160, torch.bfloat16, w_bits=4, x_bits=8, sym=True, seed=10),
 ]
 
 

@@ -297,17 +297,28 @@ def backward_efqat(dY, X, W, s_w, s_x, z_x, idx, w_bits, x_bits, x_symmetric=Fal
 
 
 def backward_efqat_direct(dY, X, W, s_w, s_x, z_x, idx, w_bits, x_bits,
-                          x_symmetric=False):
+                          x_symmetric=False, operand_model="exact"):
     """The same partial weight gradient computed the way Algorithm 1 words it:
     take the columns idx of dY, contract them with X^, never forming the other
-    rows.  Must agree with `backward_efqat` (self-check of the indexing)."""
+    rows.  Must agree with `backward_efqat` (self-check of the indexing).
+
+    operand_model as in `backward_full` (only the rounding of dY to bf16 touches
+    this contraction; the integer operand is exact either way).  Also returns
+    the sums of absolute terms that bound the rounding error of the
+    contraction and of the weight-scale reduction."""
     idx = np.asarray(idx, dtype=np.int64)
-    dYd = np.asarray(dY, dtype=F64)
+    dYd = np.asarray(dY, dtype=F64)[:, idx]
+    if operand_model == "bf16":
+        dYd = bf16_rne(dYd)
+    elif operand_model != "exact":
+        raise ValueError(operand_model)
     qx = fake_quant_x(X, s_x, z_x, x_bits, x_symmetric)
     qw = fake_quant_w(np.asarray(W)[idx], np.asarray(s_w)[idx], w_bits)
-    G = F64(F32(s_x)) * (dYd[:, idx].T @ qx["c0"])
+    G = F64(F32(s_x)) * (dYd.T @ qx["c0"])
     return dict(dW_sel=np.where(qw["flag"] == 0, G, 0.0),
-                dS_w_sel=(G * qw["t"]).sum(axis=1))
+                dS_w_sel=(G * qw["t"]).sum(axis=1),
+                dS_w_sel_abs=np.abs(G * qw["t"]).sum(axis=1),
+                G_w_sel_abs=F64(F32(s_x)) * (np.abs(dYd).T @ np.abs(qx["c0"])))
 
 
 def sgd_rows(W, V, dW_sel, idx, lr, momentum, weight_decay):

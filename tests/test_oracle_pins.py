@@ -119,6 +119,32 @@ def test_u32_and_bf16_against_torch():
     assert np.array_equal(O.bf16_rne(v), ref)
 
 
+def test_code_rule_against_literal_division_on_workload_inputs():
+    """Eq. 1 / Eq. 3 write round(x / s).  The oracle (and the CUDA path) decide the code from
+    fl32(x * fl32(1/s)) instead.  On the seeded inputs of the first two workload families the two
+    rules may differ only where x/s sits within an fp32 rounding of a tie: at most one code in
+    1e5, and never by more than one step."""
+    from paper_2411_11038_b200 import inputs as I
+    for case in I.config1() + I.config2()[:2]:
+        T = I.make_tensors(case)
+        X, W = I.as_f64(T["X"]), I.as_f64(T["W"])
+        s_w = O.init_minmax_w(W, case.w_bits)
+        s_x, z_x = O.init_minmax_x(X, case.x_bits, case.x_symmetric)
+        for fx, fw in ((1.0, 1.0), (0.8, 0.85)):          # at the MinMax start and after the scales moved
+            sx = np.float32(s_x * np.float32(fx))
+            sw = (s_w * np.float32(fw)).astype(np.float32)
+            qx = O.fake_quant_x(X, sx, z_x, case.x_bits, case.x_symmetric)
+            lo, hi = (-O.qmax_w(case.x_bits), O.qmax_w(case.x_bits)) if case.x_symmetric else (0, O.qmax_x(case.x_bits))
+            lit = np.clip(np.rint(X / np.float64(sx)) + qx["Zr"], lo, hi)
+            d = np.abs(qx["q"] - lit)
+            assert d.max() <= 1 and (d != 0).mean() <= 1e-5, (case.name, "x", d.max(), (d != 0).mean())
+            qw = O.fake_quant_w(W, sw, case.w_bits)
+            Q = O.qmax_w(case.w_bits)
+            lit = np.clip(np.rint(W / sw.astype(np.float64)[:, None]), -Q, Q)
+            d = np.abs(qw["q"] - lit)
+            assert d.max() <= 1 and (d != 0).mean() <= 1e-5, (case.name, "w", d.max(), (d != 0).mean())
+
+
 def test_fake_quant_matches_torch_fake_quantize():
     r = rng(4)
     X = torch.from_numpy(r.standard_normal((33, 17)).astype(np.float32) * 2)
@@ -392,6 +418,23 @@ def test_bf16_operand_model_is_close_and_distinct():
     assert np.array_equal(b["dW"], e["dW"])
 
 
+def test_direct_partial_backward_operand_model_and_abs_sums():
+    """The restricted loop of Algorithm 1 under the bf16 operand model and its abs-sums equal
+    the matching rows of the full backward under the same model."""
+    X, W, dY, s_w, s_x, z_x = _tiny(31, M=40, K=24, N=16, clip=True)
+    idx = [1, 4, 5, 11, 15]
+    for model in ("exact", "bf16"):
+        e = O.backward_efqat(dY, X, W, s_w, s_x, z_x, idx, 8, 8, operand_model=model)
+        d = O.backward_efqat_direct(dY, X, W, s_w, s_x, z_x, idx, 8, 8, operand_model=model)
+        for key in ("dW_sel", "dS_w_sel", "dS_w_sel_abs", "G_w_sel_abs"):
+            np.testing.assert_allclose(d[key], e[key], rtol=1e-13, atol=1e-13, err_msg=f"{model} {key}")
+    # the abs-sums are what they say: sums of |terms| of the plain loops
+    c0 = O.fake_quant_x(X, s_x, z_x, 8)["c0"]
+    brute = np.array([[sum(abs(float(dY[m, n]) * c0[m, k]) for m in range(40)) for k in range(24)] for n in idx])
+    exact = O.backward_efqat_direct(dY, X, W, s_w, s_x, z_x, idx, 8, 8)
+    np.testing.assert_allclose(exact["G_w_sel_abs"], float(s_x) * brute, rtol=1e-12)
+
+
 def test_sgd_rows_against_torch_sgd():
     r = rng(18)
     W = r.standard_normal((7, 5))
@@ -487,3 +530,39 @@ def test_conv_brute_force_seven_loops():
                             for c in range(2):
                                 acc += qx[0, hh, ww, c] * qw[n, r, s, c]
                 assert abs(Y[0, h, w, n] - acc) < 1e-12
+
+
+@pytest.mark.parametrize("stride,pad", [(1, 1), (2, 1)])
+def test_conv_bf16_operand_model_against_torch_on_rounded_operands(stride, pad):
+    """The 'bf16' operand model of the convolution backward = the exact backward evaluated by an
+    independent routine (torch conv2d autograd, fp64) on operands rounded by torch itself: dY to
+    bf16 and, for the input gradient only, w^ to bf16(fl32(s_w q_w)) with s_w per OUTPUT channel."""
+    X, W, s_w, s_x, z_x = _conv_case(41, B=2, H=6, Wd=5, C=4, N=6)
+    s_w = (s_w * (1.0 + 0.37 * np.arange(6))).astype(np.float32)      # distinct scales: a wrong axis shows
+    qx = O.fake_quant_x(X, s_x, z_x, 8)
+    qw = O.fake_quant_w(W, s_w, 4)
+    Y = O.conv_forward(X, W, s_w, s_x, z_x, None, 4, 8, stride, pad)
+    dY = rng(42).standard_normal(Y.shape)
+    b = O.conv_backward_full(dY, X, W, s_w, s_x, z_x, 4, 8, stride, pad, operand_model="bf16")
+    e = O.conv_backward_full(dY, X, W, s_w, s_x, z_x, 4, 8, stride, pad, operand_model="exact")
+    dYb = torch.tensor(dY, dtype=torch.float32).to(torch.bfloat16).to(torch.float64)
+    wb = (torch.tensor(s_w).reshape(-1, 1, 1, 1) * torch.tensor(qw["q"], dtype=torch.float32)) \
+        .to(torch.bfloat16).to(torch.float64)
+    # input gradient: dY_b against the rounded dequantised weights
+    xh = torch.tensor(qx["deq"]).permute(0, 3, 1, 2).requires_grad_(True)
+    torch.nn.functional.conv2d(xh, wb.permute(0, 3, 1, 2), stride=stride, padding=pad) \
+        .backward(dYb.permute(0, 3, 1, 2))
+    Gx = xh.grad.permute(0, 2, 3, 1).numpy()
+    np.testing.assert_allclose(b["dX"], np.where(qx["flag"] == 0, Gx, 0), atol=1e-12)
+    np.testing.assert_allclose(b["dS_x"], (Gx * qx["t"]).sum(), atol=1e-10)
+    np.testing.assert_allclose(b["dZ_x"], (Gx * qx["dz"]).sum(), atol=1e-10)
+    # weight gradient: dY_b against the exact integer activations, s_x applied afterwards
+    wh = torch.zeros(W.shape, dtype=torch.float64).permute(0, 3, 1, 2).contiguous().requires_grad_(True)
+    xc = torch.tensor(qx["c0"]).permute(0, 3, 1, 2)
+    torch.nn.functional.conv2d(xc, wh, stride=stride, padding=pad).backward(dYb.permute(0, 3, 1, 2))
+    Gw = float(s_x) * wh.grad.permute(0, 2, 3, 1).numpy()
+    np.testing.assert_allclose(b["dW"], np.where(qw["flag"] == 0, Gw, 0), atol=1e-12)
+    np.testing.assert_allclose(b["dS_w"], (Gw * qw["t"]).sum(axis=(1, 2, 3)), atol=1e-10)
+    # close to, and distinct from, the exact model; db never depends on the model
+    assert np.abs(b["dX"] - e["dX"]).max() <= 1e-2 * np.abs(e["dX"]).max()
+    assert not np.array_equal(b["dX"], e["dX"]) and np.array_equal(b["db"], e["db"])

@@ -418,3 +418,31 @@ def conv_backward_efqat(dY, X, W, s_w, s_x, z_x, idx, w_bits, x_bits, stride=1, 
     out["dS_w_sel"] = full["dS_w"][idx]
     out["dS_w_sel_abs"] = full["dS_w_abs"][idx]
     return out
+
+
+def conv_backward_efqat_direct(dY, X, W, s_w, s_x, z_x, idx, w_bits, x_bits, stride=1, pad=0,
+                               x_symmetric=False, operand_model="exact"):
+    """Partial weight gradient of the convolution the way Algorithm 1 words it:
+    take the output channels idx of dY and contract them with the patches of
+    x^, never forming the other channels' rows.  Must agree with
+    `conv_backward_efqat`.  Also returns the sums of absolute terms of the
+    contraction and of the weight-scale reduction."""
+    idx = np.asarray(idx, dtype=np.int64)
+    Wa = np.asarray(W)
+    N, R, S, C = Wa.shape
+    dYd = np.asarray(dY, dtype=F64)[..., idx]
+    if operand_model == "bf16":
+        dYd = bf16_rne(dYd)
+    elif operand_model != "exact":
+        raise ValueError(operand_model)
+    qx = fake_quant_x(X, s_x, z_x, x_bits, x_symmetric)
+    qw = fake_quant_w(Wa[idx], np.asarray(s_w)[idx], w_bits)
+    P = _patches(qx["c0"], R, S, stride, pad).reshape(-1, R * S * C)
+    dY2 = dYd.reshape(int(np.prod(dYd.shape[:3])), len(idx))
+    G = (F64(F32(s_x)) * (dY2.T @ P)).reshape(len(idx), R, S, C)
+    G_abs = (F64(F32(s_x)) * (np.abs(dY2).T @ np.abs(P))).reshape(len(idx), R, S, C)
+    ax = tuple(range(1, 4))
+    return dict(dW_sel=np.where(qw["flag"] == 0, G, 0.0),
+                dS_w_sel=(G * qw["t"]).sum(axis=ax),
+                dS_w_sel_abs=np.abs(G * qw["t"]).sum(axis=ax),
+                G_w_sel_abs=G_abs)

@@ -566,3 +566,17 @@ def test_conv_bf16_operand_model_against_torch_on_rounded_operands(stride, pad):
     # close to, and distinct from, the exact model; db never depends on the model
     assert np.abs(b["dX"] - e["dX"]).max() <= 1e-2 * np.abs(e["dX"]).max()
     assert not np.array_equal(b["dX"], e["dX"]) and np.array_equal(b["db"], e["db"])
+
+
+@pytest.mark.parametrize("stride,pad", [(1, 1), (2, 1)])
+def test_conv_direct_partial_backward_equals_rows_of_full(stride, pad):
+    X, W, s_w, s_x, z_x = _conv_case(43, B=2, H=6, Wd=5, C=4, N=6)
+    Y = O.conv_forward(X, W, s_w, s_x, z_x, None, 4, 8, stride, pad)
+    dY = rng(44).standard_normal(Y.shape)
+    for idx in ([], [2], [0, 3, 5]):
+        for model in ("exact", "bf16"):
+            e = O.conv_backward_efqat(dY, X, W, s_w, s_x, z_x, idx, 4, 8, stride, pad, operand_model=model)
+            d = O.conv_backward_efqat_direct(dY, X, W, s_w, s_x, z_x, idx, 4, 8, stride, pad, operand_model=model)
+            for key in ("dW_sel", "dS_w_sel", "dS_w_sel_abs"):
+                np.testing.assert_allclose(d[key], e[key], rtol=1e-13, atol=1e-13)
+            assert np.all(d["G_w_sel_abs"] >= np.abs(d["dW_sel"]) - 1e-12)

@@ -3,23 +3,27 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--frac R]
 
-Workload: the four BERT-base-shaped encoder linears at M = 32 x 128 = 4096 tokens with
-bf16 activations, W8A8, per-layer channel selection.  One step = one pass of the whole
-path over one batch: importance + Top-K selection for the four layers, then for each
-layer the fake-quantised forward and the partial backward (dX, dS_x, dZ_x, db, and dW /
-dS_w of the selected channels only).
+Headline workload: the two largest shapes of the GEMM-shape sweep, M = 16384 tokens with
+(K, N) = (8192, 8192) and (4096, 16384), bf16 activations, W8A8, per-layer channel selection,
+5 % of the channels unfrozen.  One step = one pass of the whole path over one batch:
+importance + Top-K selection for both layers, then for each layer the fake-quantised forward
+and the partial backward (dX, dS_x, dZ_x, db, and dW / dS_w of the selected channels only)
+with the fused SGD-momentum update of the unfrozen rows.
 
 The printed JSON line reports the step throughput in algorithmic TFLOP/s
 (2MNK forward + 2MNK(1 + k/N) backward), the backward-only sweep over the unfrozen
 fractions with its speed-up over the library's own full-QAT backward, the tensor-core
-roofline of the dominant GEMM kernel, the oracle's CPU time on the same workload and the
-end-to-end number with host buffers.
+roofline of the dominant GEMM kernel and of each GEMM kind, the oracle's CPU time on a
+bounded sample of the same workload and the end-to-end number with host buffers.  The
+BERT-base-shaped linears at M = 4096 are measured the same way under the key "bert_base".
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
 import statistics
 import sys
 import threading
@@ -37,11 +41,22 @@ FRACS = (0.0, 0.05, 0.25, 1.0)
 METRIC = ("fq-linear backward TFLOP/s & speedup vs full-QAT bwd per unfrozen %; roofline frac "
           "[value: TFLOP/s of one step of the whole path = select + fwd + partial bwd + fused sparse SGD; "
           "backward-only ms, TFLOP/s and speedups per unfrozen % under 'bwd']")
+WORKLOAD_NAME = ("configs[4]: GEMM-shape sweep, M=16384 tokens, (K,N) = (8192,8192) and (4096,16384), "
+                 "bf16 activations, W8A8, CWPL, selection recomputed every step")
 L2_FLUSH_BYTES = 256 << 20
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (set to None whenever the kernel changes after a capture).
 SGD_LR = 1e-9
-DOMINANT_TRAFFIC_BYTES = 28.93e6    # mean over the four dX launches of one step (profiles/gemm_kernel_dx_bench_cfg2.txt)
+# ncu capture of the dominant kernel on the first layer of the headline workload: the file states
+# the DRAM bytes per launch and the hash of the kernel sources it was taken from.
+TRAFFIC_FILE = os.path.join("profiles", "gemm_kernel_dx_cfg5_8192x8192.txt")
+KERNEL_SOURCES = ("gemm.cu", "ptx.cuh", "common.cuh")
+# bounded sample of the headline workload for the oracle: leading tokens and output channels
+REF_SAMPLE = dict(tokens=256, channels=1024)
+CPU_SAMPLE = dict(tokens=512, channels=2048)
+
+
+def headline_cases():
+    c = I.config5()
+    return [c[3], c[2]]
 
 
 def load_peaks():
@@ -53,12 +68,36 @@ def load_peaks():
     return dict(tflops=1590.0, tflops_sustained=1400.0, hbm_gbs=6650.0, source="fallback")
 
 
+def kernel_source_hash():
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2411_11038_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic():
+    """DRAM bytes per launch of the dominant kernel from the kept ncu summary; None once the
+    kernel sources differ from those the capture was taken from."""
+    path = os.path.join(ROOT, TRAFFIC_FILE)
+    if not os.path.exists(path):
+        return None, "no capture kept"
+    txt = open(path).read()
+    m = re.search(r"^dram_bytes_per_launch:\s*([0-9.eE+]+)", txt, re.M)
+    h = re.search(r"^kernel_source_hash:\s*([0-9a-f]+)", txt, re.M)
+    if not m or not h:
+        return None, "capture summary has no traffic line"
+    if h.group(1) != kernel_source_hash():
+        return None, "kernel changed since the capture"
+    return float(m.group(1)), TRAFFIC_FILE
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_s: float = 0.002):
         super().__init__(daemon=True)
         self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
+        self.period_s = period_s
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -90,10 +129,11 @@ class ClockSampler(threading.Thread):
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.01)
+            time.sleep(self.period_s)
 
     def summary(self):
         return dict(sm_mhz=(statistics.median(self.samples) if self.samples else None),
+                    sm_min_mhz=(min(self.samples) if self.samples else None),
                     sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=len(self.samples))
 
 
@@ -109,20 +149,27 @@ def physical_gpu_index(local_rank: int) -> int:
 
 # ----------------------------------------------------------------------------------------
 class Workload:
-    """Device-resident tensors and pre-marshalled calls of the four layers."""
+    """Device-resident tensors and pre-marshalled calls of a list of layers."""
 
-    def __init__(self, ctx, device):
+    def __init__(self, ctx, device, cases, fracs, e2e_frac=None, keep_sample=None):
         from paper_2411_11038_b200 import binding as B
         self.B, self.ctx, self.device = B, ctx, device
-        self.cases = I.config2()
+        self.cases = cases
         self.layers = []
+        self.samples = []
         for c in self.cases:
             T = I.make_tensors(c)
             D = {k: v.to(device) for k, v in T.items()}
             D["s_w"] = B.init_weight_scales(ctx, D["W"], c.w_bits)
             D["s_x"], D["z_x"] = B.init_act_qparams(ctx, D["X"], c.x_bits, c.x_symmetric)
-            D["host_X"] = T["X"].pin_memory()
-            D["host_dY"] = T["dY"].pin_memory()
+            if e2e_frac is not None:
+                D["host_X"] = T["X"].pin_memory()
+                D["host_dY"] = T["dY"].pin_memory()
+                k_e = max(B.ratio_to_k(e2e_frac, c.N), 1)
+                D["host_dW"] = torch.empty((k_e, c.K), dtype=torch.float32).pin_memory()
+                D["host_small"] = torch.empty(2 * c.N + 2, dtype=torch.float32).pin_memory()
+            if keep_sample:
+                self.samples.append(sample_of(c, T, **keep_sample))
             plan = B.LayerPlan(ctx, c.M, c.N, c.K, c.act_dtype, c.w_bits, c.x_bits, c.x_symmetric, c.N, device)
             # fused sparse SGD-momentum of Algorithm 1 on the unfrozen rows (momentum and weight decay
             # of Section 4).  The learning rate is scaled down: the synthetic dY has unit variance,
@@ -130,11 +177,10 @@ class Workload:
             # over hundreds of timed steps; the arithmetic and the traffic are those of any rate.
             D["mom"] = torch.zeros_like(D["W"])
             D["sgd"] = B.make_sgd(SGD_LR, 0.9, 1e-4, D["W"], D["mom"])
-            D["host_dW"] = torch.empty((c.N, c.K), dtype=torch.float32).pin_memory()
-            D["host_small"] = torch.empty(2 * c.N + 2, dtype=torch.float32).pin_memory()
             self.layers.append((c, D, plan))
+            del T
         self.sel = {}
-        for f in FRACS:
+        for f in fracs:
             ks = [B.ratio_to_k(f, c.N) for c in self.cases]
             plan = B.SelectPlan(ctx, B.CWPL, [D["W"] for _, D, _ in self.layers], ks)
             offs = np.concatenate([[0], np.cumsum(ks)]).astype(int)
@@ -249,53 +295,168 @@ def timed(fn, steps, warmup, flush, sync_all=None, after_warmup=None):
 
 
 # ----------------------------------------------------------------------------------------
-def oracle_step_seconds(frac, layers=None, rows=None):
-    """One pass of the oracle, as it stands, over the same workload (CPU, fp64)."""
+# the oracle on the host cores
+# ----------------------------------------------------------------------------------------
+def sample_of(case, T, tokens, channels):
+    """Leading `tokens` rows and `channels` output channels of a layer's tensors (CPU, fp64)."""
+    t, n = min(tokens, case.M), min(channels, case.N)
+    return dict(name=case.name, K=case.K, tokens=t, channels=n, w_bits=case.w_bits, x_bits=case.x_bits,
+                x_symmetric=case.x_symmetric,
+                X=I.as_f64(T["X"][:t]), W=I.as_f64(T["W"][:n]), dY=I.as_f64(T["dY"][:t, :n]),
+                bias=I.as_f64(T["bias"][:n]))
+
+
+def oracle_sample_seconds(samples, frac):
+    """One pass of the oracle, as it stands, over the sampled layers: MinMax scales, selection,
+    forward, EfQAT backward, SGD on the unfrozen rows.  Returns (seconds, algorithmic FLOPs)."""
     from oracle import efqat_oracle as O
-    cases = I.config2()
-    if layers is not None:
-        cases = [cases[i] for i in layers]
-    if rows is not None:
-        cases = [I.shrink(c, rows) for c in cases]
     flops = 0.0
     t0 = time.perf_counter()
-    for c in cases:
-        T = I.make_tensors(c)
-        X, W, dY, b = (I.as_f64(T[k]) for k in ("X", "W", "dY", "bias"))
-        s_w = O.init_minmax_w(W, c.w_bits)
-        s_x, z_x = O.init_minmax_x(X, c.x_bits, c.x_symmetric)
-        k = O.ratio_to_k(frac, c.N)
+    for s in samples:
+        X, W, dY, b = s["X"], s["W"], s["dY"], s["bias"]
+        s_w = O.init_minmax_w(W, s["w_bits"])
+        s_x, z_x = O.init_minmax_x(X, s["x_bits"], s["x_symmetric"])
+        k = O.ratio_to_k(frac, s["channels"])
         idx = O.select_cwpl([W], [k])[0]
-        O.forward(X, W, s_w, s_x, z_x, b, c.w_bits, c.x_bits, c.x_symmetric)
-        g = O.backward_efqat(dY, X, W, s_w, s_x, z_x, idx, c.w_bits, c.x_bits, c.x_symmetric)
+        O.forward(X, W, s_w, s_x, z_x, b, s["w_bits"], s["x_bits"], s["x_symmetric"])
+        g = O.backward_efqat(dY, X, W, s_w, s_x, z_x, idx, s["w_bits"], s["x_bits"], s["x_symmetric"])
         O.sgd_rows(W, np.zeros_like(W), g["dW_sel"], idx, SGD_LR, 0.9, 1e-4)
-        flops += 2.0 * c.M * c.N * c.K * 2 + 2.0 * c.M * k * c.K
-    return time.perf_counter() - t0, flops, [c.name for c in cases]
+        flops += 2.0 * s["tokens"] * s["channels"] * s["K"] * 2 + 2.0 * s["tokens"] * k * s["K"]
+    return time.perf_counter() - t0, flops
+
+
+def sample_text(samples, frac):
+    per = ", ".join(f"{s['name']} [{s['tokens']} tokens x {s['channels']} channels x K={s['K']}]" for s in samples)
+    return (f"oracle (fp64 numpy: MinMax scales, selection, forward, EfQAT backward, SGD rows) on the leading tokens "
+            f"and output channels of each layer of the workload: {per}; {int(frac * 100)}% unfrozen")
+
+
+def workload_config(frac, world):
+    return {"workload": WORKLOAD_NAME, "unfrozen": frac,
+            "l2": "inputs exceed L2; a 256 MiB buffer is also written between timed steps",
+            "arithmetic": "forward: 8-bit codes on the integer tensor cores, int32 accumulate; "
+                          "backward contractions: bf16 operands, fp32 accumulate",
+            "optimizer": "fused SGD-momentum on the unfrozen rows (momentum 0.9, weight decay 1e-4, "
+                         f"lr {SGD_LR:g} scaled for unit-variance synthetic dY)",
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
 def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     frac = args.frac
-    layers, rows = [1], 1024    # bounded sample: 1024 tokens of the 768 -> 768 attention-output layer
-    for _ in range(min(args.warmup, 3)):
-        oracle_step_seconds(frac, layers, rows)
-    tot, fl, names = 0.0, 0.0, []
+    samples = []
+    for c in headline_cases():
+        T = I.make_tensors(c)
+        samples.append(sample_of(c, T, **REF_SAMPLE))
+        del T
+    for _ in range(min(args.warmup, 2)):
+        oracle_sample_seconds(samples, frac)
+    tot, fl = 0.0, 0.0
     for _ in range(args.steps):
-        s, f, names = oracle_step_seconds(frac, layers, rows)
+        s, f = oracle_sample_seconds(samples, frac)
         tot += s
         fl += f
     val = fl / tot / 1e12
     cores = os.cpu_count()
-    sample = f"oracle fwd + EfQAT bwd (fp64 numpy) on layer {names[0]} (first {rows} tokens), {int(frac * 100)}% unfrozen"
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(args.steps, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "configs[1] BERT-base-shaped linears (bounded sample)", "unfrozen": frac},
-        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "config": workload_config(frac, world),
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": sample_text(samples, frac)},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+# ----------------------------------------------------------------------------------------
+def measure(wl, ctx, frac, steps, warmup, peaks, sync_all, max_over_ranks, world, sampler=None, extras=True):
+    """Headline pass, per-kernel pass and backward sweep of one workload."""
+    B = wl.B
+    mark = {}
+
+    def start_counting():
+        mark["launches"] = B.launch_count()
+        if sampler is not None:
+            sampler.start()
+
+    total_ms = timed(lambda: wl.step(frac), steps, warmup, wl.flush, sync_all, start_counting)
+    if sampler is not None:
+        sampler.stop_flag = True
+    launches = B.launch_count() - mark["launches"]
+    if sampler is not None:
+        sampler.join(timeout=2)
+    ms_per_step = max_over_ranks(total_ms) / steps
+    value = world * wl.flops(frac) / (ms_per_step * 1e-3) / 1e12
+
+    # The same K steps once more with a pair of CUDA events around every GEMM launch.  The events
+    # serialise launches that otherwise overlap their set-up with the previous kernel's tail, so
+    # they stay out of the headline pass above.
+    prof_ms = timed(lambda: wl.step(frac), steps, 3, wl.flush, sync_all, lambda: ctx.profile_enable(True))
+    kinds = [ctx.profile_read(i) for i in range(3)]      # (total ms, launches) of the K profiled steps
+    ctx.profile_enable(False)
+    gf = wl.gemm_flops(frac)
+    names = ["gemm_kernel<fwd epilogue>", "gemm_kernel<dX epilogue>", "gemm_kernel<dW partial epilogue>"]
+    # forward: 8-bit integer tensor-core operations, nominal rate twice the bf16 one
+    kind_peak = [2.0 * peaks["tflops"], peaks["tflops"], peaks["tflops"]]
+    per_kind = {}
+    for i, n in enumerate(names):
+        ms_i, n_i = kinds[i]
+        ach = (gf[i] * steps) / (ms_i * 1e-3) / 1e12 if n_i and ms_i > 0 else None
+        per_kind[n] = {"ms_per_step": ms_i / steps, "launches_per_step": n_i / steps,
+                       "achieved": ach, "unit": "Top/s (int8)" if i == 0 else "TFLOP/s (bf16)",
+                       "peak": kind_peak[i], "frac": (ach / kind_peak[i]) if ach else None}
+    dom = max(range(3), key=lambda i: kinds[i][0])
+    dom_ms, dom_n = kinds[dom]
+    achieved = per_kind[names[dom]]["achieved"]
+    traffic, traffic_src = recorded_traffic() if wl.cases[0].name.startswith("cfg5") else (None, "not captured")
+    roofline = {"bound": "tensor", "kernel": names[dom], "achieved": achieved, "peak": kind_peak[dom],
+                "unit": "TFLOP/s", "frac": (achieved / kind_peak[dom]) if achieved else None,
+                "traffic": traffic, "traffic_source": traffic_src,
+                "peak_source": f"{peaks['source']} burst bf16 GEMM" + (" x 2 (int8 nominal ratio)" if dom == 0 else ""),
+                "launches": dom_n, "avg_launch_ms": dom_ms / max(dom_n, 1),
+                "timed_in": "second pass of the same K steps with per-kernel CUDA events",
+                "ms_per_step_with_kernel_events": max_over_ranks(prof_ms) / steps,
+                "per_kind": per_kind}
+
+    bwd_report, sel_ms = {}, None
+    if extras:
+        sweep_steps = max(20, steps // 4)
+        bwd = {}
+        for f in sorted(wl.sel):
+            wl.select(f)
+            bwd[f] = max_over_ranks(timed(lambda: wl.backward(f), sweep_steps, 5, wl.flush, sync_all) / sweep_steps)
+        for f in sorted(wl.sel):
+            fl = wl.flops(f, fwd=False)
+            tf = fl / (bwd[f] * 1e-3) / 1e12
+            bwd_report[f"{int(round(f * 100))}%"] = {
+                "ms": bwd[f], "tflops": tf, "frac_of_sustained_peak": tf / peaks["tflops_sustained"],
+                "speedup_vs_full_qat": bwd[1.0] / bwd[f], "ideal_speedup": 2.0 / (1.0 + f)}
+        sel_ms = max_over_ranks(timed(lambda: wl.select(frac), sweep_steps, 5, wl.flush, sync_all) / sweep_steps)
+        roofline["whole_backward"] = {
+            "tflops": bwd_report[f"{int(round(frac * 100))}%"]["tflops"], "peak": peaks["tflops_sustained"],
+            "frac": bwd_report[f"{int(round(frac * 100))}%"]["frac_of_sustained_peak"],
+            "peak_source": f"{peaks['source']} sustained bf16 GEMM",
+            "what": "prepare + dX GEMM + partial dW GEMM + finalize (with SGD) on the algorithmic FLOPs 2MNK(1+k/N)"}
+    return dict(ms_per_step=ms_per_step, value=value, launches=int(launches), roofline=roofline, bwd=bwd_report,
+                select_ms=sel_ms)
+
+
+def run_capture(args):
+    """Short run for a profiler: the first layer of the headline workload alone, a few steps."""
+    from paper_2411_11038_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = B.Context(0)
+    wl = Workload(ctx, dev, headline_cases()[:1], (args.frac,))
+    for _ in range(3):
+        wl.flush.zero_()
+        wl.step(args.frac)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    print(json.dumps({"capture": wl.cases[0].name, "kernel_source_hash": kernel_source_hash()}))
 
 
 def run_ours(args):
@@ -311,65 +472,18 @@ def run_ours(args):
     max_over_ranks = reps.max_over_ranks
 
     ctx = B.Context(local)
-    wl = Workload(ctx, dev)
     frac = args.frac
     peaks = load_peaks()
+    want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline and not args.skip_extras
+    wl = Workload(ctx, dev, headline_cases(), FRACS if not args.skip_extras else (frac, 1.0), e2e_frac=frac,
+                  keep_sample=CPU_SAMPLE if want_cpu else None)
 
     # ---- headline: K steps of the whole path, device-resident inputs
     sampler = ClockSampler(physical_gpu_index(local))
-    mark = {}
-
-    def start_counting():
-        mark["launches"] = B.launch_count()
-        sampler.start()
-
-    total_ms = timed(lambda: wl.step(frac), args.steps, args.warmup, wl.flush, sync_all, start_counting)
-    sampler.stop_flag = True
-    launches = B.launch_count() - mark["launches"]
-    sampler.join(timeout=2)
-    total_ms = max_over_ranks(total_ms)
-    ms_per_step = total_ms / args.steps
-    value = world * wl.flops(frac) / (ms_per_step * 1e-3) / 1e12
-
-    # ---- roofline of the dominant kernel (largest share of GEMM time): the same K steps once
-    # more with a pair of CUDA events around every GEMM launch.  The events serialise launches
-    # that otherwise overlap their set-up with the previous kernel's tail, so they stay out of
-    # the headline pass above.
-    prof_ms = timed(lambda: wl.step(frac), args.steps, 3, wl.flush, sync_all, lambda: ctx.profile_enable(True))
-    kinds = [ctx.profile_read(i) for i in range(3)]      # (total ms, launches) of the K profiled steps
-    ctx.profile_enable(False)
-    gf = wl.gemm_flops(frac)
-    names = ["gemm_kernel<fwd epilogue>", "gemm_kernel<dX epilogue>", "gemm_kernel<dW partial epilogue>"]
-    dom = max(range(3), key=lambda i: kinds[i][0])
-    dom_ms, dom_n = kinds[dom]
-    avg_launch_ms = dom_ms / max(dom_n, 1)
-    # algorithmic FLOPs of all launches of that kind in the timed region / their summed duration
-    achieved = (gf[dom] * args.steps) / (dom_ms * 1e-3) / 1e12 if dom_n else None
-    roofline = {"bound": "tensor", "kernel": names[dom], "achieved": achieved, "peak": peaks["tflops"],
-                "unit": "TFLOP/s", "frac": (achieved / peaks["tflops"]) if achieved else None,
-                "traffic": DOMINANT_TRAFFIC_BYTES, "peak_source": f"{peaks['source']} burst bf16 GEMM",
-                "launches": dom_n, "avg_launch_ms": avg_launch_ms,
-                "timed_in": "second pass of the same K steps with per-kernel CUDA events",
-                "ms_per_step_with_kernel_events": max_over_ranks(prof_ms) / args.steps,
-                "gemm_ms_per_step": {n: kinds[i][0] / args.steps for i, n in enumerate(names)}}
-
-    # ---- backward-only sweep over the unfrozen fractions
-    sweep_steps = max(20, args.steps // 4)
-    bwd = {}
-    for f in (() if args.skip_extras else FRACS):
-        wl.select(f)
-        ms = timed(lambda: wl.backward(f), sweep_steps, 5, wl.flush, sync_all) / sweep_steps
-        ms = max_over_ranks(ms)
-        bwd[f] = ms
-    bwd_report = {}
-    for f in (() if args.skip_extras else FRACS):
-        fl = wl.flops(f, fwd=False)
-        bwd_report[f"{int(round(f * 100))}%"] = {
-            "ms": bwd[f], "tflops": fl / (bwd[f] * 1e-3) / 1e12, "speedup_vs_full_qat": bwd[1.0] / bwd[f],
-            "ideal_speedup": 2.0 / (1.0 + f)}
-    sel_ms = None
-    if not args.skip_extras:
-        sel_ms = max_over_ranks(timed(lambda: wl.select(frac), sweep_steps, 5, wl.flush, sync_all) / sweep_steps)
+    all_clock = ClockSampler(physical_gpu_index(local), period_s=0.02)
+    all_clock.start()
+    head = measure(wl, ctx, frac, args.steps, args.warmup, peaks, sync_all, max_over_ranks, world, sampler,
+                   extras=not args.skip_extras)
 
     # ---- end to end: inputs from pinned host memory, parameter gradients back to it
     e2e_steps = 3 if args.skip_extras else max(10, args.steps // 4)
@@ -377,36 +491,50 @@ def run_ours(args):
     bi, bo = wl.e2e_bytes(frac)
     e2e_val = world * wl.flops(frac) / (e2e_ms * 1e-3) / 1e12
     status = ctx.device_status()
+    samples = wl.samples
+    del wl
+    torch.cuda.empty_cache()
+
+    # ---- the BERT-base-shaped linears (M = 4096), measured the same way
+    bert = None
+    if not args.skip_extras:
+        wl2 = Workload(ctx, dev, I.config2(), FRACS)
+        b = measure(wl2, ctx, frac, max(args.steps, 50), max(args.warmup, 5), peaks, sync_all, max_over_ranks, world)
+        bert = {"workload": "configs[1]: BERT-base-shaped linears 768->2304, 768->768, 768->3072, 3072->768 at "
+                            "M=4096, bf16 activations, W8A8, CWPL",
+                "ms_per_step": b["ms_per_step"], "value": b["value"], "unit": "TFLOP/s", "bwd": b["bwd"],
+                "select_ms": b["select_ms"], "roofline": b["roofline"]}
+        status = status or ctx.device_status()
+        del wl2
+        torch.cuda.empty_cache()
+    all_clock.stop_flag = True
+    all_clock.join(timeout=2)
 
     # ---- the oracle on this machine's host cores (rank 0, single GPU only)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.skip_extras:
-        s, fl, names_c = oracle_step_seconds(frac)
+    if want_cpu:
+        s, fl = oracle_sample_seconds(samples, frac)
         cpu = {"value": fl / s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
-               "seconds": s, "sample": f"one full step of the workload ({', '.join(names_c)}), oracle fwd + EfQAT bwd "
-                                        f"in fp64 numpy, {int(frac * 100)}% unfrozen"}
+               "seconds": s, "sample": sample_text(samples, frac)}
 
     if rank == 0:
+        clocks = sampler.summary()
+        clocks["whole_run"] = all_clock.summary()
+        clocks["time_x_mhz"] = (head["ms_per_step"] * clocks["sm_mhz"]) if clocks["sm_mhz"] else None
         print(json.dumps({
-            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": head["value"], "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "configs[1]: BERT-base-shaped linears 768->2304, 768->768, 768->3072, 3072->768 "
-                                   "at M=4096, bf16 activations, W8A8, CWPL",
-                       "unfrozen": frac, "l2": "256 MiB buffer written between timed steps",
-                       "arithmetic": "forward: 8-bit codes on the integer tensor cores, int32 accumulate; "
-                                     "backward contractions: bf16 operands, fp32 accumulate",
-                       "optimizer": "fused SGD-momentum on the unfrozen rows (momentum 0.9, weight decay 1e-4, "
-                                    f"lr {SGD_LR:g} scaled for unit-variance synthetic dY)",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "clocks": sampler.summary(),
+            "config": workload_config(frac, world),
+            "clocks": clocks,
             "e2e": {"value": e2e_val, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": bi,
                     "d2h_bytes_per_step": bo},
-            "gpu_launches": int(launches),
-            "roofline": roofline,
+            "gpu_launches": head["launches"],
+            "roofline": head["roofline"],
             "cpu_baseline": cpu,
-            "bwd": bwd_report,
-            "select_ms": sel_ms,
+            "bwd": head["bwd"],
+            "select_ms": head["select_ms"],
+            "bert_base": bert,
             "device_status": status,
             "paper_context": "paper reports 1.44-1.64x backward speed-up on A10/A100 (whole network)",
         }))
@@ -416,16 +544,20 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--frac", type=float, default=0.05, choices=list(FRACS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-extras", action="store_true",
-                    help="only the headline timed steps and a 3-step end-to-end leg (short run for profilers)")
+                    help="only the headline timed steps and a 3-step end-to-end leg")
+    ap.add_argument("--capture", action="store_true",
+                    help="three steps of the first headline layer alone (small run for a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.capture:
+        run_capture(args)
     else:
         run_ours(args)
 

@@ -66,3 +66,19 @@ def test_backward_with_network_selected_counts(ctx, stack, li):
     assert (len(idx) == 0) == (li == 5)
     U.check_forward(ctx, case, T, D, s_w, s_x, z_x)
     U.check_backward(ctx, case, T, D, s_w, s_x, z_x, idx)
+
+
+@pytest.mark.parametrize("li", [0, 4, 5])
+def test_network_layer_shapes_at_full_token_count(ctx, stack, li):
+    """The three layer shapes of the stack (1024 -> 1024, 1024 -> 4096, 4096 -> 1024) at the full
+    M = 24 x 384 = 9216 tokens, W4A8, with the channel counts the network-wide ranking assigns."""
+    cases, Ws = stack
+    ref = O.select_cwpn([w.numpy() for w in Ws], 22118)
+    case = cases[li]
+    assert case.M == 9216
+    T = I.make_tensors(case)
+    T["W"] = Ws[li]
+    s_w, s_x, z_x = U.oracle_qparams(case, T, (0.8, 0.9, 0.6))
+    D = U.to_dev(T, s_w, s_x, z_x)
+    U.check_forward(ctx, case, T, D, s_w, s_x, z_x)
+    U.check_backward(ctx, case, T, D, s_w, s_x, z_x, ref[li])

@@ -34,28 +34,6 @@ CASES = [
 ]
 
 
-def _abs_bounds(case, T, s_w, s_x, z_x):
-    """Sum of |terms| of every output of the three contractions (same loops as the definition)."""
-    X64, W64, dY64 = (I.as_f64(T[k]) for k in ("X", "W", "dY"))
-    qx = O.fake_quant_x(X64, s_x, z_x, case.x_bits)
-    qw = O.fake_quant_w(W64, s_w, case.w_bits)
-    N, R, S, C = W64.shape
-    Bn, H, Wd, _ = X64.shape
-    Ho, Wo = dY64.shape[1:3]
-    pad = case.pad
-    P = O._patches(np.abs(qx["deq"]), R, S, 1, pad).reshape(-1, R * S * C)
-    Yabs = (P @ np.abs(qw["deq"]).reshape(N, -1).T).reshape(Bn, Ho, Wo, N)
-    dY2 = np.abs(dY64).reshape(-1, N)
-    Pc = O._patches(np.abs(qx["c0"]), R, S, 1, pad).reshape(-1, R * S * C)
-    Gw_abs = (float(s_x) * (dY2.T @ Pc)).reshape(N, R, S, C)
-    Gp = (dY2 @ np.abs(qw["deq"]).reshape(N, -1)).reshape(Bn, Ho, Wo, R, S, C)
-    Gxp = np.zeros((Bn, H + 2 * pad, Wd + 2 * pad, C))
-    for r in range(R):
-        for s in range(S):
-            Gxp[:, r:r + Ho, s:s + Wo, :] += Gp[:, :, :, r, s, :]
-    return Yabs, Gxp[:, pad:pad + H, pad:pad + Wd, :], Gw_abs
-
-
 @pytest.mark.parametrize("case", CASES, ids=lambda c: c.name)
 def test_conv_forward_backward_parity(ctx, case):
     T = I.make_tensors(case)
@@ -68,7 +46,7 @@ def test_conv_forward_backward_parity(ctx, case):
     D = U.to_dev(T, s_w, s_x, z_x)
     geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, 1, case.pad)
     is_bf16 = case.act_dtype == torch.bfloat16
-    Yabs, Gx_abs, Gw_abs = _abs_bounds(case, T, s_w, s_x, z_x)
+    Yabs, Gx_abs, Gw_abs = U.conv_abs_bounds(case, T, s_w, s_x, z_x)
 
     Y = B.fq_linear_fwd(ctx, D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"], case.w_bits, case.x_bits,
                         False, conv=geom)

@@ -24,9 +24,7 @@ import hashlib
 import json
 import os
 import re
-import statistics
 import sys
-import threading
 import time
 
 import numpy as np
@@ -36,6 +34,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from paper_2411_11038_b200 import inputs as I  # noqa: E402
+from paper_2411_11038_b200.clocks import ClockSampler, physical_gpu_index  # noqa: E402
 
 FRACS = (0.0, 0.05, 0.25, 1.0)
 METRIC = ("fq-linear backward TFLOP/s & speedup vs full-QAT bwd per unfrozen %; roofline frac "
@@ -89,62 +88,6 @@ def recorded_traffic():
     if h.group(1) != kernel_source_hash():
         return None, "kernel changed since the capture"
     return float(m.group(1)), TRAFFIC_FILE
-
-
-class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
-
-    def __init__(self, index: int, period_s: float = 0.002):
-        super().__init__(daemon=True)
-        self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
-        self.period_s = period_s
-        try:
-            import pynvml
-            pynvml.nvmlInit()
-            self.nv = pynvml
-            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
-            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
-        except Exception:
-            self.nv = None
-
-    def run(self):
-        if self.nv is None:
-            return
-        nv = self.nv
-        names = {
-            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
-            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
-            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
-            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
-        }
-        while not self.stop_flag:
-            try:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
-                try:
-                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
-                except Exception:
-                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
-                for bit, name in names.items():
-                    if r & bit:
-                        self.reasons.add(name)
-            except Exception:
-                pass
-            time.sleep(self.period_s)
-
-    def summary(self):
-        return dict(sm_mhz=(statistics.median(self.samples) if self.samples else None),
-                    sm_min_mhz=(min(self.samples) if self.samples else None),
-                    sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=len(self.samples))
-
-
-def physical_gpu_index(local_rank: int) -> int:
-    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
-    if vis:
-        try:
-            return int(vis.split(",")[local_rank])
-        except Exception:
-            return local_rank
-    return local_rank
 
 
 # ----------------------------------------------------------------------------------------
@@ -378,14 +321,14 @@ def measure(wl, ctx, frac, steps, warmup, peaks, sync_all, max_over_ranks, world
     mark = {}
 
     def start_counting():
-        mark["launches"] = B.launch_count()
+        mark["launches"] = ctx.launch_count()
         if sampler is not None:
             sampler.start()
 
     total_ms = timed(lambda: wl.step(frac), steps, warmup, wl.flush, sync_all, start_counting)
     if sampler is not None:
         sampler.stop_flag = True
-    launches = B.launch_count() - mark["launches"]
+    launches = ctx.launch_count() - mark["launches"]
     if sampler is not None:
         sampler.join(timeout=2)
     ms_per_step = max_over_ranks(total_ms) / steps

@@ -95,26 +95,15 @@ const char* efqat_status_string(int status);
  * stream work of interest was enqueued.  *code = 0 or an EFQAT_DEV_* value. */
 int efqat_device_status(efqat_ctx* ctx, int* code);
 
-/* ---- measurement aids --------------------------------------------------------- */
-/* Per-kernel timing for benchmarks.  While enabled, each of the three tensor-core
- * launches (which = 0 forward GEMM, 1 grad-input GEMM, 2 weight-gradient GEMM) is
- * bracketed by a pair of CUDA events on the caller's stream.  The events are created by
- * the enabling call (never on the hot path); at most 8192 launches per kind are kept
- * between two reads, later ones are not recorded. */
-int efqat_profile_enable(efqat_ctx* ctx, int enable);
-/* Synchronises the device, returns the summed duration (ms) and number of recorded
- * launches of kernel `which` since the previous read, and clears the record. */
-int efqat_profile_read(efqat_ctx* ctx, int which, float* ms_total, int* launches);
-/* Number of kernels the library has launched in this process. */
-int64_t efqat_launch_count(void);
-
 /* ---- host-only helpers ---------------------------------------------------------- */
 /* floor(ratio * n): number of unfrozen channels for ratio r (Eq. 7). */
 int64_t efqat_ratio_to_k(double ratio, int64_t n);
 /* Checks a layer description + quantizer spec exactly as the compute calls do. */
 int efqat_validate_layer(const efqat_layer_desc* layer, const efqat_qspec* q);
 /* Workspace bytes for efqat_fq_linear_fwd / _bwd on `layer` with at most k_sel_max
- * selected channels (pass N to cover full-QAT). */
+ * selected channels (pass N to cover full-QAT).  The size depends on the SM count of the
+ * GPU: the query reads it from the current CUDA device, which must be the device the
+ * compute calls will run on (they require their context's device to be current too). */
 int efqat_workspace_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, int64_t k_sel_max, size_t* out);
 /* Workspace bytes for efqat_select_channels over L layers with total_channels rows. */
 int efqat_select_workspace_bytes(int L, int64_t total_channels, size_t* out);
@@ -187,16 +176,19 @@ int efqat_init_weight_scales(efqat_ctx* ctx, const efqat_qspec* q, const float* 
  * out a fixed arena and forbids further allocation, a latency-critical loop that must not
  * enter the allocator, a process whose device memory pool belongs to another component.
  * The partial sums live in a 4 MiB device array built into the library (held on every
- * GPU that loads it, for the life of the process).  Needs no efqat_ctx.  The call
- * allocates nothing and frees nothing.
+ * GPU that loads it, for the life of the process).  Needs no efqat_ctx.  The call itself
+ * calls no allocating routine and frees nothing.
  *   dY: device, [M,N] row-major in `dtype` (EFQAT_F32 / EFQAT_BF16), 16-byte aligned;
  *   db: device, fp32 [N];  N % 8 == 0 and N <= 16384, else EFQAT_ERR_ALIGN /
  *   EFQAT_ERR_TOO_LARGE; the CUDA device owning dY must be current.
- * The first call on each device looks up the array's device address; make that call
- * before starting any stream capture.  All calls share the one array and it keeps what the
- * previous call left there (each call overwrites every element it reads, so nothing needs
- * clearing), hence two calls whose kernels may overlap on the GPU -- different streams
- * without ordering -- race with each other: serialise them. */
+ * The first call on each device is a warm-up: it looks up the array's device address, and
+ * under CUDA's lazy module loading the runtime may load this library's device code (the
+ * array included) at that moment, which takes device memory.  Make that first call before
+ * entering the region in which nothing may be allocated, and before starting any stream
+ * capture.  All calls share the one array and it keeps what the previous call left there
+ * (each call overwrites every element it reads, so nothing needs clearing), hence two calls
+ * whose kernels may overlap on the GPU -- different streams without ordering -- race with
+ * each other: serialise them. */
 int efqat_colsum_noalloc(int dtype, const void* dY, int64_t M, int64_t N, float* db, efqat_stream_t stream);
 
 /* ---- helper: the tensor-core contraction shared by a3, a4 and a6 (Eq. 5 shapes) -------- */

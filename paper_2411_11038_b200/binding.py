@@ -1,6 +1,6 @@
 """ctypes binding of libefqat.so: argument marshalling only.
 
-Function names mirror include/efqat.h.  Tensors are torch CUDA tensors used purely as
+Function names mirror include/efqat.h and include/efqat_aux.h.  Tensors are torch CUDA tensors used purely as
 device memory; every computation happens inside the library's kernels.  Importing this
 module does not load the library; the first call does, and fails loudly if the shared
 object has not been built (python -m paper_2411_11038_b200.build).
@@ -27,6 +27,7 @@ EXPORTS = [
     "efqat_fq_linear_bwd", "efqat_fake_quant_act", "efqat_fake_quant_weight",
     "efqat_init_act_qparams", "efqat_init_weight_scales", "efqat_gemm_bf16",
     "efqat_profile_enable", "efqat_profile_read", "efqat_launch_count", "efqat_colsum_noalloc",
+    "efqat_selftest_bounded_wait",
 ]
 
 
@@ -87,8 +88,9 @@ def load() -> C.CDLL:
     lib.efqat_profile_enable.argtypes = [vp, i32]
     lib.efqat_profile_read.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(i32)]
     lib.efqat_colsum_noalloc.argtypes = [i32, vp, i64, i64, vp, vp]
-    lib.efqat_launch_count.argtypes = []
+    lib.efqat_launch_count.argtypes = [vp]
     lib.efqat_launch_count.restype = i64
+    lib.efqat_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("efqat_status_string", "efqat_ratio_to_k", "efqat_launch_count"):
@@ -160,6 +162,15 @@ class Context:
         _check(load().efqat_profile_read(self.handle, int(which), C.byref(ms), C.byref(n)), "efqat_profile_read")
         return ms.value, n.value
 
+    def launch_count(self) -> int:
+        """Kernels launched through this context so far."""
+        return int(load().efqat_launch_count(self.handle))
+
+    def selftest_bounded_wait(self, limit_ns: int = 1_000_000):
+        """efqat_selftest_bounded_wait: a wait nobody satisfies; read the outcome with device_status()."""
+        _check(load().efqat_selftest_bounded_wait(self.handle, int(limit_ns), _stream()),
+               "efqat_selftest_bounded_wait")
+
     def close(self):
         if getattr(self, "handle", None):
             load().efqat_destroy(self.handle)
@@ -192,10 +203,6 @@ def layer_desc(M: int, N: int, K: int, act_dtype: int, conv: Optional[ConvGeom] 
         d.B, d.H, d.W, d.Cin, d.R, d.S, d.stride, d.pad = (conv.B, conv.H, conv.W, conv.Cin, conv.R, conv.S,
                                                          conv.stride, conv.pad)
     return d
-
-
-def launch_count() -> int:
-    return int(load().efqat_launch_count())
 
 
 def ratio_to_k(ratio: float, n: int) -> int:

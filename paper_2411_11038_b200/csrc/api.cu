@@ -1,10 +1,10 @@
 // C ABI of the library: argument validation, workspace carving and the launch sequence
 // of each entry point.  Every step of the path runs in this library's kernels; there is
 // no host fallback.
-#include <atomic>
 #include <new>
 #include <vector>
 
+#include "../../include/efqat_aux.h"
 #include "internal.h"
 
 using namespace efqat;
@@ -16,15 +16,26 @@ struct efqat_ctx {
   int device;
   int sm_count;
   int* d_status;
+  long long launches;     // kernels launched through this context
   int prof_on;
   std::vector<cudaEvent_t> ev[PROF_KINDS];   // start/stop pairs, created by efqat_profile_enable
   int ev_used[PROF_KINDS];
 };
 
-static std::atomic<long long> g_launches{0};
+// The context whose entry point is executing on this thread: launchers deep in the call tree
+// add to its counter without every signature carrying the context.
+static thread_local efqat_ctx* t_ctx = nullptr;
 namespace efqat {
-void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void count_launches(int n) {
+  if (t_ctx) t_ctx->launches += n;
+}
 }  // namespace efqat
+namespace {
+struct Entered {
+  explicit Entered(efqat_ctx* c) { t_ctx = c; }
+  ~Entered() { t_ctx = nullptr; }
+};
+}  // namespace
 
 namespace {
 
@@ -166,6 +177,7 @@ int efqat_create(efqat_ctx** out, int device) {
   if (!c) return EFQAT_ERR_CUDA;
   c->device = device;
   c->prof_on = 0;
+  c->launches = 0;
   for (int k = 0; k < PROF_KINDS; ++k) c->ev_used[k] = 0;
   int rc = EFQAT_OK;
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
@@ -213,6 +225,8 @@ const char* efqat_status_string(int s) {
 
 int efqat_device_status(efqat_ctx* ctx, int* code) {
   if (!ctx || !code) return EFQAT_ERR_NULL;
+  const int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
   if (cudaDeviceSynchronize() != cudaSuccess) return EFQAT_ERR_CUDA;
   if (cudaMemcpy(code, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EFQAT_ERR_CUDA;
   if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) return EFQAT_ERR_CUDA;
@@ -238,6 +252,8 @@ int efqat_profile_enable(efqat_ctx* ctx, int enable) {
 int efqat_profile_read(efqat_ctx* ctx, int which, float* ms_total, int* launches) {
   if (!ctx || !ms_total || !launches) return EFQAT_ERR_NULL;
   if (which < 0 || which >= PROF_KINDS) return EFQAT_ERR_MODE;
+  const int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
   if (cudaDeviceSynchronize() != cudaSuccess) return EFQAT_ERR_CUDA;
   double total = 0.0;
   for (int i = 0; i < ctx->ev_used[which]; ++i) {
@@ -252,7 +268,17 @@ int efqat_profile_read(efqat_ctx* ctx, int which, float* ms_total, int* launches
   return EFQAT_OK;
 }
 
-int64_t efqat_launch_count(void) { return static_cast<int64_t>(g_launches.load()); }
+int64_t efqat_launch_count(efqat_ctx* ctx) { return ctx ? static_cast<int64_t>(ctx->launches) : 0; }
+
+int efqat_selftest_bounded_wait(efqat_ctx* ctx, uint64_t limit_ns, efqat_stream_t stream) {
+  if (!ctx) return EFQAT_ERR_NULL;
+  if (limit_ns < 1000 || limit_ns > 1000000000ull) return EFQAT_ERR_SHAPE;    // 1 us .. 1 s
+  const int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
+  launch_wait_selftest(ctx->d_status, limit_ns, stream);
+  return last_error();
+}
 
 int64_t efqat_ratio_to_k(double ratio, int64_t n) {
   if (!(ratio > 0.0) || n <= 0) return 0;
@@ -268,9 +294,15 @@ int efqat_workspace_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, i
   if (rc != EFQAT_OK) return rc;
   if (k_sel_max < 0 || k_sel_max > layer->N) return EFQAT_ERR_K_RANGE;
   // the partial-product buffer is the only section that is not monotone in k_sel
-  // (fewer channels -> more splits of the contraction); take its maximum.  148 SMs
-  // is assumed when no context is at hand; a larger part would only lower the split count.
-  const int sm = 148;
+  // (fewer channels -> more splits of the contraction); take its maximum.  The split rule
+  // depends on the SM count: that of the current CUDA device, the one the compute calls
+  // require to be current as well (148, a B200, where no device can be asked).
+  int sm = 148, dev = -1, n = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 &&
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+    sm = n;
+  else
+    cudaGetLastError();
   int64_t p_max = 0;
   for (int64_t k = 1; k <= k_sel_max; ++k) {
     const int64_t nc = (k < layer->N) ? round_up(k, 16) : layer->N;
@@ -308,6 +340,7 @@ int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_des
     for (int l = 0; l < (mode == EFQAT_CWPL ? L : 1); ++l) want += k[l];
     if (want > 0) return EFQAT_ERR_NULL;
   }
+  Entered in(ctx);
   return run_select(mode, L, layers, weights, k, idx, offsets, importance_or_null, base, ws_bytes - slack,
                     ctx->d_status, stream);
 }
@@ -325,6 +358,7 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   if (rc != EFQAT_OK) return rc;
   const LayerWs w = carve(ws, layer, 0, ctx->sm_count, 0);
   if (ws_bytes < w.bytes) return EFQAT_ERR_WORKSPACE;
+  Entered in(ctx);
   const int64_t M = layer->M, N = layer->N, K = layer->K;
   cudaStream_t st = stream;
 
@@ -398,6 +432,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   if (rc != EFQAT_OK) return rc;
   const LayerWs w = carve(ws, layer, k_sel, ctx->sm_count, -1);
   if (ws_bytes < w.bytes) return EFQAT_ERR_WORKSPACE;
+  Entered in(ctx);
   cudaStream_t st = stream;
   const int act_bf16 = layer->act_dtype == EFQAT_BF16;
 
@@ -496,6 +531,7 @@ int efqat_gemm_bf16(efqat_ctx* ctx, const void* A, const void* B, int64_t M, int
   if (!aligned16(A) || !aligned16(B) || !aligned16(out)) return EFQAT_ERR_ALIGN;
   int rc = guard_device(ctx);
   if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
   GemmArgs g = {};
   g.A = static_cast<const bf16*>(A); g.B = static_cast<const bf16*>(B);
   g.Mr = M; g.Nc = N; g.Kc = K;
@@ -523,6 +559,7 @@ int efqat_fake_quant_act(efqat_ctx* ctx, const efqat_qspec* q, int dtype, const 
   if (count < 0) return EFQAT_ERR_SHAPE;
   rc = guard_device(ctx);
   if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
   ActQ* scratch = reinterpret_cast<ActQ*>(reinterpret_cast<char*>(ctx->d_status) + 128);
   launch_prep_act(s_x, z_x, q->x_bits, q->x_symmetric, scratch, ctx->d_status, stream);
   launch_quant_act_export(x, dtype, count, scratch, codes_or_null, clip_or_null, stream);
@@ -538,6 +575,7 @@ int efqat_fake_quant_weight(efqat_ctx* ctx, const efqat_qspec* q, const float* W
   if (N < 0 || K < 1) return EFQAT_ERR_SHAPE;
   rc = guard_device(ctx);
   if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
   launch_quant_weight_export(W, N, K, s_w, q->w_bits, codes_or_null, clip_or_null, ctx->d_status, stream);
   return last_error();
 }
@@ -552,6 +590,7 @@ int efqat_init_act_qparams(efqat_ctx* ctx, const efqat_qspec* q, int dtype, cons
   if (!ws || ws_bytes < 8192) return EFQAT_ERR_WORKSPACE;
   rc = guard_device(ctx);
   if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
   launch_minmax_act(x, dtype, count, q->x_bits, q->x_symmetric, s_x, z_x, static_cast<float*>(ws), stream);
   return last_error();
 }
@@ -564,6 +603,7 @@ int efqat_init_weight_scales(efqat_ctx* ctx, const efqat_qspec* q, const float* 
   if (N < 1 || K < 1) return EFQAT_ERR_SHAPE;
   rc = guard_device(ctx);
   if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
   launch_absmax_rows(W, N, K, q->w_bits, s_w, stream);
   return last_error();
 }

@@ -36,6 +36,7 @@ static const int GEMM_THREADS = 64 + 32 * EPI_WARPS;
 static const int ACC_STRIDE = 256;              // TMEM columns between the two accumulators
 static const int TMEM_COLS = 512;
 static const int HB_BYTES = 32 * 64;            // staging block of one epilogue warp: 32 rows x 64 B
+static const double L2_PANEL_BYTES = 32.0 * 1024 * 1024;   // operand slice kept resident in L2 by the tile order
 
 // Convolution geometry as the kernel needs it (mode 0 = plain matrices).
 struct ConvP {
@@ -63,6 +64,7 @@ struct GemmParams {
   int b_stage_bytes;
   int splits;
   int tiles_m, tiles_n;
+  int panel_dir, panel;   // order of the tiles in the work list (see tile_coords)
   int blk_cols;       // output columns per 64-byte staging row: 32 (bf16) or 16 (fp32)
   int out_bufs;       // staging buffers per epilogue warp (2 when shared memory allows)
   const float* col_scale;
@@ -83,9 +85,38 @@ struct __align__(16) SmemCtl {
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t xbar[EPI_WARPS];
+  uint64_t drain;           // abort path only: completion of the MMAs issued before the abort
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// Position (tm, tn) of tile t of the work list.  CTAs take consecutive tiles, so the tiles in
+// flight at one time are a run of the list; the order decides what that run shares in L2.
+//   panel_dir 0: row-major over (tm, tn): the run shares few A row blocks and sweeps all of B.
+//   panel_dir 1: the tile grid is cut into panels of `panel` tile columns; inside a panel the
+//                order is row-major, so the panel's slice of B stays in L2 while A streams past
+//                it once per panel.
+//   panel_dir 2: panels of `panel` tile rows, column-major inside: the mirror image.
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int t, int& tm, int& tn) {
+  if (p.panel_dir == 1) {
+    const int per = p.tiles_m * p.panel;
+    const int pn = t / per, r = t - pn * per;
+    const int first = pn * p.panel;
+    const int width = (p.tiles_n - first < p.panel) ? p.tiles_n - first : p.panel;
+    tm = r / width;
+    tn = first + (r - tm * width);
+  } else if (p.panel_dir == 2) {
+    const int per = p.tiles_n * p.panel;
+    const int pm = t / per, r = t - pm * per;
+    const int first = pm * p.panel;
+    const int height = (p.tiles_m - first < p.panel) ? p.tiles_m - first : p.panel;
+    tn = r / height;
+    tm = first + (r - tn * height);
+  } else {
+    tm = t / p.tiles_n;
+    tn = t - tm * p.tiles_n;
+  }
+}
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
@@ -134,6 +165,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_init(&ctl->acc_empty[b], (CTA2 ? 2 : 1) * EPI_WARPS);
     }
     for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&ctl->xbar[w], 1);
+    mbar_init(&ctl->drain, 1);
     ctl->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmA);
@@ -176,8 +208,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool live = true;
       for (int w = unit; w < total_items && live; w += num_units) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
-        const int m0 = (t / p.tiles_n) * TILE_M + rank * BM;
-        const int n0 = (t % p.tiles_n) * p.BN + rank * bn_cta;     // first B column staged by this CTA
+        int tm, tn;
+        tile_coords(p, t, tm, tn);
+        const int m0 = tm * TILE_M + rank * BM;
+        const int n0 = tn * p.BN + rank * bn_cta;     // first B column staged by this CTA
         int n_eff = static_cast<int>(p.Nc - n0);
         if (n_eff > bn_cta) n_eff = bn_cta;
         n_eff = (n_eff + 15) & ~15;
@@ -286,7 +320,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             } else {
               // forward / grad-input: tile rows = one box of 128 pixels; contraction block kb = (tap, 64 channels)
-              const int tmi = t / p.tiles_n;
+              const int tmi = tm;
               const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
               const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
               const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
@@ -322,7 +356,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool ok = true;
       for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
-        const int n0 = (t % p.tiles_n) * p.BN;
+        int tm, tn;
+        tile_coords(p, t, tm, tn);
+        const int n0 = tn * p.BN;
         int n_eff = static_cast<int>(p.Nc - n0);
         if (n_eff > p.BN) n_eff = p.BN;
         n_eff = (n_eff + 15) & ~15;
@@ -384,6 +420,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (CTA2) umma_commit_pair(&ctl->acc_full[buf], 3); else umma_commit(&ctl->acc_full[buf]);
         }
       }
+      if (!ok) {
+        // MMAs issued before the abort may still be reading the ring and writing TMEM: nothing
+        // of this CTA is torn down before they have completed (own barrier only, bounded)
+        if (CTA2) umma_commit_pair(&ctl->drain, 1); else umma_commit(&ctl->drain);
+        mbar_wait(&ctl->drain, 0, 20000000ull);
+      }
     }
   } else {
     // ------------------------------------------------------------- epilogue (warps 2..9)
@@ -413,8 +455,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       Geo g;
       g.split = w / tiles_mn;
       g.t = w - g.split * tiles_mn;
-      const int m0 = (g.t / p.tiles_n) * TILE_M + rank * BM;
-      g.n0 = (g.t % p.tiles_n) * p.BN;
+      int tm, tn;
+      tile_coords(p, g.t, tm, tn);
+      const int m0 = tm * TILE_M + rank * BM;
+      g.n0 = tn * p.BN;
       int n_eff = static_cast<int>(p.Nc - g.n0);
       if (n_eff > p.BN) n_eff = p.BN;
       g.n_eff = (n_eff + 15) & ~15;
@@ -428,7 +472,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       g.rows_live = g.row0 < p.Mr;
       if (EPI != EPI_PART && p.cv.mode != 0) {
         // convolution: this warp's 32 rows are a sub-box of the tile's pixel box
-        const int tmi = g.t / p.tiles_n;
+        const int tmi = tm;
         const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
         const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
         const int pix = q * 32;
@@ -439,8 +483,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       return g;
     };
+    int x_issued = 0;                        // X blocks requested so far (lane 0 only)
     auto fetch_x = [&](const Geo& g, int jb) {     // lane 0: one 32-row x 64-byte block of X
       uint64_t* xb = &ctl->xbar[e];
+      ++x_issued;
       mbar_arrive_expect_tx(xb, HB_BYTES);
       if (p.cv.mode != 0) tma_load_4d(my_x, &tmX, xb, g.n0 + jb * bc, g.pw0, g.ph0, g.pb0);
       else tma_load_2d(my_x, &tmX, xb, g.n0 + jb * bc, g.row0);
@@ -529,6 +575,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ++x_it;
 #pragma unroll
             for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const uint4*>(stg64_addr(my_x, lane, i));
+            // The next bulk copy overwrites this buffer through the async proxy.  Plain barriers do
+            // not order generic-proxy reads against it (the loads may legally be delayed up to
+            // their first use, far behind the copy's issue): the proxy fence does.
+            fence_proxy_async();
             __syncwarp();
             // the block now lives in registers: fetch the next one (of this or the next tile) behind the math
             if (lane == 0) {
@@ -678,6 +728,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       g = gn;
     }
+    // after an abort a requested X block may still be on its way into this warp's buffer
+    if (EPI == EPI_DX && !ok && lane == 0 && x_issued > x_it) mbar_wait(&ctl->xbar[e], x_it & 1, 20000000ull);
     if (EPI != EPI_PART && lane == 0) tma_store_wait_all();
   }
   tc_fence_before();
@@ -693,17 +745,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-static EncodeTiledFn g_encode = nullptr;
 
-int gemm_init() {
-  if (g_encode) return EFQAT_OK;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
-      qres != cudaDriverEntryPointSuccess)
-    return EFQAT_ERR_CUDA;
-  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  return EFQAT_OK;
+// The driver's tensor-map encoder, looked up once (a constant of the process, not state).
+static EncodeTiledFn tensor_map_encoder() {
+  static const EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess || !f ||
+        qres != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
 }
 
 // 2-D row-major matrix [rows, cols] with pitch ld (elements); box = row_bytes (128 or 64, the
@@ -717,7 +770,7 @@ static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows,
   const cuuint32_t estr[2] = {1u, 1u};
   const CUtensorMapDataType dt = (is_bf16 == 2) ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                  : (is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
-  const CUresult r = g_encode(m, dt, 2,
+  const CUresult r = tensor_map_encoder()(m, dt, 2,
                               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                               row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -736,7 +789,7 @@ static int make_map_4d(CUtensorMap* m, const void* base, int is_bf16, int64_t B,
   const cuuint32_t box[4] = {static_cast<cuuint32_t>(row_bytes / es), static_cast<cuuint32_t>(bw),
                              static_cast<cuuint32_t>(bh), static_cast<cuuint32_t>(bb)};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  const CUresult r = g_encode(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+  const CUresult r = tensor_map_encoder()(m, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
                               const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                               row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -820,15 +873,6 @@ template <int A_MN, int B_MN, int EPI, int CTA2>
 static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const CUtensorMap& tx,
                   const GemmParams& p, int grid, size_t smem, cudaStream_t st) {
   auto kern = gemm_kernel<A_MN, B_MN, EPI, CTA2>;
-  static bool configured[64] = {};   // per instantiation and device
-  int dev = 0;
-  cudaGetDevice(&dev);
-  if (dev < 0 || dev >= 64) return EFQAT_ERR_CUDA;
-  if (!configured[dev]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return EFQAT_ERR_CUDA;
-    configured[dev] = true;
-  }
   count_launches(1);
   if (launch_dependent(kern, static_cast<unsigned>(grid), GEMM_THREADS, smem, st, CTA2 ? 2 : 1, ta, tb, to, tx, p) !=
       cudaSuccess)
@@ -836,10 +880,28 @@ static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMa
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
+template <int A_MN, int B_MN, int EPI, int CTA2>
+static bool allow_full_smem() {
+  return cudaFuncSetAttribute(gemm_kernel<A_MN, B_MN, EPI, CTA2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              227 * 1024) == cudaSuccess;
+}
+
+// Per device, with that device current (efqat_create): every instantiation of the kernel may
+// use the whole shared memory of an SM.
+int gemm_init() {
+  if (!tensor_map_encoder()) return EFQAT_ERR_CUDA;
+  const bool ok = allow_full_smem<0, 0, EPI_FWD, 0>() && allow_full_smem<0, 0, EPI_FWD, 1>() &&
+                  allow_full_smem<0, 0, EPI_FWD_I8, 0>() && allow_full_smem<0, 0, EPI_FWD_I8, 1>() &&
+                  allow_full_smem<0, 1, EPI_DX, 0>() && allow_full_smem<0, 1, EPI_DX, 1>() &&
+                  allow_full_smem<1, 1, EPI_PART, 0>() && allow_full_smem<1, 1, EPI_PART, 1>() &&
+                  allow_full_smem<0, 0, EPI_PART, 0>() && allow_full_smem<0, 1, EPI_PART, 0>() &&
+                  allow_full_smem<1, 0, EPI_PART, 0>();
+  return ok ? EFQAT_OK : EFQAT_ERR_CUDA;
+}
+
 int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, int* grid_out) {
   if (a.Mr < 1 || a.Nc < 1 || a.Kc < 1) return EFQAT_ERR_SHAPE;
-  int rc = gemm_init();
-  if (rc != EFQAT_OK) return rc;
+  int rc = EFQAT_OK;
   GemmParams p = {};
   p.Mr = a.Mr;
   p.Nc = a.Nc;
@@ -910,6 +972,30 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     } else {
       p.tiles_m = c.tiles_w * c.tiles_h * tiles_b;             // one tile per box of 128 pixels
       p.nkb = cv->R * cv->S * c.cchunks;
+    }
+  }
+  // Order of the work list.  One tile reads tile_rows x Kc of A and BN x Kc of B.  With the
+  // plain row-major order the tiles in flight sweep every tile column, i.e. all of B, once per
+  // wave; when B is larger than what L2 keeps, each wave fetches it from DRAM again (measured
+  // on M = 16384, 8192 x 8192: 5.6 GB read for 0.67 GB of operands).  Panels sized to about
+  // L2_PANEL_BYTES keep one operand's slice resident while the other streams past it once per
+  // panel; the direction with the smaller estimated DRAM traffic wins, and plain order stays
+  // when a whole operand fits the panel budget anyway.
+  {
+    const double es = i8 ? 1.0 : 2.0;
+    const double kc_bytes = static_cast<double>(p.nkb) * p.bk * es / (p.splits > 0 ? p.splits : 1);
+    const double a_tile = static_cast<double>(pair ? 2 * BM : BM) * kc_bytes;
+    const double b_tile = static_cast<double>(p.BN) * kc_bytes;
+    const double a_all = a_tile * p.tiles_m, b_all = b_tile * p.tiles_n;
+    p.panel_dir = 0;
+    p.panel = 0;
+    if (b_all > L2_PANEL_BYTES && a_all > L2_PANEL_BYTES && p.tiles_m > 1 && p.tiles_n > 1) {
+      int gn = static_cast<int>(L2_PANEL_BYTES / b_tile), gm = static_cast<int>(L2_PANEL_BYTES / a_tile);
+      if (gn < 1) gn = 1;
+      if (gm < 1) gm = 1;
+      const double t_n = a_all * static_cast<double>(ceil_div(p.tiles_n, gn)) + b_all;   // column panels
+      const double t_m = b_all * static_cast<double>(ceil_div(p.tiles_m, gm)) + a_all;   // row panels
+      if (t_n <= t_m) { p.panel_dir = 1; p.panel = gn; } else { p.panel_dir = 2; p.panel = gm; }
     }
   }
   p.blk_cols = a.out_bf16 ? 32 : 16;

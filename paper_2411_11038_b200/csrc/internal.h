@@ -11,8 +11,11 @@ namespace efqat {
 
 typedef __nv_bfloat16 bf16;
 
-// Number of kernels this library has launched in this process (reported by efqat_launch_count).
+// Adds n to the launch counter of the context whose entry point is running on this thread
+// (reported by efqat_launch_count); a no-op outside an entry point that has a context.
 void count_launches(int n);
+// Bounded-wait self-test (selftest.cu): one mbarrier nobody arrives on, waited for limit_ns.
+void launch_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
 
 // Launch with programmatic stream serialization: the kernel may begin while the previous
 // launch of the stream drains; it must call pdl_wait() before reading or writing global memory.
@@ -44,24 +47,13 @@ inline cudaError_t launch_dependent(void (*kern)(KArgs...), unsigned grid, unsig
 // ---- elementwise.cu -----------------------------------------------------------------
 void launch_prep_act(const float* s_x, const float* z_x, int x_bits, int x_sym, ActQ* out, int* status,
                      cudaStream_t st);
-void launch_quant_act_operand(const void* X, int dtype, int64_t count, const ActQ* q, bf16* out, cudaStream_t st);
 void launch_quant_act_export(const void* X, int dtype, int64_t count, const ActQ* q, int32_t* codes,
                              uint8_t* clip, cudaStream_t st);
-// mode 0: integer codes q_w as bf16; mode 1: dequantised bf16(fl32(s_w*q_w)).
-void launch_quant_weight_operand(const float* W, int64_t N, int64_t K, const float* s_w, int w_bits, int mode,
-                                 bf16* out, int* status, cudaStream_t st);
 void launch_quant_weight_export(const float* W, int64_t N, int64_t K, const float* s_w, int w_bits,
                                 int32_t* codes, uint8_t* clip, int* status, cudaStream_t st);
-void launch_to_bf16(const float* in, int64_t count, bf16* out, cudaStream_t st);
-void launch_gather_cols(const void* dY, int dtype, int64_t M, int64_t N, const int32_t* idx, int64_t k_sel,
-                        int64_t pitch, bf16* out, int* status, cudaStream_t st);
 // ws: COLSUM_SLABS * N floats
 static const int COLSUM_SLABS = 64;
 void launch_colsum(const void* dY, int dtype, int64_t M, int64_t N, float* ws, float* db, cudaStream_t st);
-void launch_dx_finalize(const float* partials, int n, float* dS_x, float* dZ_x, cudaStream_t st);
-void launch_dw_finalize(const float* P, int splits, int64_t split_stride, int64_t k_sel, int64_t N, int64_t K,
-                        const float* W, const float* s_w, const int32_t* idx_or_null, const ActQ* xq, int w_bits,
-                        float* dW_sel, float* dS_w_sel, const efqat_sgd* opt, int* status, cudaStream_t st);
 void launch_minmax_act(const void* x, int dtype, int64_t count, int x_bits, int x_sym, float* s_x, float* z_x,
                        float* ws, cudaStream_t st);
 void launch_absmax_rows(const float* W, int64_t N, int64_t K, int w_bits, float* s_w, cudaStream_t st);
@@ -164,7 +156,9 @@ struct GemmArgs {
 int gemm_dx_num_partials(int64_t Mr, int64_t Nc);
 // Split count along the contraction for EPI_PART.
 int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count);
-int gemm_init();  // resolves the tensor-map encoder; returns an efqat_status
+// Once per device with that device current: resolves the tensor-map encoder and lets every
+// instantiation of the GEMM kernel use the full shared memory; returns an efqat_status.
+int gemm_init();
 void conv_pixel_box(int W, int H, int B, int target, int* tw, int* th, int* tb);
 // tiles_out (optional): number of output tiles = number of partial pairs EPI_DX wrote.
 // grid_out (optional): number of CTAs launched.

@@ -6,7 +6,9 @@ For every layer: forward ms, backward ms at each unfrozen fraction, algorithmic 
 (2MNK forward, 2MNK(1 + k/N) backward, Eq. 7-8 of the paper), the speed-up of the partial
 backward over this library's own full-QAT backward next to the ideal 2/(1+r), and the
 selection time.  Every number is the median over `iters` runs timed with CUDA events, with a
-256 MiB buffer written between runs so that nothing is served from a warm L2.
+256 MiB buffer written between runs so that nothing is served from a warm L2.  Each record
+carries the SM clock (median, minimum) and the clock-event reasons sampled through NVML while
+that record's measurements ran.
 """
 from __future__ import annotations
 
@@ -19,6 +21,7 @@ import torch
 
 from . import binding as B
 from . import inputs as I
+from .clocks import ClockSampler, physical_gpu_index
 
 FRACS = {1: (0.0, 26 / 512, 1.0), 2: (0.0, 0.05, 0.25, 1.0), 3: (0.0, 0.10, 1.0), 4: (0.0, 0.10, 1.0),
          5: (0.0, 0.01, 0.05, 0.10, 0.25, 0.50, 1.0)}
@@ -61,6 +64,23 @@ def layer_on_device(ctx, case: I.LayerCase, dev):
     return D, plan
 
 
+def clocked(fn):
+    """Runs a record-producing function with the clock sampler on and attaches its summary."""
+    def wrapper(*args, **kwargs):
+        sampler = ClockSampler(physical_gpu_index(0), period_s=0.005)
+        sampler.start()
+        try:
+            rec = fn(*args, **kwargs)
+        finally:
+            sampler.stop_flag = True
+            sampler.join(timeout=2)
+        for r in (rec if isinstance(rec, list) else [rec]):
+            r.setdefault("clocks", sampler.summary())
+        return rec
+    return wrapper
+
+
+@clocked
 def sweep_layer(ctx, case, fracs, timer, dev, ks=None):
     D, plan = layer_on_device(ctx, case, dev)
     g = 2.0 * case.M * case.N * case.K
@@ -86,6 +106,7 @@ def sweep_layer(ctx, case, fracs, timer, dev, ks=None):
     return rec
 
 
+@clocked
 def sweep_network(ctx, timer, dev):
     """Config 4: one global ranking over the 144 layers, then the per-layer steps with the
     counts that ranking assigns (the 4096->1024 layers end up fully frozen)."""
@@ -111,6 +132,7 @@ def sweep_network(ctx, timer, dev):
     return out
 
 
+@clocked
 def sweep_layerwise(ctx, timer, dev):
     """Layer-wise mode (LWPN) over the four W8A8 sweep shapes as one stack: the selection kernel
     ranks whole layers by mean |w| and unfreezes the top half; a frozen layer then runs the 0 %

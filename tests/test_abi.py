@@ -19,7 +19,8 @@ def lib():
 
 
 def test_exports_every_declared_symbol(lib):
-    header = open(os.path.join(ROOT, "include", "efqat.h")).read()
+    inc = os.path.join(ROOT, "include")
+    header = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     declared = set(re.findall(r"\b(efqat_[a-z0-9_]+)\s*\(", header))
     assert declared == set(B.EXPORTS)
     for name in declared:

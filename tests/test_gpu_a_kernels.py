@@ -203,3 +203,25 @@ def test_select_many_layers(ctx):
     _same_sets(got, O.select_cwpl([w.numpy() for w in Ws], ks))
     got, _, _ = B.select_channels(ctx, B.CWPN, [w.cuda() for w in Ws], [500])
     _same_sets(got, O.select_cwpn([w.numpy() for w in Ws], 500))
+
+
+def test_bounded_wait_runs_out_and_reports(ctx):
+    """A device-side wait that nothing satisfies gives up after its limit, the kernel returns,
+    the status word reads EFQAT_DEV_WAIT_TIMEOUT, and the context keeps working afterwards."""
+    import time
+    assert ctx.device_status() == 0
+    t0 = time.perf_counter()
+    ctx.selftest_bounded_wait(2_000_000)            # 2 ms
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0
+    assert ctx.device_status() == 3
+    assert B.status_string(3) == "device: bounded wait expired"
+    assert ctx.device_status() == 0                  # reading cleared it
+    W = torch.randn(64, 128, device="cuda")
+    s = B.init_weight_scales(ctx, W, 8)
+    torch.cuda.synchronize()
+    assert torch.equal(s, W.abs().amax(dim=1) / 127) or torch.allclose(s, W.abs().amax(dim=1) / 127, rtol=1e-6)
+    assert ctx.device_status() == 0
+    lib = B.load()
+    assert lib.efqat_selftest_bounded_wait(ctx.handle, 10, None) == -2       # limit outside 1 us .. 1 s
+    assert lib.efqat_selftest_bounded_wait(None, 1000000, None) == -1

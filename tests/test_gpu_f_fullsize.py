@@ -282,3 +282,35 @@ def test_config5_4096_dense_reductions(ctx):
         U.assert_fp32_class(out["dS_w_sel"].cpu().numpy(), bm["dS_w"][chan], bm["dS_w_abs"][chan], tag + " dS_w",
                             atol=1e-30)
         U.assert_fp32_class(_np(out["db"]), bm["db"], np.abs(dY64).sum(axis=0), tag + " db")
+
+
+@pytest.mark.parametrize("which", ["conv_28x28_3x3", "linear_4096x4096"])
+def test_backward_is_bit_reproducible_at_full_size(ctx, which):
+    """Thirty backward calls on the same inputs, with host-side pauses of varying length between
+    them so that the launches meet the GPU in different states: dX, dS_x, dZ_x, dW_sel and db
+    must come out bit-identical every time (every reduction has a fixed order, and nothing may
+    depend on timing)."""
+    import time
+    if which.startswith("conv"):
+        case = I.config3()[3]
+        geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, 1, case.pad)
+        frac = 0.10
+    else:
+        case, geom, frac = I.config5()[1], None, 0.05
+    T = I.make_tensors(case)
+    s_w, s_x, z_x = U.oracle_qparams(case, T, (0.6, 0.9, 0.3 if geom is None else 0.0))
+    D = U.to_dev(T, s_w, s_x, z_x)
+    k = B.ratio_to_k(frac, case.N)
+    sel, _, _ = B.select_channels(ctx, B.CWPL, [D["W"]], [k])
+    first = None
+    for it in range(30):
+        out = B.fq_linear_bwd(ctx, D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], sel[0], k, case.w_bits,
+                              case.x_bits, False, want_db=True, conv=geom)
+        torch.cuda.synchronize()
+        cur = {kk: v.clone() for kk, v in out.items()}
+        if first is None:
+            first = cur
+        for kk in first:
+            assert torch.equal(cur[kk], first[kk]), f"{case.name}: {kk} differs in repeat {it}"
+        time.sleep(0.002 * (it % 5))
+    assert ctx.device_status() == 0

@@ -49,6 +49,19 @@ def test_colsum_noalloc_matches_backward_db_twice(dtype):
     assert ctx.device_status() == 0
 
 
+@pytest.mark.parametrize("M,N", [(2304, 16384), (8, 16384), (8, 64)])
+def test_colsum_noalloc_at_the_ends_of_its_range(M, N):
+    """The widest matrix the built-in array holds (all 64 slabs of partial sums, up to the array's
+    last element) and matrices with fewer rows than one slab."""
+    g = torch.Generator().manual_seed(M * 31 + N)
+    dY = torch.randn((M, N), generator=g).to(torch.bfloat16).cuda()
+    for _ in range(2):
+        got = B.colsum_noalloc(dY).cpu().numpy()
+        ref = dY.double().sum(dim=0).cpu().numpy()
+        abs_sum = dY.double().abs().sum(dim=0).cpu().numpy()
+        assert np.all(np.abs(got - ref) <= 1e-5 * abs_sum)
+
+
 def test_colsum_noalloc_rejects_what_it_cannot_hold():
     lib = B.load()
     dY = torch.zeros((8, 16392), dtype=torch.float32).cuda()

@@ -15,7 +15,9 @@ Every function follows a passage of the EfQAT paper (arxiv 2411.11038):
   Eq. 6   block importance = mean |w| of the block
   Table 2 modes CWPL / CWPN / LWPN, all three using Top-K
   Algorithm 1  partial weight gradient on the unfrozen channels only
-  Section 4 "Setup"  straight-through estimator for the rounding, SGD momentum
+  Section 4 "Setup"  straight-through estimator for the rounding, SGD momentum,
+                     Adam for the quantization parameters
+  Appendix A.2  optional log2 parameterisation of the scales
 
 Readings of points the paper leaves open (rounding ties, how x/s is evaluated,
 gradient of the quantizer w.r.t. scale and zero point, tie-breaks in Top-K, the
@@ -332,6 +334,39 @@ def sgd_rows(W, V, dW_sel, idx, lr, momentum, weight_decay):
         V2[n] = momentum * V2[n] + g
         W2[n] = W2[n] - lr * V2[n]
     return W2, V2
+
+
+def adam_qparams(p, m, v, grad, idx, step, lr, beta1=0.9, beta2=0.999, eps=1e-8,
+                 theta=None):
+    """Adam step (Kingma & Ba, as cited in Section 4 "Setup" for the quantization
+    parameters) on the entries idx of the parameter vector p with the compact
+    gradient grad[i] = dL/dp[idx[i]]; entries outside idx and their moments are
+    returned untouched (a frozen channel's scale is not updated, Algorithm 1).
+
+        m <- b1 m + (1-b1) g      v <- b2 v + (1-b2) g^2
+        p <- p - lr (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps),   t = step >= 1
+
+    theta given (Appendix A.2, scales only): the optimised variable is
+    theta = log2(p); its gradient is dL/dp * p * ln 2 by the chain rule through
+    p = 2^theta, the same step is taken on theta and p <- 2^theta.  Zero points
+    are always trained raw.  Returns new (p, m, v) or (p, m, v, theta).  fp64."""
+    p2, m2, v2 = (np.array(a, dtype=F64).reshape(-1) for a in (p, m, v))
+    th2 = None if theta is None else np.array(theta, dtype=F64).reshape(-1)
+    g = np.asarray(grad, dtype=F64).reshape(-1)
+    idx = np.arange(p2.size) if idx is None else np.asarray(idx, dtype=np.int64)
+    bc1 = 1.0 - beta1 ** step
+    bc2 = 1.0 - beta2 ** step
+    for i, n in enumerate(idx):
+        gi = g[i] if th2 is None else g[i] * p2[n] * np.log(2.0)
+        m2[n] = beta1 * m2[n] + (1.0 - beta1) * gi
+        v2[n] = beta2 * v2[n] + (1.0 - beta2) * gi * gi
+        upd = lr * (m2[n] / bc1) / (np.sqrt(v2[n] / bc2) + eps)
+        if th2 is None:
+            p2[n] = p2[n] - upd
+        else:
+            th2[n] = th2[n] - upd
+            p2[n] = 2.0 ** th2[n]
+    return (p2, m2, v2) if th2 is None else (p2, m2, v2, th2)
 
 
 # ----------------------------------------------------------------------------

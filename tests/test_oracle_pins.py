@@ -457,6 +457,48 @@ def test_sgd_rows_against_torch_sgd():
     np.testing.assert_allclose(W2[idx], p.detach().numpy(), rtol=1e-14)
 
 
+def test_adam_qparams_against_torch_adam():
+    """Three Adam steps on a subset of entries equal torch.optim.Adam on those entries alone;
+    the other entries and their moments never move.  With the log2 parameterisation the same
+    holds for theta with the gradient that autograd sends through p = 2^theta."""
+    r = rng(51)
+    p0 = r.random(9) * 0.05 + 0.01
+    idx = [0, 3, 4, 8]
+    frozen = [1, 2, 5, 6, 7]
+    grads = [r.standard_normal(4) * 10 ** r.uniform(-3, 2) for _ in range(3)]
+    kw = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    # raw parameters
+    p, m, v = p0.copy(), np.zeros(9), np.zeros(9)
+    tp = torch.tensor(p0[idx], dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([tp], lr=1e-3, betas=(0.9, 0.999), eps=1e-8)
+    for t, g in enumerate(grads, 1):
+        p, m, v = O.adam_qparams(p, m, v, g, idx, t, **kw)
+        tp.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(p[idx], tp.detach().numpy(), rtol=1e-12)
+        np.testing.assert_allclose(m[idx], opt.state[tp]["exp_avg"].numpy(), rtol=1e-12)
+        np.testing.assert_allclose(v[idx], opt.state[tp]["exp_avg_sq"].numpy(), rtol=1e-12)
+        assert np.array_equal(p[frozen], p0[frozen]) and not m[frozen].any() and not v[frozen].any()
+    # first step by hand: m^ = g, v^ = g^2, so the step is lr * sign(g) up to eps
+    p1, _, _ = O.adam_qparams(p0, np.zeros(9), np.zeros(9), grads[0], idx, 1, **kw)
+    np.testing.assert_allclose(p1[idx], p0[idx] - 1e-3 * grads[0] / (np.abs(grads[0]) + 1e-8), rtol=1e-12)
+    # log2 parameterisation: torch differentiates through p = 2^theta
+    p, m, v, th = p0.copy(), np.zeros(9), np.zeros(9), np.log2(p0)
+    tth = torch.tensor(np.log2(p0[idx]), dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([tth], lr=1e-3, betas=(0.9, 0.999), eps=1e-8)
+    for t, g in enumerate(grads, 1):
+        p, m, v, th = O.adam_qparams(p, m, v, g, idx, t, theta=th, **kw)
+        opt.zero_grad()
+        (torch.pow(2.0, tth) * torch.tensor(g, dtype=torch.float64)).sum().backward()     # dL/dp = g
+        opt.step()
+        np.testing.assert_allclose(th[idx], tth.detach().numpy(), rtol=1e-12)
+        np.testing.assert_allclose(p[idx], 2.0 ** tth.detach().numpy(), rtol=1e-12)
+        assert np.array_equal(p[frozen], p0[frozen]) and np.all(p > 0)
+    # scalar form (activation scale / zero point): idx = None updates every entry
+    q, mq, vq = O.adam_qparams([0.02], [0.0], [0.0], [3.0], None, 1, **kw)
+    np.testing.assert_allclose(q, [0.02 - 1e-3 * 3.0 / (3.0 + 1e-8)], rtol=1e-12)
+
+
 # ---------------------------------------------------------------------------
 # convolution
 # ---------------------------------------------------------------------------

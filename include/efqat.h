@@ -150,6 +150,40 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
                         float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null, void* ws,
                         size_t ws_bytes, efqat_stream_t stream);
 
+/* ---- optimizer step of the quantization parameters (Section 4 "Setup": Adam for the
+ * quantization parameters; Algorithm 1: "update the unfrozen weight channels and their
+ * scales", "update the scales and zero points of the activations"; Appendix A.2: optional
+ * log2 parameterisation of the scales) --------------------------------------------------- */
+/* Adam:  m <- beta1 m + (1-beta1) g;  v <- beta2 v + (1-beta2) g^2;
+ *        p <- p - lr (m / (1-beta1^step)) / (sqrt(v / (1-beta2^step)) + eps),  step >= 1.
+ * log2_scale != 0: for the scales the optimised variable is theta = log2(s), with gradient
+ * g * s * ln 2, and s <- 2^theta afterwards; the zero point is always trained raw. */
+typedef struct {
+  float lr, beta1, beta2, eps;
+  int64_t step;
+  int log2_scale;
+} efqat_adam;
+/* Parameters and optimizer state of one layer (device, fp32, caller-owned).  s_w, m_sw, v_sw,
+ * theta_sw: [N] (theta_sw only used, and required, in log2 mode: initialise it with
+ * efqat_log2_scale_init).  s_x, z_x: [1].  state_x: [8] = first and second moment of s_x,
+ * first and second moment of z_x, theta of s_x, three unused; zero it before the first step
+ * (and set element 4 with efqat_log2_scale_init in log2 mode). */
+typedef struct {
+  float* s_w; float* m_sw; float* v_sw; float* theta_sw;
+  float* s_x; float* z_x; float* state_x;
+} efqat_qparam_state;
+/* One launch: the weight scales of the channels idx[0..k_sel) (idx may be NULL when
+ * k_sel == N; scales and moments of the other channels are not touched) from the compact
+ * gradient dS_w_sel [k_sel], the activation scale from dS_x [1], and the activation zero
+ * point from dZ_x [1] (dZ_x NULL, e.g. for the symmetric quantizer: zero point left alone).
+ * The gradients are the outputs of efqat_fq_linear_bwd.  A raw scale that the step drives
+ * to zero or below is reported as EFQAT_DEV_BAD_SCALE by the next forward / backward. */
+int efqat_qparam_adam(efqat_ctx* ctx, const efqat_adam* opt, const efqat_qparam_state* state, int64_t N,
+                      const int32_t* idx, int64_t k_sel, const float* dS_w_sel, const float* dS_x,
+                      const float* dZ_x, efqat_stream_t stream);
+/* theta[i] = log2(s[i]) for i < n (Appendix A.2). */
+int efqat_log2_scale_init(efqat_ctx* ctx, const float* s, float* theta, int64_t n, efqat_stream_t stream);
+
 /* ---- helpers: quantizer export and MinMax initialisation ---------------------------- */
 /* Eq. 1: codes int32 [count] (asymmetric: 0..2^b-1; symmetric: signed), clip uint8 [count]
  * (0 in range, 1 clipped low, 2 clipped high), either may be NULL.  x in `dtype`. */

@@ -27,7 +27,7 @@ EXPORTS = [
     "efqat_fq_linear_bwd", "efqat_fake_quant_act", "efqat_fake_quant_weight",
     "efqat_init_act_qparams", "efqat_init_weight_scales", "efqat_gemm_bf16",
     "efqat_profile_enable", "efqat_profile_read", "efqat_launch_count", "efqat_colsum_noalloc",
-    "efqat_selftest_bounded_wait",
+    "efqat_selftest_bounded_wait", "efqat_qparam_adam", "efqat_log2_scale_init",
 ]
 
 
@@ -44,6 +44,16 @@ class LayerDesc(C.Structure):
 class Sgd(C.Structure):
     _fields_ = [("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
                 ("W_inout", C.c_void_p), ("mom_inout", C.c_void_p)]
+
+
+class Adam(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("step", C.c_int64), ("log2_scale", C.c_int)]
+
+
+class QParamState(C.Structure):
+    _fields_ = [("s_w", C.c_void_p), ("m_sw", C.c_void_p), ("v_sw", C.c_void_p), ("theta_sw", C.c_void_p),
+                ("s_x", C.c_void_p), ("z_x", C.c_void_p), ("state_x", C.c_void_p)]
 
 
 class EfqatError(RuntimeError):
@@ -91,6 +101,8 @@ def load() -> C.CDLL:
     lib.efqat_launch_count.argtypes = [vp]
     lib.efqat_launch_count.restype = i64
     lib.efqat_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
+    lib.efqat_qparam_adam.argtypes = [vp, C.POINTER(Adam), C.POINTER(QParamState), i64, vp, i64, vp, vp, vp, vp]
+    lib.efqat_log2_scale_init.argtypes = [vp, vp, vp, i64, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("efqat_status_string", "efqat_ratio_to_k", "efqat_launch_count"):
@@ -354,6 +366,36 @@ def make_sgd(lr: float, momentum: float, weight_decay: float, W: torch.Tensor, m
 
 
 # ---------------------------------------------------------------------------------------
+class QParamOptimizer:
+    """efqat_qparam_adam for one layer: owns the Adam moments (and theta = log2 s in log2 mode) of
+    the layer's weight scales, activation scale and activation zero point."""
+
+    def __init__(self, ctx: Context, s_w, s_x, z_x, lr: float, beta1=0.9, beta2=0.999, eps=1e-8,
+                 log2_scale: bool = False):
+        self.ctx, self.s_w, self.s_x, self.z_x = ctx, _dev(s_w), _dev(s_x), z_x
+        self.N = int(s_w.numel())
+        dev = s_w.device
+        self.m_sw = torch.zeros(self.N, dtype=torch.float32, device=dev)
+        self.v_sw = torch.zeros(self.N, dtype=torch.float32, device=dev)
+        self.theta_sw = torch.zeros(self.N, dtype=torch.float32, device=dev) if log2_scale else None
+        self.state_x = torch.zeros(8, dtype=torch.float32, device=dev)
+        self.opt = Adam(lr, beta1, beta2, eps, 0, 1 if log2_scale else 0)
+        if log2_scale:
+            lib = load()
+            _check(lib.efqat_log2_scale_init(ctx.handle, _ptr(s_w), _ptr(self.theta_sw), self.N, _stream()),
+                   "efqat_log2_scale_init")
+            _check(lib.efqat_log2_scale_init(ctx.handle, _ptr(s_x), C.c_void_p(self.state_x.data_ptr() + 16), 1,
+                                             _stream()), "efqat_log2_scale_init")
+        self.state = QParamState(_ptr(s_w), _ptr(self.m_sw), _ptr(self.v_sw), _ptr(self.theta_sw), _ptr(s_x),
+                                 _ptr(z_x), _ptr(self.state_x))
+
+    def step(self, idx, k_sel: int, dS_w_sel, dS_x, dZ_x=None):
+        self.opt.step += 1
+        rc = load().efqat_qparam_adam(self.ctx.handle, C.byref(self.opt), C.byref(self.state), self.N, _ptr(idx),
+                                      int(k_sel), _ptr(dS_w_sel), _ptr(dS_x), _ptr(dZ_x), _stream())
+        _check(rc, "efqat_qparam_adam")
+
+
 def fake_quant_act(ctx: Context, x, s_x, z_x, x_bits=8, x_symmetric=False):
     """efqat_fake_quant_act: returns (codes int32, clip uint8) shaped like x."""
     _dev(x)

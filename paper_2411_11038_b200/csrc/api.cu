@@ -548,6 +548,36 @@ int efqat_gemm_bf16(efqat_ctx* ctx, const void* A, const void* B, int64_t M, int
   return last_error();
 }
 
+int efqat_qparam_adam(efqat_ctx* ctx, const efqat_adam* opt, const efqat_qparam_state* state, int64_t N,
+                      const int32_t* idx, int64_t k_sel, const float* dS_w_sel, const float* dS_x,
+                      const float* dZ_x, efqat_stream_t stream) {
+  if (!ctx || !opt || !state || !dS_x || !state->s_x || !state->state_x) return EFQAT_ERR_NULL;
+  if (N < 1) return EFQAT_ERR_SHAPE;
+  if (k_sel < 0 || k_sel > N) return EFQAT_ERR_K_RANGE;
+  if (k_sel > 0 && (!dS_w_sel || !state->s_w || !state->m_sw || !state->v_sw)) return EFQAT_ERR_NULL;
+  if (k_sel > 0 && k_sel < N && !idx) return EFQAT_ERR_NULL;
+  if (opt->log2_scale && k_sel > 0 && !state->theta_sw) return EFQAT_ERR_NULL;
+  if (dZ_x && !state->z_x) return EFQAT_ERR_NULL;
+  if (opt->step < 1 || !(opt->beta1 >= 0.f && opt->beta1 < 1.f) || !(opt->beta2 >= 0.f && opt->beta2 < 1.f) ||
+      !(opt->eps > 0.f))
+    return EFQAT_ERR_SHAPE;
+  const int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
+  launch_qparam_adam(*opt, *state, N, (k_sel < N) ? idx : nullptr, k_sel, dS_w_sel, dS_x, dZ_x, ctx->d_status, stream);
+  return last_error();
+}
+
+int efqat_log2_scale_init(efqat_ctx* ctx, const float* s, float* theta, int64_t n, efqat_stream_t stream) {
+  if (!ctx || !s || !theta) return EFQAT_ERR_NULL;
+  if (n < 1) return EFQAT_ERR_SHAPE;
+  const int rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  Entered in(ctx);
+  launch_log2_init(s, theta, n, ctx->d_status, stream);
+  return last_error();
+}
+
 int efqat_fake_quant_act(efqat_ctx* ctx, const efqat_qspec* q, int dtype, const void* x, int64_t count,
                          const float* s_x, const float* z_x, int32_t* codes_or_null, uint8_t* clip_or_null,
                          efqat_stream_t stream) {

@@ -93,6 +93,12 @@ struct FinArgs {
 };
 void launch_finalize(FinArgs a, cudaStream_t st);
 
+// ---- optim.cu -----------------------------------------------------------------------
+void launch_qparam_adam(const efqat_adam& a, const efqat_qparam_state& st, int64_t N, const int32_t* idx,
+                        int64_t k_sel, const float* dS_w_sel, const float* dS_x, const float* dZ_x, int* status,
+                        cudaStream_t stream);
+void launch_log2_init(const float* s, float* theta, int64_t n, int* status, cudaStream_t stream);
+
 // ---- select.cu ----------------------------------------------------------------------
 size_t select_workspace_bytes(int L, int64_t total_channels);
 int run_select(int mode, int L, const efqat_layer_desc* layers, const float* const* weights, const int64_t* k,

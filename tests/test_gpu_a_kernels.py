@@ -7,6 +7,8 @@ import torch
 
 from oracle import efqat_oracle as O
 from paper_2411_11038_b200 import binding as B
+from paper_2411_11038_b200 import inputs as I
+from tests import parity_util as U
 
 pytestmark = pytest.mark.gpu
 
@@ -225,3 +227,87 @@ def test_bounded_wait_runs_out_and_reports(ctx):
     lib = B.load()
     assert lib.efqat_selftest_bounded_wait(ctx.handle, 10, None) == -2       # limit outside 1 us .. 1 s
     assert lib.efqat_selftest_bounded_wait(None, 1000000, None) == -1
+
+
+@pytest.mark.parametrize("log2_scale", [False, True])
+def test_qparam_adam_matches_oracle(ctx, log2_scale):
+    """Three fused Adam steps on the weight scales of the selected channels, the activation scale
+    and the zero point (raw and with theta = log2 s) against the fp64 oracle; the scales and
+    moments of the frozen channels stay bit-identical."""
+    r = np.random.default_rng(61 + int(log2_scale))
+    N = 777
+    idx = np.sort(r.choice(N, 123, replace=False)).astype(np.int32)
+    frozen = np.setdiff1d(np.arange(N), idx)
+    s_w0 = (r.random(N) * 0.05 + 0.002).astype(np.float32)
+    s_x0, z_x0 = np.float32(0.0173), np.float32(117.3)
+    s_w = torch.from_numpy(s_w0.copy()).cuda()
+    s_x = torch.tensor([float(s_x0)], device="cuda")
+    z_x = torch.tensor([float(z_x0)], device="cuda")
+    lr = 1e-3
+    opt = B.QParamOptimizer(ctx, s_w, s_x, z_x, lr, log2_scale=log2_scale)
+    # the ABI carries the hyper-parameters as fp32: the oracle gets the same (rounded) values
+    hp = dict(lr=float(np.float32(lr)), beta1=float(np.float32(0.9)), beta2=float(np.float32(0.999)),
+              eps=float(np.float32(1e-8)))
+    # oracle state
+    pw, mw, vw = s_w0.astype(np.float64), np.zeros(N), np.zeros(N)
+    px, mx, vx = np.array([s_x0], np.float64), np.zeros(1), np.zeros(1)
+    pz, mz, vz = np.array([z_x0], np.float64), np.zeros(1), np.zeros(1)
+    thw, thx = (np.log2(pw), np.log2(px)) if log2_scale else (None, None)
+    idx_dev = torch.from_numpy(idx).cuda()
+    for t in range(1, 4):
+        gw = (r.standard_normal(len(idx)) * 10.0 ** r.uniform(-3, 3, len(idx))).astype(np.float32)
+        gx, gz = np.float32(r.standard_normal() * 50), np.float32(r.standard_normal() * 0.01)
+        opt.step(idx_dev, len(idx), torch.from_numpy(gw).cuda(), torch.tensor([float(gx)], device="cuda"),
+                 torch.tensor([float(gz)], device="cuda"))
+        if log2_scale:
+            pw, mw, vw, thw = O.adam_qparams(pw, mw, vw, gw, idx, t, theta=thw, **hp)
+            px, mx, vx, thx = O.adam_qparams(px, mx, vx, [gx], None, t, theta=thx, **hp)
+        else:
+            pw, mw, vw = O.adam_qparams(pw, mw, vw, gw, idx, t, **hp)
+            px, mx, vx = O.adam_qparams(px, mx, vx, [gx], None, t, **hp)
+        pz, mz, vz = O.adam_qparams(pz, mz, vz, [gz], None, t, **hp)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(s_w.cpu().numpy(), pw, rtol=1e-5)
+        np.testing.assert_allclose(opt.m_sw.cpu().numpy(), mw, rtol=1e-5, atol=1e-30)
+        np.testing.assert_allclose(opt.v_sw.cpu().numpy(), vw, rtol=1e-5, atol=1e-30)
+        np.testing.assert_allclose(s_x.item(), px[0], rtol=1e-5)
+        np.testing.assert_allclose(z_x.item(), pz[0], rtol=1e-6)
+        if log2_scale:
+            np.testing.assert_allclose(opt.theta_sw.cpu().numpy()[idx], thw[idx], rtol=1e-5)
+        assert np.array_equal(s_w.cpu().numpy()[frozen], s_w0[frozen])
+        assert not opt.m_sw.cpu().numpy()[frozen].any() and not opt.v_sw.cpu().numpy()[frozen].any()
+    assert ctx.device_status() == 0
+    # every selected scale moved, by about lr per step in the first steps (Adam's normalised update)
+    moved = np.abs(s_w.cpu().numpy()[idx] - s_w0[idx])
+    assert np.all(moved > 0)
+    lib = B.load()
+    import ctypes as C
+    bad = B.Adam(lr, 0.9, 0.999, 1e-8, 0, 0)             # step must be >= 1
+    assert lib.efqat_qparam_adam(ctx.handle, C.byref(bad), C.byref(opt.state), N, None, 0, None,
+                                 C.c_void_p(s_x.data_ptr()), None, None) == -2
+
+
+def test_backward_then_qparam_adam_end_to_end(ctx):
+    """Gradients straight from efqat_fq_linear_bwd into efqat_qparam_adam on the device, against
+    the oracle's backward followed by the oracle's Adam step."""
+    case = I.LayerCase("adam_e2e", 192, 128, 96, act_dtype=torch.float32, seed=77)
+    T = I.make_tensors(case)
+    s_w, s_x, z_x = U.oracle_qparams(case, T, (0.8, 0.85, 0.4))
+    D = U.to_dev(T, s_w, s_x, z_x)
+    idx = O.select_cwpl([T["W"].numpy()], [12])[0]
+    idx_dev = torch.from_numpy(idx).cuda()
+    out = B.fq_linear_bwd(ctx, D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx_dev, 12, 8, 8, False)
+    opt = B.QParamOptimizer(ctx, D["s_w"], D["s_x"], D["z_x"], 1e-4)
+    opt.step(idx_dev, 12, out["dS_w_sel"], out["dS_x"], out["dZ_x"])
+    torch.cuda.synchronize()
+    ref = O.backward_efqat(I.as_f64(T["dY"]), I.as_f64(T["X"]), I.as_f64(T["W"]), s_w, s_x, z_x, idx, 8, 8,
+                           operand_model="bf16")
+    hp = dict(lr=float(np.float32(1e-4)), beta1=float(np.float32(0.9)), beta2=float(np.float32(0.999)),
+              eps=float(np.float32(1e-8)))
+    pw, _, _ = O.adam_qparams(s_w, np.zeros(96), np.zeros(96), ref["dS_w_sel"], idx, 1, **hp)
+    px, _, _ = O.adam_qparams([s_x], [0.0], [0.0], [ref["dS_x"]], None, 1, **hp)
+    pz, _, _ = O.adam_qparams([z_x], [0.0], [0.0], [ref["dZ_x"]], None, 1, **hp)
+    np.testing.assert_allclose(D["s_w"].cpu().numpy(), pw, rtol=1e-5)
+    np.testing.assert_allclose(D["s_x"].item(), px[0], rtol=1e-5)
+    np.testing.assert_allclose(D["z_x"].item(), pz[0], rtol=1e-6)
+    assert ctx.device_status() == 0

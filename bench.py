@@ -387,6 +387,98 @@ def measure(wl, ctx, frac, steps, warmup, peaks, sync_all, max_over_ranks, world
                 select_ms=sel_ms)
 
 
+def measure_network(ctx, dev, sync_all, max_over_ranks):
+    """The BERT-large-shaped stack (configs[3]): 144 quantized linears at M = 9216 tokens, W4A8,
+    chained on one stream through efqat_network_fwd / _bwd with a weight-operand cache per layer,
+    network-wide (CWPN) and layer-wise (LWPN) selection, and the freezing frequency f of
+    Section 3.2.  Reported: ms per network backward per unfrozen ratio, the selection cost and
+    its share when amortised over f samples, cached against uncached calls."""
+    import math
+    from paper_2411_11038_b200 import binding as B
+    from paper_2411_11038_b200 import network as NW
+    cases = I.config4()
+    batch = 24                                       # sequences of 384 tokens per step
+    pools = {}
+
+    def pool(width, count, seed):
+        if width not in pools:
+            g = torch.Generator().manual_seed(seed)
+            pools[width] = [torch.randn((cases[0].M, width), generator=g).to(torch.bfloat16).to(dev)
+                            for _ in range(count)]
+        return pools[width]
+
+    p1, p4 = pool(1024, 8, 4901), pool(4096, 4, 4902)     # 151 MB each: rotating through them defeats L2
+    states = []
+    for i, c in enumerate(cases):
+        g = torch.Generator().manual_seed(c.seed)
+        W = (torch.randn((c.N, c.K), generator=g) * math.sqrt(2.0 / c.K)).to(dev)
+        X = (p1 if c.K == 1024 else p4)[i % (8 if c.K == 1024 else 4)]
+        dY = (p1 if c.N == 1024 else p4)[(i + 3) % (8 if c.N == 1024 else 4)]
+        states.append(NW.LayerState(c, W, X, dY, None))
+    total = sum(c.N for c in cases)
+    net = NW.EfqatNetwork(ctx, states, B.CWPN, B.ratio_to_k(0.1, total), f_samples=batch, batch_samples=batch,
+                          use_cache=True, sgd=(SGD_LR, 0.9, 1e-4), adam=dict(lr=1e-6))
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    gemm = sum(2.0 * c.M * c.N * c.K for c in cases)
+
+    def t(fn, steps=10, warm=3):
+        return max_over_ranks(timed(fn, steps, warm, flush, sync_all) / steps)
+
+    out = {"workload": "configs[3]: BERT-large-shaped stack, 24 blocks x (4 x 1024->1024, 1024->4096, 4096->1024) = "
+                       "144 layers, M=9216 tokens, W4A8, bf16 activations, inputs rotate through pools larger than L2",
+           "layers": len(cases), "channels": total, "samples_per_step": batch}
+    rows = {}
+    for mode, name, ratios in ((B.CWPN, "CWPN", (0.0, 0.05, 0.10, 0.25, 1.0)), (B.LWPN, "LWPN", (0.05, 0.10, 0.25))):
+        for r in ratios:
+            budget = B.ratio_to_k(r, total) if mode == B.CWPN else int(r * len(cases))
+            net.use_selection(mode, budget)
+            net.reselect()
+            ks = net.counts()
+            fl = sum(2.0 * c.M * c.K * (c.N + k) for c, k in zip(cases, ks))
+            ms = t(net.backward)
+            rows[f"{name} {int(round(r * 100))}%"] = {
+                "bwd_ms": ms, "tflops": fl / (ms * 1e-3) / 1e12, "unfrozen_channels": int(sum(ks)),
+                "layers_with_unfrozen_channels": int(sum(1 for k in ks if k))}
+    full = rows["CWPN 100%"]["bwd_ms"]
+    for v in rows.values():
+        v["speedup_vs_full_qat"] = full / v["bwd_ms"]
+    out["backward"] = rows
+    # the schedule's own costs at the 10 % network-wide budget
+    net.use_selection(B.CWPN, B.ratio_to_k(0.1, total))
+    sel_ms = t(net.reselect)                              # importance + ranking + counts to the host
+    net.reselect()
+    fwd_ms = t(net.forward)
+    tail_ms = t(net.optimizer_tail)
+    bwd_ms = rows["CWPN 10%"]["bwd_ms"]
+    unc = NW.EfqatNetwork(ctx, states, B.CWPN, B.ratio_to_k(0.1, total), f_samples=batch, batch_samples=batch,
+                          use_cache=False, sgd=(SGD_LR, 0.9, 1e-4), adam=None)
+    unc.reselect()
+    out["uncached"] = {"fwd_ms": t(unc.forward), "bwd_ms": t(unc.backward)}
+    del unc
+    out["cached"] = {"fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "adam_and_cache_refresh_ms": tail_ms}
+    out["fwd_tops"] = gemm / (fwd_ms * 1e-3) / 1e12
+    out["select_ms"] = sel_ms
+    out["freezing_frequency"] = {
+        str(f): {"selections_per_step": min(1.0, batch / f),
+                 "amortised_select_ms_per_step": sel_ms * min(1.0, batch / f),
+                 "share_of_backward": sel_ms * min(1.0, batch / f) / (bwd_ms + sel_ms * min(1.0, batch / f))}
+        for f in (batch, 4096, 16384)}
+    # whole training steps under the real schedule: every step, and f = 4096 samples (171 steps apart)
+    for f, steps in ((batch, 24), (4096, 172)):
+        net.schedule = NW.FreezeSchedule(f, batch)
+        net.train_step()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            net.train_step()
+        torch.cuda.synchronize()
+        out["freezing_frequency"][str(f)]["train_step_ms_wall"] = 1e3 * (time.perf_counter() - t0) / steps
+        out["freezing_frequency"][str(f)]["selections_in_run"] = net.schedule.selections
+    out["paper_context"] = ("Table 5 (A100, BERT-base, f=4096): CWPN backward 1.36x / 1.33x / 1.23x faster than QAT at "
+                            "5 / 10 / 25 %, LWPN 1.49x / 1.48x / 1.44x, 0 % 1.55x")
+    return out
+
+
 def run_capture(args):
     """Short run for a profiler: the first layer of the headline workload alone, a few steps."""
     from paper_2411_11038_b200 import binding as B
@@ -450,6 +542,12 @@ def run_ours(args):
         status = status or ctx.device_status()
         del wl2
         torch.cuda.empty_cache()
+    # ---- the 144-layer stack: whole-network backward, weight-operand cache, freezing frequency
+    network = None
+    if not args.skip_extras and not args.no_network:
+        network = measure_network(ctx, dev, sync_all, max_over_ranks)
+        status = status or ctx.device_status()
+        torch.cuda.empty_cache()
     all_clock.stop_flag = True
     all_clock.join(timeout=2)
 
@@ -478,6 +576,7 @@ def run_ours(args):
             "bwd": head["bwd"],
             "select_ms": head["select_ms"],
             "bert_base": bert,
+            "network": network,
             "device_status": status,
             "paper_context": "paper reports 1.44-1.64x backward speed-up on A10/A100 (whole network)",
         }))
@@ -494,6 +593,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the headline timed steps and a 3-step end-to-end leg")
+    ap.add_argument("--no-network", action="store_true", help="skip the 144-layer stack")
     ap.add_argument("--capture", action="store_true",
                     help="three steps of the first headline layer alone (small run for a profiler)")
     args = ap.parse_args()

@@ -150,6 +150,62 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
                         float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null, void* ws,
                         size_t ws_bytes, efqat_stream_t stream);
 
+/* ---- weight-operand cache and whole-network calls (Section 3.2 "Freezing Frequency";
+ * Algorithm 1 runs the layer step over every layer of the network) --------------------- */
+/* Between two selections the frozen channels keep their weights and scales, hence their
+ * integer codes.  A caller-owned cache per layer holds the quantized weight operands of both
+ * passes (forward: the codes; backward: the dequantised weights of the grad-input GEMM), so
+ * that a forward / backward no longer reads W or re-quantizes it; after an optimizer step
+ * only the rows that step touched are rebuilt.  A cached operand is bit-identical to the one
+ * the uncached calls build, as long as every row whose weights or scale changed since its
+ * last rebuild is passed to efqat_weight_cache_update before the next cached call: keeping it
+ * current is the caller's contract, nothing in the block records validity. */
+/* Bytes of the cache block of `layer` (device memory, any alignment). */
+int efqat_weight_cache_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, size_t* out);
+/* Rebuilds rows idx[0..k_sel) of the cache from W fp32 [N,K] and s_w [N] (k_sel == N: every
+ * row, idx may be NULL; k_sel == 0: nothing).  idx: device int32, ascending, as returned by
+ * efqat_select_channels.  Call it once with k_sel = N before the first cached call. */
+int efqat_weight_cache_update(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const float* W,
+                              const float* s_w, const int32_t* idx, int64_t k_sel, void* cache, size_t cache_bytes,
+                              efqat_stream_t stream);
+/* efqat_fq_linear_fwd with the weight operand taken from the cache: W is not read. */
+int efqat_fq_linear_fwd_cached(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
+                               const float* s_w, const float* s_x, const float* z_x, const float* bias_or_null,
+                               void* Y, const void* cache, size_t cache_bytes, void* ws, size_t ws_bytes,
+                               efqat_stream_t stream);
+/* efqat_fq_linear_bwd with the grad-input operand taken from the cache; W is read only on the
+ * unfrozen rows (clip mask, dS_w, fused SGD). */
+int efqat_fq_linear_bwd_cached(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
+                               const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
+                               const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,
+                               float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null,
+                               const void* cache, size_t cache_bytes, void* ws, size_t ws_bytes,
+                               efqat_stream_t stream);
+
+/* One layer of a network: the arguments of the layer calls above, gathered (HOST struct, device
+ * pointers inside, meanings as documented there).  cache_or_null == NULL selects the uncached
+ * calls.  Layers may share one workspace `ws` (sized for the largest): the calls are ordered
+ * on the stream. */
+typedef struct {
+  efqat_layer_desc layer;
+  efqat_qspec q;
+  const void* X; const float* W; const float* s_w; const float* s_x; const float* z_x;
+  const float* bias_or_null; void* Y;                                   /* forward */
+  const void* dY; const int32_t* idx; int64_t k_sel;                    /* backward */
+  void* dX; float* dW_sel; float* dS_w_sel; float* dS_x; float* dZ_x; float* db_or_null;
+  const efqat_sgd* opt_or_null;
+  void* cache_or_null; size_t cache_bytes;
+  void* ws; size_t ws_bytes;
+} efqat_net_layer;
+/* Forward of layers[0..L) in order / backward of layers[L-1..0] in reverse order, enqueued on
+ * one stream with no host synchronisation in between (each launch overlaps its set-up with
+ * the tail of the one before it).  Stops at, and returns, the first host-side error. */
+int efqat_network_fwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream);
+int efqat_network_bwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream);
+/* efqat_weight_cache_update on rows idx of every layer that has a cache and k_sel > 0 (after
+ * the optimizer steps of a training step). */
+int efqat_network_cache_update(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream);
+
 /* ---- optimizer step of the quantization parameters (Section 4 "Setup": Adam for the
  * quantization parameters; Algorithm 1: "update the unfrozen weight channels and their
  * scales", "update the scales and zero points of the activations"; Appendix A.2: optional

@@ -28,6 +28,8 @@ EXPORTS = [
     "efqat_init_act_qparams", "efqat_init_weight_scales", "efqat_gemm_bf16",
     "efqat_profile_enable", "efqat_profile_read", "efqat_launch_count", "efqat_colsum_noalloc",
     "efqat_selftest_bounded_wait", "efqat_qparam_adam", "efqat_log2_scale_init",
+    "efqat_weight_cache_bytes", "efqat_weight_cache_update", "efqat_fq_linear_fwd_cached",
+    "efqat_fq_linear_bwd_cached", "efqat_network_fwd", "efqat_network_bwd", "efqat_network_cache_update",
 ]
 
 
@@ -54,6 +56,19 @@ class Adam(C.Structure):
 class QParamState(C.Structure):
     _fields_ = [("s_w", C.c_void_p), ("m_sw", C.c_void_p), ("v_sw", C.c_void_p), ("theta_sw", C.c_void_p),
                 ("s_x", C.c_void_p), ("z_x", C.c_void_p), ("state_x", C.c_void_p)]
+
+
+class NetLayer(C.Structure):
+    """efqat_net_layer: the arguments of one layer's forward / backward calls, gathered."""
+    _fields_ = [("layer", LayerDesc), ("q", QSpec),
+                ("X", C.c_void_p), ("W", C.c_void_p), ("s_w", C.c_void_p), ("s_x", C.c_void_p), ("z_x", C.c_void_p),
+                ("bias_or_null", C.c_void_p), ("Y", C.c_void_p),
+                ("dY", C.c_void_p), ("idx", C.c_void_p), ("k_sel", C.c_int64),
+                ("dX", C.c_void_p), ("dW_sel", C.c_void_p), ("dS_w_sel", C.c_void_p), ("dS_x", C.c_void_p),
+                ("dZ_x", C.c_void_p), ("db_or_null", C.c_void_p),
+                ("opt_or_null", C.POINTER(Sgd)),
+                ("cache_or_null", C.c_void_p), ("cache_bytes", C.c_size_t),
+                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t)]
 
 
 class EfqatError(RuntimeError):
@@ -103,6 +118,14 @@ def load() -> C.CDLL:
     lib.efqat_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
     lib.efqat_qparam_adam.argtypes = [vp, C.POINTER(Adam), C.POINTER(QParamState), i64, vp, i64, vp, vp, vp, vp]
     lib.efqat_log2_scale_init.argtypes = [vp, vp, vp, i64, vp]
+    lib.efqat_weight_cache_bytes.argtypes = [C.POINTER(LayerDesc), C.POINTER(QSpec), C.POINTER(sz)]
+    lib.efqat_weight_cache_update.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(QSpec), vp, vp, vp, i64, vp, sz, vp]
+    lib.efqat_fq_linear_fwd_cached.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(QSpec), vp, vp, vp, vp, vp, vp,
+                                               vp, sz, vp, sz, vp]
+    lib.efqat_fq_linear_bwd_cached.argtypes = [vp, C.POINTER(LayerDesc), C.POINTER(QSpec), vp, vp, vp, vp, vp, vp,
+                                               vp, i64, vp, vp, vp, vp, vp, vp, C.POINTER(Sgd), vp, sz, vp, sz, vp]
+    for nm in ("efqat_network_fwd", "efqat_network_bwd", "efqat_network_cache_update"):
+        getattr(lib, nm).argtypes = [vp, i32, C.POINTER(NetLayer), vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("efqat_status_string", "efqat_ratio_to_k", "efqat_launch_count"):
@@ -239,6 +262,12 @@ def select_workspace_bytes(L: int, total_channels: int) -> int:
     return out.value
 
 
+def weight_cache_bytes(desc: LayerDesc, spec: QSpec) -> int:
+    out = C.c_size_t(0)
+    _check(load().efqat_weight_cache_bytes(C.byref(desc), C.byref(spec), C.byref(out)), "efqat_weight_cache_bytes")
+    return out.value
+
+
 def alloc_workspace(nbytes: int, device) -> torch.Tensor:
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
@@ -292,7 +321,11 @@ class LayerPlan:
 
     def __init__(self, ctx: Context, M: int, N: int, K: int, act_dtype: torch.dtype, w_bits: int, x_bits: int,
                  x_symmetric: bool, k_sel_max: int, device, conv: Optional[ConvGeom] = None,
-                 x_shape=None, y_shape=None):
+                 x_shape=None, y_shape=None, with_cache: bool = False, ws: Optional[torch.Tensor] = None,
+                 outputs: Optional["LayerPlan"] = None):
+        """with_cache: also allocate the layer's weight-operand cache (fill it with cache_update).
+        ws: a workspace shared with other plans (calls on one stream only).  outputs: another plan
+        of the same shape whose output tensors this one reuses (layers timed one after another)."""
         self.ctx = ctx
         self.M, self.N, self.K = M, N, K
         self.act_dtype = act_dtype
@@ -300,16 +333,26 @@ class LayerPlan:
         self.desc = layer_desc(M, N, K, code, conv)
         self.spec = QSpec(w_bits, x_bits, 1 if x_symmetric else 0)
         self.k_sel_max = k_sel_max
-        self.ws = alloc_workspace(workspace_bytes(self.desc, self.spec, k_sel_max), device)
+        self.ws_bytes = workspace_bytes(self.desc, self.spec, k_sel_max)
+        if ws is not None and ws.numel() < self.ws_bytes:
+            raise ValueError("shared workspace too small for this layer")
+        self.ws = ws if ws is not None else alloc_workspace(self.ws_bytes, device)
         xs = tuple(x_shape) if x_shape is not None else (M, K)
         ys = tuple(y_shape) if y_shape is not None else (M, N)
-        self.Y = torch.empty(ys, dtype=act_dtype, device=device)
-        self.dX = torch.empty(xs, dtype=act_dtype, device=device)
-        self.dW_sel = torch.empty((max(k_sel_max, 1), K), dtype=torch.float32, device=device)
+        if outputs is not None:
+            if (outputs.M, outputs.N, outputs.K, outputs.act_dtype) != (M, N, K, act_dtype) or \
+                    outputs.k_sel_max < k_sel_max:
+                raise ValueError("output tensors can only be shared between plans of one shape")
+            self.Y, self.dX, self.dW_sel, self.db = outputs.Y, outputs.dX, outputs.dW_sel, outputs.db
+        else:
+            self.Y = torch.empty(ys, dtype=act_dtype, device=device)
+            self.dX = torch.empty(xs, dtype=act_dtype, device=device)
+            self.dW_sel = torch.empty((max(k_sel_max, 1), K), dtype=torch.float32, device=device)
+            self.db = torch.empty(N, dtype=torch.float32, device=device)
         self.dS_w_sel = torch.empty(max(k_sel_max, 1), dtype=torch.float32, device=device)
         self.dS_x = torch.empty(1, dtype=torch.float32, device=device)
         self.dZ_x = torch.empty(1, dtype=torch.float32, device=device)
-        self.db = torch.empty(N, dtype=torch.float32, device=device)
+        self.cache = alloc_workspace(weight_cache_bytes(self.desc, self.spec), device) if with_cache else None
 
     def fwd(self, X, W, s_w, s_x, z_x, bias=None):
         rc = load().efqat_fq_linear_fwd(self.ctx.handle, C.byref(self.desc), C.byref(self.spec), _ptr(X), _ptr(W),
@@ -328,6 +371,82 @@ class LayerPlan:
         _check(rc, "efqat_fq_linear_bwd")
         return dict(dX=self.dX, dW_sel=self.dW_sel[:k_sel], dS_w_sel=self.dS_w_sel[:k_sel], dS_x=self.dS_x,
                     dZ_x=self.dZ_x, db=self.db if want_db else None)
+
+
+    # ---- weight-operand cache ------------------------------------------------------------
+    def cache_update(self, W, s_w, idx=None, k_sel: Optional[int] = None):
+        """efqat_weight_cache_update: rows idx[0..k_sel) of the cache (default: every row)."""
+        k = self.N if k_sel is None else int(k_sel)
+        rc = load().efqat_weight_cache_update(self.ctx.handle, C.byref(self.desc), C.byref(self.spec), _ptr(W),
+                                              _ptr(s_w), _ptr(idx), k, _ptr(self.cache), self.cache.numel(), _stream())
+        _check(rc, "efqat_weight_cache_update")
+
+    def fwd_cached(self, X, s_w, s_x, z_x, bias=None):
+        rc = load().efqat_fq_linear_fwd_cached(self.ctx.handle, C.byref(self.desc), C.byref(self.spec), _ptr(X),
+                                               _ptr(s_w), _ptr(s_x), _ptr(z_x), _ptr(bias), _ptr(self.Y),
+                                               _ptr(self.cache), self.cache.numel(), _ptr(self.ws), self.ws.numel(),
+                                               _stream())
+        _check(rc, "efqat_fq_linear_fwd_cached")
+        return self.Y
+
+    def bwd_cached(self, dY, X, W, s_w, s_x, z_x, idx, k_sel: int, want_db: bool = True, sgd: Optional[Sgd] = None):
+        rc = load().efqat_fq_linear_bwd_cached(self.ctx.handle, C.byref(self.desc), C.byref(self.spec), _ptr(dY),
+                                               _ptr(X), _ptr(W), _ptr(s_w), _ptr(s_x), _ptr(z_x), _ptr(idx), int(k_sel),
+                                               _ptr(self.dX), _ptr(self.dW_sel), _ptr(self.dS_w_sel), _ptr(self.dS_x),
+                                               _ptr(self.dZ_x), _ptr(self.db) if want_db else None,
+                                               C.byref(sgd) if sgd is not None else None, _ptr(self.cache),
+                                               self.cache.numel(), _ptr(self.ws), self.ws.numel(), _stream())
+        _check(rc, "efqat_fq_linear_bwd_cached")
+        return dict(dX=self.dX, dW_sel=self.dW_sel[:k_sel], dS_w_sel=self.dS_w_sel[:k_sel], dS_x=self.dS_x,
+                    dZ_x=self.dZ_x, db=self.db if want_db else None)
+
+    def net_layer(self, X, W, s_w, s_x, z_x, bias, dY, sgd: Optional[Sgd] = None, want_db: bool = True,
+                  use_cache: bool = True) -> NetLayer:
+        """This layer's entry of an efqat_net_layer array (idx / k_sel are set per step)."""
+        n = NetLayer()
+        n.layer, n.q = self.desc, self.spec
+        n.X, n.W, n.s_w, n.s_x, n.z_x = (t.data_ptr() for t in (X, W, s_w, s_x, z_x))
+        n.bias_or_null = bias.data_ptr() if bias is not None else None
+        n.Y = self.Y.data_ptr()
+        n.dY = dY.data_ptr()
+        n.idx, n.k_sel = None, 0
+        n.dX, n.dW_sel, n.dS_w_sel = self.dX.data_ptr(), self.dW_sel.data_ptr(), self.dS_w_sel.data_ptr()
+        n.dS_x, n.dZ_x = self.dS_x.data_ptr(), self.dZ_x.data_ptr()
+        n.db_or_null = self.db.data_ptr() if want_db else None
+        n.opt_or_null = C.pointer(sgd) if sgd is not None else None
+        if use_cache and self.cache is not None:
+            n.cache_or_null, n.cache_bytes = self.cache.data_ptr(), self.cache.numel()
+        n.ws, n.ws_bytes = self.ws.data_ptr(), self.ws.numel()
+        return n
+
+
+class NetworkPlan:
+    """efqat_network_fwd / _bwd / _cache_update over a fixed list of layers: the efqat_net_layer
+    array is marshalled once; a step only rewrites the per-layer (idx, k_sel)."""
+
+    def __init__(self, ctx: Context, entries: Sequence[NetLayer], keep=()):
+        self.ctx, self.L = ctx, len(entries)
+        self.arr = (NetLayer * self.L)(*entries)
+        self.keep = (list(entries), list(keep))     # the structs (and Sgd objects) the pointers refer to
+
+    def set_selection(self, idx: torch.Tensor, offsets_host: Sequence[int]):
+        """Per-layer views of the concatenated index list of efqat_select_channels."""
+        self.idx = idx
+        base, es = idx.data_ptr(), idx.element_size()
+        for l in range(self.L):
+            k = int(offsets_host[l + 1] - offsets_host[l])
+            self.arr[l].k_sel = k
+            self.arr[l].idx = (base + es * int(offsets_host[l])) if k else None
+
+    def fwd(self):
+        _check(load().efqat_network_fwd(self.ctx.handle, self.L, self.arr, _stream()), "efqat_network_fwd")
+
+    def bwd(self):
+        _check(load().efqat_network_bwd(self.ctx.handle, self.L, self.arr, _stream()), "efqat_network_bwd")
+
+    def cache_update(self):
+        _check(load().efqat_network_cache_update(self.ctx.handle, self.L, self.arr, _stream()),
+               "efqat_network_cache_update")
 
 
 def _plan_for(ctx, X, W, w_bits, x_bits, x_symmetric, k_sel_max, conv):

@@ -139,6 +139,46 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   return w;
 }
 
+// A plain layer runs its forward on the integer tensor cores: 8-bit codes, int32 accumulation,
+// zero point taken out exactly in the epilogue.  int32 holds K * 255 * 127 up to K = 65536; the
+// limit here leaves a factor 2.  The row pitch of the 8-bit operands must be a multiple of 16
+// bytes for TMA, and tiles are kept to multiples of 32 columns, the coarser of the instruction's
+// N granularities.  Short contractions (K <= 256: output-bound layers whose 128-wide k-blocks
+// would be half padding) measured slower this way and stay on the bf16 path.
+bool fwd_on_i8(const efqat_layer_desc* l) {
+  return !spatial_conv(l) && l->K >= 512 && l->K <= 32768 && l->K % 16 == 0 && l->N % 32 == 0;
+}
+
+// Sections of a layer's weight-operand cache (see cache.cu).
+struct WCache {
+  int8_t* codes8;     // [N,K] 8-bit codes (integer forward) ...
+  int32_t* wsum;      // [N] ... and their row sums
+  bf16* codes16;      // [N,K] codes as bf16 (every other forward)
+  bf16* what;         // [N,K] dequantised weights (grad-input GEMM)
+  size_t bytes;
+};
+
+WCache carve_cache(void* cache, const efqat_layer_desc* l) {
+  WCache c = {};
+  char* base = cache ? reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(cache) + 255) & ~uintptr_t(255)) : nullptr;
+  size_t off = 0;
+  auto take = [&](int64_t bytes) {
+    char* r = base ? base + off : nullptr;
+    off += static_cast<size_t>(round_up(bytes, 256));
+    return r;
+  };
+  const int64_t nk = l->N * l->K;
+  if (fwd_on_i8(l)) {
+    c.codes8 = reinterpret_cast<int8_t*>(take(nk));
+    c.wsum = reinterpret_cast<int32_t*>(take(l->N * 4));
+  } else {
+    c.codes16 = reinterpret_cast<bf16*>(take(nk * 2));
+  }
+  c.what = reinterpret_cast<bf16*>(take(nk * 2));
+  c.bytes = off + 256;
+  return c;
+}
+
 int guard_device(const efqat_ctx* ctx) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device) return EFQAT_ERR_CUDA;
@@ -345,10 +385,16 @@ int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_des
                     ctx->d_status, stream);
 }
 
-int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
-                        const float* W, const float* s_w, const float* s_x, const float* z_x,
-                        const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream) {
-  if (!ctx || !X || !W || !s_w || !s_x || !Y) return EFQAT_ERR_NULL;
+}  // extern "C"
+
+namespace {
+
+// Forward of one layer.  cache != NULL: the weight operand comes from the layer's cache and W is
+// not read (it may be NULL).
+int fwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X, const float* W,
+             const float* s_w, const float* s_x, const float* z_x, const float* bias_or_null, void* Y, void* ws,
+             size_t ws_bytes, const void* cache, size_t cache_bytes, efqat_stream_t stream) {
+  if (!ctx || !X || (!W && !cache) || !s_w || !s_x || !Y) return EFQAT_ERR_NULL;
   int rc = check_layer(layer, q);
   if (rc != EFQAT_OK) return rc;
   if (!q->x_symmetric && !z_x) return EFQAT_ERR_NULL;
@@ -358,6 +404,11 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   if (rc != EFQAT_OK) return rc;
   const LayerWs w = carve(ws, layer, 0, ctx->sm_count, 0);
   if (ws_bytes < w.bytes) return EFQAT_ERR_WORKSPACE;
+  WCache wc = {};
+  if (cache) {
+    wc = carve_cache(const_cast<void*>(cache), layer);
+    if (cache_bytes < wc.bytes) return EFQAT_ERR_WORKSPACE;
+  }
   Entered in(ctx);
   const int64_t M = layer->M, N = layer->N, K = layer->K;
   cudaStream_t st = stream;
@@ -366,18 +417,12 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   // a2: both quantizers in one launch
   PrepArgs pa = {};
   pa.M = M; pa.N = N; pa.K = K;
-  pa.W = W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
+  pa.W = cache ? nullptr : W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric; pa.Xc = w.Xc;
   pa.x_count = x_elems(layer);
   pa.status = ctx->d_status;
-  // A plain layer runs its forward on the integer tensor cores: 8-bit codes (the code buffers
-  // of the bf16 path are reused, half filled), int32 accumulation, zero point taken out exactly in
-  // the epilogue.  int32 holds K * 255 * 127 up to K = 65536; the limit here leaves a factor 2.
-  // (row pitch of the 8-bit operands must be a multiple of 16 bytes for TMA; tiles are kept to
-  // multiples of 32 columns, the coarser of the instruction's N granularities)
-  // Short contractions (K <= 256: output-bound layers whose 128-wide k-blocks would be half
-  // padding) measured slower this way and stay on the bf16 path.
-  const bool i8 = !spatial_conv(layer) && K >= 512 && K <= 32768 && K % 16 == 0 && N % 32 == 0;
+  // integer forward: the code buffers of the bf16 path are reused, half filled
+  const bool i8 = fwd_on_i8(layer);
   if (i8) {
     pa.i8 = 1;
     pa.Wq8 = reinterpret_cast<int8_t*>(w.Wq);
@@ -388,8 +433,9 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   ConvArgs cva;
   GemmArgs g = {};
   g.i8 = i8 ? 1 : 0;
-  g.wsum = w.wsum;
-  g.A = w.Xc; g.B = w.Wq;
+  g.wsum = cache ? wc.wsum : w.wsum;
+  g.A = w.Xc;
+  g.B = !cache ? w.Wq : (i8 ? reinterpret_cast<const bf16*>(wc.codes8) : wc.codes16);
   g.Mr = M; g.Nc = N; g.Kc = K;
   g.lda = K; g.ldb = K;
   g.a_mn = 0; g.b_mn = 0;
@@ -408,11 +454,13 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   return last_error();
 }
 
-int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
-                        const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
-                        const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,
-                        float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null, void* ws,
-                        size_t ws_bytes, efqat_stream_t stream) {
+// Backward of one layer.  cache != NULL: the grad-input GEMM reads the dequantised weights of the
+// layer's cache instead of rebuilding them (W is still read for the clip mask of the unfrozen rows).
+int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY, const void* X,
+             const float* W, const float* s_w, const float* s_x, const float* z_x, const int32_t* idx, int64_t k_sel,
+             void* dX, float* dW_sel, float* dS_w_sel, float* dS_x, float* dZ_x, float* db_or_null,
+             const efqat_sgd* opt_or_null, void* ws, size_t ws_bytes, const void* cache, size_t cache_bytes,
+             efqat_stream_t stream) {
   if (!ctx || !dY || !X || !W || !s_w || !s_x || !dX || !dS_x || !dZ_x) return EFQAT_ERR_NULL;
   int rc = check_layer(layer, q);
   if (rc != EFQAT_OK) return rc;
@@ -432,6 +480,11 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   if (rc != EFQAT_OK) return rc;
   const LayerWs w = carve(ws, layer, k_sel, ctx->sm_count, -1);
   if (ws_bytes < w.bytes) return EFQAT_ERR_WORKSPACE;
+  WCache wc = {};
+  if (cache) {
+    wc = carve_cache(const_cast<void*>(cache), layer);
+    if (cache_bytes < wc.bytes) return EFQAT_ERR_WORKSPACE;
+  }
   Entered in(ctx);
   cudaStream_t st = stream;
   const int act_bf16 = layer->act_dtype == EFQAT_BF16;
@@ -442,7 +495,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   const bf16* dYb = act_bf16 ? static_cast<const bf16*>(dY) : w.dYb;
   PrepArgs pa = {};
   pa.M = M; pa.N = N; pa.K = K;
-  pa.W = W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
+  pa.W = cache ? nullptr : W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric;
   pa.Xc = k_sel > 0 ? w.Xc : nullptr;
   pa.x_count = x_elems(layer);
@@ -458,7 +511,7 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   {
     GemmArgs g = {};
     if (sconv) g.conv = &cv_dx;
-    g.A = dYb; g.B = w.Wq;
+    g.A = dYb; g.B = cache ? wc.what : w.Wq;
     g.Mr = sconv ? x_elems(layer) / layer->Cin : M;
     g.Nc = sconv ? layer->Cin : K;
     g.Kc = sconv ? static_cast<int64_t>(layer->R) * layer->S * N : N;
@@ -521,6 +574,115 @@ int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
   fa.status = ctx->d_status;
   launch_finalize(fa, st);
   return last_error();
+}
+
+}  // namespace
+
+extern "C" {
+
+int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
+                        const float* W, const float* s_w, const float* s_x, const float* z_x,
+                        const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream) {
+  if (!W) return EFQAT_ERR_NULL;
+  return fwd_impl(ctx, layer, q, X, W, s_w, s_x, z_x, bias_or_null, Y, ws, ws_bytes, nullptr, 0, stream);
+}
+
+int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
+                        const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
+                        const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,
+                        float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null, void* ws,
+                        size_t ws_bytes, efqat_stream_t stream) {
+  return bwd_impl(ctx, layer, q, dY, X, W, s_w, s_x, z_x, idx, k_sel, dX, dW_sel, dS_w_sel, dS_x, dZ_x, db_or_null,
+                  opt_or_null, ws, ws_bytes, nullptr, 0, stream);
+}
+
+int efqat_weight_cache_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, size_t* out) {
+  if (!out) return EFQAT_ERR_NULL;
+  const int rc = check_layer(layer, q);
+  if (rc != EFQAT_OK) return rc;
+  *out = carve_cache(nullptr, layer).bytes;
+  return EFQAT_OK;
+}
+
+int efqat_weight_cache_update(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const float* W,
+                              const float* s_w, const int32_t* idx, int64_t k_sel, void* cache, size_t cache_bytes,
+                              efqat_stream_t stream) {
+  if (!ctx || !W || !s_w || !cache) return EFQAT_ERR_NULL;
+  int rc = check_layer(layer, q);
+  if (rc != EFQAT_OK) return rc;
+  if (k_sel < 0 || k_sel > layer->N) return EFQAT_ERR_K_RANGE;
+  if (k_sel > 0 && k_sel < layer->N && !idx) return EFQAT_ERR_NULL;
+  if (!aligned16(W)) return EFQAT_ERR_ALIGN;
+  rc = guard_device(ctx);
+  if (rc != EFQAT_OK) return rc;
+  const WCache wc = carve_cache(cache, layer);
+  if (cache_bytes < wc.bytes) return EFQAT_ERR_WORKSPACE;
+  Entered in(ctx);
+  CacheArgs a = {};
+  a.N = layer->N; a.K = layer->K; a.rows = k_sel;
+  a.W = W; a.s_w = s_w; a.w_bits = q->w_bits;
+  a.idx = (k_sel < layer->N) ? idx : nullptr;
+  a.codes8 = wc.codes8; a.wsum = wc.wsum; a.codes16 = wc.codes16; a.what = wc.what;
+  a.status = ctx->d_status;
+  launch_weight_cache(a, stream);
+  return last_error();
+}
+
+int efqat_fq_linear_fwd_cached(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
+                               const float* s_w, const float* s_x, const float* z_x, const float* bias_or_null,
+                               void* Y, const void* cache, size_t cache_bytes, void* ws, size_t ws_bytes,
+                               efqat_stream_t stream) {
+  if (!cache) return EFQAT_ERR_NULL;
+  return fwd_impl(ctx, layer, q, X, nullptr, s_w, s_x, z_x, bias_or_null, Y, ws, ws_bytes, cache, cache_bytes, stream);
+}
+
+int efqat_fq_linear_bwd_cached(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
+                               const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
+                               const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,
+                               float* dS_x, float* dZ_x, float* db_or_null, const efqat_sgd* opt_or_null,
+                               const void* cache, size_t cache_bytes, void* ws, size_t ws_bytes,
+                               efqat_stream_t stream) {
+  if (!cache) return EFQAT_ERR_NULL;
+  return bwd_impl(ctx, layer, q, dY, X, W, s_w, s_x, z_x, idx, k_sel, dX, dW_sel, dS_w_sel, dS_x, dZ_x, db_or_null,
+                  opt_or_null, ws, ws_bytes, cache, cache_bytes, stream);
+}
+
+int efqat_network_fwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream) {
+  if (!ctx || !layers) return EFQAT_ERR_NULL;
+  if (L < 1) return EFQAT_ERR_SHAPE;
+  for (int l = 0; l < L; ++l) {
+    const efqat_net_layer& n = layers[l];
+    const int rc = fwd_impl(ctx, &n.layer, &n.q, n.X, n.W, n.s_w, n.s_x, n.z_x, n.bias_or_null, n.Y, n.ws, n.ws_bytes,
+                            n.cache_or_null, n.cache_bytes, stream);
+    if (rc != EFQAT_OK) return rc;
+  }
+  return EFQAT_OK;
+}
+
+int efqat_network_bwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream) {
+  if (!ctx || !layers) return EFQAT_ERR_NULL;
+  if (L < 1) return EFQAT_ERR_SHAPE;
+  for (int l = L - 1; l >= 0; --l) {
+    const efqat_net_layer& n = layers[l];
+    const int rc = bwd_impl(ctx, &n.layer, &n.q, n.dY, n.X, n.W, n.s_w, n.s_x, n.z_x, n.idx, n.k_sel, n.dX, n.dW_sel,
+                            n.dS_w_sel, n.dS_x, n.dZ_x, n.db_or_null, n.opt_or_null, n.ws, n.ws_bytes,
+                            n.cache_or_null, n.cache_bytes, stream);
+    if (rc != EFQAT_OK) return rc;
+  }
+  return EFQAT_OK;
+}
+
+int efqat_network_cache_update(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream) {
+  if (!ctx || !layers) return EFQAT_ERR_NULL;
+  if (L < 1) return EFQAT_ERR_SHAPE;
+  for (int l = 0; l < L; ++l) {
+    const efqat_net_layer& n = layers[l];
+    if (!n.cache_or_null || n.k_sel == 0) continue;
+    const int rc = efqat_weight_cache_update(ctx, &n.layer, &n.q, n.W, n.s_w, n.idx, n.k_sel, n.cache_or_null,
+                                             n.cache_bytes, stream);
+    if (rc != EFQAT_OK) return rc;
+  }
+  return EFQAT_OK;
 }
 
 int efqat_gemm_bf16(efqat_ctx* ctx, const void* A, const void* B, int64_t M, int64_t N, int64_t K, int a_mn,

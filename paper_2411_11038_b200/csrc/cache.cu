@@ -1,0 +1,98 @@
+// Weight-operand cache (Section 3.2 "Freezing Frequency").  Between two selections a frozen
+// channel's weights and scale do not move, so neither do its integer codes; only the rows the
+// optimizer has just stepped need quantizing again.  The cache is a caller-owned block that
+// holds, per layer, exactly what the prepare launch would otherwise rebuild on every call:
+//   forward operand : the weight codes (8-bit with their row sums for layers whose forward
+//                     runs on the integer tensor cores, else as bf16 integers);
+//   backward operand: the dequantised weights bf16(s_w[n] * q_w[n,k]) of the grad-input GEMM.
+// One warp per row; rows come from idx (the unfrozen channels) or are all N rows.  The
+// arithmetic is the prepare launch's own (quant_weight, one fp32 multiply), so a cached
+// operand is bit-identical to a rebuilt one.
+#include "internal.h"
+
+namespace efqat {
+
+namespace {
+
+__device__ __forceinline__ uint32_t pk2c(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__global__ void __launch_bounds__(256) weight_cache_kernel(const CacheArgs a) {
+  pdl_trigger();
+  pdl_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t kv = a.K / 8;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * 8 + warp; i < a.rows; i += static_cast<int64_t>(gridDim.x) * 8) {
+    int64_t n = i;
+    if (a.idx) {
+      n = a.idx[i];
+      // index contract of the layer calls: inside [0, N), strictly ascending
+      if (n < 0 || n >= a.N || (i > 0 && a.idx[i - 1] >= n)) {
+        if (lane == 0) record_status(a.status, EFQAT_DEV_BAD_INDEX);
+        continue;
+      }
+    }
+    float sw = __ldg(a.s_w + n);
+    if (!scale_ok(sw)) {
+      if (lane == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
+      sw = 1.f;
+    }
+    const RowQ p = make_rowq(sw, a.w_bits);
+    const float* row = a.W + n * a.K;
+    int sum = 0;
+    for (int64_t v0 = lane; v0 < kv; v0 += 64) {       // two independent 32-byte loads in flight
+      float4 w4[2][2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (v0 + 32 * u < kv) {
+          w4[u][0] = __ldg(reinterpret_cast<const float4*>(row + (v0 + 32 * u) * 8));
+          w4[u][1] = __ldg(reinterpret_cast<const float4*>(row + (v0 + 32 * u) * 8) + 1);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        if (v0 + 32 * u < kv) {
+          const float w[8] = {w4[u][0].x, w4[u][0].y, w4[u][0].z, w4[u][0].w,
+                              w4[u][1].x, w4[u][1].y, w4[u][1].z, w4[u][1].w};
+          float q[8], d[8];
+          uint32_t b0 = 0, b1 = 0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const QElem e = quant_weight(w[j], p);
+            q[j] = e.c0;
+            d[j] = __fmul_rn(p.s, e.c0);
+            sum += e.code;
+            const uint32_t byte = static_cast<uint32_t>(e.code) & 255u;
+            if (j < 4) b0 |= byte << (8 * j); else b1 |= byte << (8 * (j - 4));
+          }
+          const int64_t o = n * a.K + (v0 + 32 * u) * 8;
+          if (a.codes8) *reinterpret_cast<uint2*>(a.codes8 + o) = make_uint2(b0, b1);
+          if (a.codes16)
+            *reinterpret_cast<uint4*>(a.codes16 + o) =
+                make_uint4(pk2c(q[0], q[1]), pk2c(q[2], q[3]), pk2c(q[4], q[5]), pk2c(q[6], q[7]));
+          *reinterpret_cast<uint4*>(a.what + o) =
+              make_uint4(pk2c(d[0], d[1]), pk2c(d[2], d[3]), pk2c(d[4], d[5]), pk2c(d[6], d[7]));
+        }
+      }
+    }
+    if (a.wsum) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) a.wsum[n] = sum;
+    }
+  }
+}
+
+}  // namespace
+
+void launch_weight_cache(const CacheArgs& a, cudaStream_t st) {
+  if (a.rows < 1) return;
+  int64_t grid = ceil_div(a.rows, 8);
+  if (grid > 148 * 16) grid = 148 * 16;
+  count_launches(1);
+  launch_dependent(weight_cache_kernel, static_cast<unsigned>(grid), 256, 0, st, 1, a);
+}
+
+}  // namespace efqat

@@ -449,6 +449,7 @@ static int flat_blocks(int64_t vectors, int64_t per_block) {
 void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   a.nb_w = flat_blocks(a.N * (a.K / 8), 256 * 4);       // 32 KiB of fp32 weights per block
   if (a.i8) a.nb_w = static_cast<int>(ceil_div(a.N, 8) < 148 * 12 ? ceil_div(a.N, 8) : 148 * 12);   // a warp per row
+  if (!a.W) a.nb_w = 0;                          // weight operand supplied by the layer's cache
   a.nb_x = 0;
   if (a.Xc || (a.i8 && a.Xc8)) a.nb_x = flat_blocks(a.x_count / 8, 256 * 8);   // 32 KiB (bf16) / 64 KiB (fp32) per block
   const bool gather = a.dY && a.dYsel && a.k_sel > 0 && a.k_sel < a.N;
@@ -458,6 +459,7 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   a.dy_on = (a.dY && (a.colsum_ws || a.dYb)) ? 1 : 0;
   const int nb_y = (a.col_blocks * a.dy_on + a.nb_g) * a.slabs;
   const int grid = a.nb_w + a.nb_x + nb_y;
+  if (grid == 0) return;                         // cached weights, nothing unfrozen, no bias gradient wanted
   count_launches(1);
   if (w_mode == 0) {
     if (act_bf16) launch_dependent(prepare_kernel<0, bf16>, grid, 256, 0, st, 1, a);

@@ -99,6 +99,19 @@ void launch_qparam_adam(const efqat_adam& a, const efqat_qparam_state& st, int64
                         cudaStream_t stream);
 void launch_log2_init(const float* s, float* theta, int64_t n, int* status, cudaStream_t stream);
 
+// ---- cache.cu -----------------------------------------------------------------------
+// Rebuilds rows of a layer's weight-operand cache: rows idx[0..rows) (idx null: rows 0..rows).
+// codes8 + wsum (integer forward) or codes16 (bf16 forward) and what (backward) as laid out
+// by the cache carving of the entry points.
+struct CacheArgs {
+  int64_t N, K, rows;
+  const float* W; const float* s_w; int w_bits;
+  const int32_t* idx;
+  int8_t* codes8; int32_t* wsum; bf16* codes16; bf16* what;
+  int* status;
+};
+void launch_weight_cache(const CacheArgs& a, cudaStream_t st);
+
 // ---- select.cu ----------------------------------------------------------------------
 size_t select_workspace_bytes(int L, int64_t total_channels);
 int run_select(int mode, int L, const efqat_layer_desc* layers, const float* const* weights, const int64_t* k,

@@ -82,17 +82,22 @@ def fwd_reference(case, T, s_w, s_x, z_x):
     return Y, Yabs
 
 
-def check_forward(ctx, case, T, D, s_w, s_x, z_x):
-    Y = B.fq_linear_fwd(ctx, D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D.get("bias"),
-                        case.w_bits, case.x_bits, case.x_symmetric)
-    torch.cuda.synchronize()
-    assert ctx.device_status() == 0
+def check_forward_values(case, T, Y, s_w, s_x, z_x):
+    """Compares a forward output Y (device tensor) with the oracle's on the CPU tensors T."""
     ref, ref_abs = fwd_reference(case, T, s_w, s_x, z_x)
     got = np32(Y)
     is_bf16 = case.act_dtype == torch.bfloat16
     assert_bf16_class(got, ref, f"{case.name} Y")
     assert_fp32_class(got, ref, ref_abs, f"{case.name} Y", out_is_bf16=is_bf16)
     return got
+
+
+def check_forward(ctx, case, T, D, s_w, s_x, z_x):
+    Y = B.fq_linear_fwd(ctx, D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D.get("bias"),
+                        case.w_bits, case.x_bits, case.x_symmetric)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    return check_forward_values(case, T, Y, s_w, s_x, z_x)
 
 
 def check_backward(ctx, case, T, D, s_w, s_x, z_x, idx_np, sgd=None, full_ref=None):

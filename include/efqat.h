@@ -16,7 +16,9 @@
  *     paper Section 3.1 footnote).  Convolution: X NHWC [B,H,W,Cin], W [N,R,S,Cin],
  *     Y/dY [B,Ho,Wo,N]; its GEMM view is M = B*Ho*Wo, K = R*S*Cin.
  *   - Alignment: every base pointer 16-byte aligned; N % 8 == 0 and K % 8 == 0 (Cin % 8 == 0
- *     for convolutions).  Violations return EFQAT_ERR_ALIGN; there is no slow path.
+ *     for convolutions: an input with fewer channels, such as a 3-channel image, is stored
+ *     with zero channels up to 8, and so is its filter).  Violations return EFQAT_ERR_ALIGN;
+ *     there is no slow path.
  *   - Activations (X, dY, Y, dX) are fp32 or bf16 (efqat_dtype); weights, scales, zero
  *     point, bias and all gradients of parameters are fp32.
  */
@@ -43,7 +45,7 @@ typedef enum {
   EFQAT_ERR_MODE = -6,       /* unknown efqat_mode */
   EFQAT_ERR_WORKSPACE = -7,  /* workspace too small or NULL */
   EFQAT_ERR_K_RANGE = -8,    /* k_sel / budget outside its range */
-  EFQAT_ERR_UNIMPL = -9,     /* combination not built (e.g. conv stride != 1) */
+  EFQAT_ERR_UNIMPL = -9,     /* combination not built (e.g. conv stride > 2, filter beyond 7 x 7) */
   EFQAT_ERR_CUDA = -10,      /* a CUDA runtime / driver call failed */
   EFQAT_ERR_TOO_LARGE = -11, /* a size exceeds a fixed built-in maximum (efqat_colsum_noalloc) */
   /* device-side conditions, reported by efqat_device_status (positive) */
@@ -66,7 +68,10 @@ typedef struct {
 } efqat_qspec;
 
 /* One quantized layer.  Linear: is_conv = 0 and only M, N, K, act_dtype are read.
- * Convolution: is_conv = 1, stride 1, pad < R; M and K must equal B*Ho*Wo and R*S*Cin. */
+ * Convolution: is_conv = 1, stride 1 or 2 (the same along H and W), filters up to 7 x 7
+ * (R*S <= 49), pad < R and pad < S, Ho = (H + 2*pad - R) / stride + 1 (Wo alike); M and K must
+ * equal B*Ho*Wo and R*S*Cin.  This covers the paper's networks: 1x1 and 3x3 convolutions, the
+ * stride-2 3x3 and 1x1 shortcut convolutions and the 7x7 stride-2 input layer (Section 4). */
 typedef struct {
   int64_t M, N, K;
   int is_conv;

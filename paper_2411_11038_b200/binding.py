@@ -453,8 +453,8 @@ def _plan_for(ctx, X, W, w_bits, x_bits, x_symmetric, k_sel_max, conv):
     N = int(W.shape[0])
     K = int(W.numel() // N)
     if conv is not None:
-        Ho = conv.H + 2 * conv.pad - conv.R + 1
-        Wo = conv.W + 2 * conv.pad - conv.S + 1
+        Ho = (conv.H + 2 * conv.pad - conv.R) // conv.stride + 1
+        Wo = (conv.W + 2 * conv.pad - conv.S) // conv.stride + 1
         M = conv.B * Ho * Wo
         return LayerPlan(ctx, M, N, K, X.dtype, w_bits, x_bits, x_symmetric, k_sel_max, X.device, conv,
                          x_shape=X.shape, y_shape=(conv.B, Ho, Wo, N))

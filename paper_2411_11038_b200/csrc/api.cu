@@ -41,6 +41,11 @@ namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Output extent of a convolution along one axis.
+inline int64_t conv_out(int64_t in, int64_t filt, int64_t pad, int64_t stride) {
+  return (in + 2 * pad - filt) / stride + 1;
+}
+
 int check_bits(const efqat_qspec* q) {
   if (!q) return EFQAT_ERR_NULL;
   if (q->w_bits < 2 || q->w_bits > 8 || q->x_bits < 2 || q->x_bits > 8) return EFQAT_ERR_BITS;
@@ -57,14 +62,14 @@ int check_layer(const efqat_layer_desc* l, const efqat_qspec* q) {
   if ((l->N & 7) || (l->K & 7)) return EFQAT_ERR_ALIGN;
   if (l->is_conv) {
     if (l->B < 1 || l->H < 1 || l->W < 1 || l->Cin < 1 || l->R < 1 || l->S < 1) return EFQAT_ERR_SHAPE;
-    if (l->stride != 1) return EFQAT_ERR_UNIMPL;
+    if (l->stride < 1) return EFQAT_ERR_SHAPE;
+    if (l->stride > 2 || l->R * l->S > 49) return EFQAT_ERR_UNIMPL;     // strides 1 and 2, filters up to 7 x 7
     if (l->pad < 0 || l->pad >= l->R || l->pad >= l->S) return EFQAT_ERR_SHAPE;
     if (l->Cin & 7) return EFQAT_ERR_ALIGN;
-    const int64_t Ho = l->H + 2 * l->pad - l->R + 1, Wo = l->W + 2 * l->pad - l->S + 1;
-    if (Ho < 1 || Wo < 1) return EFQAT_ERR_SHAPE;
+    if (l->H + 2 * l->pad < l->R || l->W + 2 * l->pad < l->S) return EFQAT_ERR_SHAPE;
+    const int64_t Ho = conv_out(l->H, l->R, l->pad, l->stride), Wo = conv_out(l->W, l->S, l->pad, l->stride);
     if (l->M != static_cast<int64_t>(l->B) * Ho * Wo) return EFQAT_ERR_SHAPE;
     if (l->K != static_cast<int64_t>(l->R) * l->S * l->Cin) return EFQAT_ERR_SHAPE;
-    if ((l->R != 1 || l->S != 1 || l->pad != 0) && (l->Cin & 63)) return EFQAT_ERR_UNIMPL;   // tap-wise tiles need Cin % 64 == 0
   }
   return EFQAT_OK;
 }
@@ -87,17 +92,20 @@ struct LayerWs {
 
 int64_t sel_pitch(int64_t k_sel) { return round_up(k_sel, 64); }
 
-// A 1x1 convolution without padding is the linear layer on the [B*H*W, Cin] matrix.
-bool spatial_conv(const efqat_layer_desc* l) { return l->is_conv && (l->R != 1 || l->S != 1 || l->pad != 0); }
+// A 1x1 convolution with stride 1 and no padding is the linear layer on the [B*H*W, Cin] matrix.
+bool spatial_conv(const efqat_layer_desc* l) {
+  return l->is_conv && (l->R != 1 || l->S != 1 || l->pad != 0 || l->stride != 1);
+}
 
 ConvArgs conv_args(const efqat_layer_desc* l, int mode) {
   ConvArgs c = {};
   c.mode = mode;
   c.B = l->B; c.H = l->H; c.W = l->W; c.Cin = l->Cin;
-  c.Ho = l->H + 2 * l->pad - l->R + 1;
-  c.Wo = l->W + 2 * l->pad - l->S + 1;
+  c.Ho = static_cast<int>(conv_out(l->H, l->R, l->pad, l->stride));
+  c.Wo = static_cast<int>(conv_out(l->W, l->S, l->pad, l->stride));
   c.N = static_cast<int>(l->N);
   c.R = l->R; c.S = l->S; c.pad = l->pad;
+  c.stride = l->stride;
   return c;
 }
 
@@ -105,11 +113,20 @@ int64_t x_elems(const efqat_layer_desc* l) {
   return spatial_conv(l) ? static_cast<int64_t>(l->B) * l->H * l->W * l->Cin : l->M * l->K;
 }
 
+// (dS_x, dZ_x) partial pairs of the grad-input launches: for a convolution, one launch per class
+// of input pixels (stride x stride classes), each tiled by its own pixel box.
 int dx_partials(const efqat_layer_desc* l) {
   if (!spatial_conv(l)) return gemm_dx_num_partials(l->M, l->K);
-  int tw, th, tb;
-  conv_pixel_box(l->W, l->H, l->B, 128, &tw, &th, &tb);
-  return static_cast<int>(ceil_div(l->W, tw) * ceil_div(l->H, th) * ceil_div(l->B, tb) * ceil_div(l->Cin, 64) * 8);
+  int64_t n = 0;
+  for (int ah = 0; ah < l->stride; ++ah)
+    for (int aw = 0; aw < l->stride; ++aw) {
+      const int64_t Wc = ceil_div(l->W - aw, l->stride), Hc = ceil_div(l->H - ah, l->stride);
+      if (Wc < 1 || Hc < 1) continue;
+      int tw, th, tb;
+      conv_pixel_box(static_cast<int>(Wc), static_cast<int>(Hc), l->B, 128, &tw, &th, &tb);
+      n += ceil_div(Wc, tw) * ceil_div(Hc, th) * ceil_div(l->B, tb) * ceil_div(l->Cin, 64) * 8;
+    }
+  return static_cast<int>(n);
 }
 
 LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, int64_t p_elems_override) {
@@ -524,8 +541,29 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
     g.X = X; g.x_dtype = layer->act_dtype;
     g.partials = w.dxpart;
     g.status = ctx->d_status;
-    rc = timed_gemm(ctx, 1, g, st, &tiles, &dx_grid);
-    if (rc != EFQAT_OK) return rc;
+    if (!sconv) {
+      rc = timed_gemm(ctx, 1, g, st, &tiles, &dx_grid);
+      if (rc != EFQAT_OK) return rc;
+    } else {
+      // One launch per class of input pixels (a single class for stride 1).  Classes that no
+      // filter tap reaches (a 1x1 filter with stride 2 reads one pixel in four) get no launch:
+      // their gradient is zero, written by one fill of dX beforehand.
+      if (layer->stride > 1 && (layer->R < layer->stride || layer->S < layer->stride)) {
+        if (cudaMemsetAsync(dX, 0, static_cast<size_t>(x_elems(layer)) * (act_bf16 ? 2 : 4), st) != cudaSuccess)
+          return EFQAT_ERR_CUDA;
+      }
+      for (int ah = 0; ah < layer->stride; ++ah)
+        for (int aw = 0; aw < layer->stride; ++aw) {
+          cv_dx.cls_h = ah;
+          cv_dx.cls_w = aw;
+          g.partials = w.dxpart + 2 * static_cast<int64_t>(tiles);
+          int t1 = 0, g1 = 0;
+          rc = timed_gemm(ctx, 1, g, st, &t1, &g1);
+          if (rc != EFQAT_OK) return rc;
+          tiles += t1;
+          if (g1 > dx_grid) dx_grid = g1;
+        }
+    }
   }
   // a6: weight gradient of the unfrozen channels only, as split partial products
   if (k_sel > 0) {

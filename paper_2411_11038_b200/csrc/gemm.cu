@@ -36,6 +36,7 @@ static const int GEMM_THREADS = 64 + 32 * EPI_WARPS;
 static const int ACC_STRIDE = 256;              // TMEM columns between the two accumulators
 static const int TMEM_COLS = 512;
 static const int HB_BYTES = 32 * 64;            // staging block of one epilogue warp: 32 rows x 64 B
+static const int MAX_TAPS = 49;                // filter taps of one launch (7 x 7)
 static const double L2_PANEL_BYTES = 32.0 * 1024 * 1024;   // operand slice kept resident in L2 by the tile order
 
 // Convolution geometry as the kernel needs it (mode 0 = plain matrices).
@@ -44,9 +45,16 @@ struct ConvP {
   int tw, th, tb;           // pixel box: one 128-row tile (modes 1, 2) or one 64-row contraction block (mode 3)
   int tiles_w, tiles_h;     // boxes along W and H (boxes along B follow from the tile / block count)
   int dimH, dimB;           // extent of the tiled pixel space in H and B (store / load guards)
-  int R, S, pad;
   int C;                    // channels of the 4-D A tensor (Cin for modes 1 and 3, N for mode 2)
-  int cchunks;              // 64-channel chunks of C
+  int cchunks;              // 64-channel chunks of C (the last one zero-filled past C by the TMA unit)
+  int wcols;                // columns of one filter tap in the weight matrix (= Cin)
+  // Filter taps of this launch.  Tap t reads the A tensor through map tap_map[t] (strided
+  // convolutions see the input as stride x stride interleaved sub-grids, one tensor map each)
+  // with its pixel box shifted by (tap_dw[t], tap_dh[t]); tap_rs[t] = r * S + s is its position
+  // in the filter.  Grad-input launches carry only the taps that reach their pixel class.
+  int ntaps;
+  int8_t tap_dh[MAX_TAPS], tap_dw[MAX_TAPS];
+  uint8_t tap_map[MAX_TAPS], tap_rs[MAX_TAPS];
 };
 
 struct GemmParams {
@@ -65,6 +73,7 @@ struct GemmParams {
   int splits;
   int tiles_m, tiles_n;
   int panel_dir, panel;   // order of the tiles in the work list (see tile_coords)
+  int hint_a, hint_b;     // L2 eviction policy of the A / B operand loads (plain matrices): see ptx::l2_policy
   int blk_cols;       // output columns per 64-byte staging row: 32 (bf16) or 16 (fp32)
   int out_bufs;       // staging buffers per epilogue warp (2 when shared memory allows)
   const float* col_scale;
@@ -132,7 +141,8 @@ template <int A_MN, int B_MN, int EPI, int CTA2>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmX,
-            const GemmParams p) {
+            const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
+            const __grid_constant__ CUtensorMap tmA3, const GemmParams p) {
   constexpr bool FWD = (EPI == EPI_FWD || EPI == EPI_FWD_I8);   // forward epilogue (scale, bias)
   constexpr bool I8 = (EPI == EPI_FWD_I8);                       // ... on 8-bit integer operands
   extern __shared__ uint8_t smem_raw[];
@@ -172,6 +182,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     prefetch_tmap(&tmB);
     if (EPI != EPI_PART) prefetch_tmap(&tmOut);
     if (EPI == EPI_DX) prefetch_tmap(&tmX);
+    if (p.cv.mode == 1 || p.cv.mode == 3) {
+      prefetch_tmap(&tmA1);
+      prefetch_tmap(&tmA2);
+      prefetch_tmap(&tmA3);
+    }
   }
   if (warp == 1) {
     if (CTA2) {
@@ -206,6 +221,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     {
       int it = 0;
       bool live = true;
+      const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
       for (int w = unit; w < total_items && live; w += num_units) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
         int tm, tn;
@@ -253,13 +269,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int chunk_stride = p.kps * CHUNK_BYTES;
             if (a_mrg && lane < 2) {
               const int c = lane;
-              if (CTA2) tma_load_2d_pair(a_reg + c * chunk_stride, &tmA, fb, m0 + 64 * c, kb0 * BK);
-              else tma_load_2d(a_reg + c * chunk_stride, &tmA, &ctl->full[s], m0 + 64 * c, kb0 * BK);
+              if (CTA2) tma_load_2d_pair_hint(a_reg + c * chunk_stride, &tmA, fb, m0 + 64 * c, kb0 * BK, pol_a);
+              else tma_load_2d_hint(a_reg + c * chunk_stride, &tmA, &ctl->full[s], m0 + 64 * c, kb0 * BK, pol_a);
             }
             if (b_mrg && lane >= 2 && lane - 2 < b_chunks) {
               const int c = lane - 2;
-              if (CTA2) tma_load_2d_pair(b_reg + c * chunk_stride, &tmB, fb, n0 + 64 * c, kb0 * BK);
-              else tma_load_2d(b_reg + c * chunk_stride, &tmB, &ctl->full[s], n0 + 64 * c, kb0 * BK);
+              if (CTA2) tma_load_2d_pair_hint(b_reg + c * chunk_stride, &tmB, fb, n0 + 64 * c, kb0 * BK, pol_b);
+              else tma_load_2d_hint(b_reg + c * chunk_stride, &tmB, &ctl->full[s], n0 + 64 * c, kb0 * BK, pol_b);
             }
           }
           const int u = (lane - 8) >> 1;
@@ -272,33 +288,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (CTA2) {
               if (do_a) {
                 if (A_MN) {
-                  tma_load_2d_pair(sa, &tmA, fb, m0, kb * BK);
-                  tma_load_2d_pair(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK);
+                  tma_load_2d_pair_hint(sa, &tmA, fb, m0, kb * BK, pol_a);
+                  tma_load_2d_pair_hint(sa + CHUNK_BYTES, &tmA, fb, m0 + 64, kb * BK, pol_a);
                 } else {
-                  tma_load_2d_pair(sa, &tmA, fb, kb * p.bk, m0);
+                  tma_load_2d_pair_hint(sa, &tmA, fb, kb * p.bk, m0, pol_a);
                 }
               } else {
                 if (B_MN) {
                   for (int c = 0; c < b_chunks; ++c)
-                    tma_load_2d_pair(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK);
+                    tma_load_2d_pair_hint(sb + c * CHUNK_BYTES, &tmB, fb, n0 + 64 * c, kb * BK, pol_b);
                 } else {
-                  tma_load_2d_pair(sb, &tmB, fb, kb * p.bk, n0);
+                  tma_load_2d_pair_hint(sb, &tmB, fb, kb * p.bk, n0, pol_b);
                 }
               }
             } else if (p.cv.mode == 0) {
               if (do_a) {
                 if (A_MN) {
-                  tma_load_2d(sa, &tmA, &ctl->full[s], m0, kb * BK);
-                  tma_load_2d(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK);
+                  tma_load_2d_hint(sa, &tmA, &ctl->full[s], m0, kb * BK, pol_a);
+                  tma_load_2d_hint(sa + CHUNK_BYTES, &tmA, &ctl->full[s], m0 + 64, kb * BK, pol_a);
                 } else {
-                  tma_load_2d(sa, &tmA, &ctl->full[s], kb * p.bk, m0);
+                  tma_load_2d_hint(sa, &tmA, &ctl->full[s], kb * p.bk, m0, pol_a);
                 }
               } else {
                 if (B_MN) {
                   for (int c = 0; c < b_chunks; ++c)
-                    tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK);
+                    tma_load_2d_hint(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], n0 + 64 * c, kb * BK, pol_b);
                 } else {
-                  tma_load_2d(sb, &tmB, &ctl->full[s], kb * p.bk, n0);
+                  tma_load_2d_hint(sb, &tmB, &ctl->full[s], kb * p.bk, n0, pol_b);
                 }
               }
             } else if (p.cv.mode == 3) {
@@ -307,12 +323,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               const int bb = kb / (p.cv.tiles_w * p.cv.tiles_h);
               const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
               if (do_a) {
+                const int cpad = p.cv.cchunks * 64;       // tile rows per tap (channels padded to 64)
                 for (int j = 0; j < 2; ++j) {
                   const int k = m0 + 64 * j;
-                  int rs = k / p.cv.C, c = k - rs * p.cv.C;
-                  if (rs >= p.cv.R * p.cv.S) { rs = 0; c = p.cv.C; }     // past the last tap: all zeros
-                  const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
-                  tma_load_4d(sa + j * CHUNK_BYTES, &tmA, &ctl->full[s], c, w0 + sx - p.cv.pad, h0 + r - p.cv.pad, b0);
+                  int t = k / cpad, c = k - t * cpad;
+                  if (t >= p.cv.ntaps) { t = 0; c = p.cv.C; }     // past the last tap: all zeros
+                  const int mi = p.cv.tap_map[t];
+                  const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
+                  tma_load_4d(sa + j * CHUNK_BYTES, ma, &ctl->full[s], c, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
                 }
               } else {
                 for (int c = 0; c < b_chunks; ++c)
@@ -324,18 +342,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
               const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
               const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
-              const int rs = kb / p.cv.cchunks, cc = kb - rs * p.cv.cchunks;
-              const int r = rs / p.cv.S, sx = rs - r * p.cv.S;
-              const int dw = (p.cv.mode == 1) ? sx - p.cv.pad : p.cv.pad - sx;
-              const int dh = (p.cv.mode == 1) ? r - p.cv.pad : p.cv.pad - r;
+              const int t = kb / p.cv.cchunks, cc = kb - t * p.cv.cchunks;
+              const int rs = p.cv.tap_rs[t];
               if (do_a) {
-                tma_load_4d(sa, &tmA, &ctl->full[s], cc * 64, w0 + dw, h0 + dh, b0);
-              } else if (B_MN) {     // W^ viewed as [N rows, R*S*Cin columns]: rows = contraction, Nc = Cin
+                const int mi = p.cv.tap_map[t];
+                const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
+                tma_load_4d(sa, ma, &ctl->full[s], cc * 64, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
+              } else if (B_MN) {     // W^ viewed as [N rows, R*S*Cin columns]: rows = contraction
                 for (int c = 0; c < b_chunks; ++c)
-                  tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s],
-                              rs * static_cast<int>(p.Nc) + n0 + 64 * c, cc * 64);
-              } else {               // weight codes [N, R*S*Cin]
-                tma_load_2d(sb, &tmB, &ctl->full[s], rs * p.cv.C + cc * 64, n0);
+                  tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], rs * p.cv.wcols + n0 + 64 * c, cc * 64);
+              } else {               // weight codes [N, R*S*Cin]: columns past this tap's channels meet zeros of A
+                tma_load_2d(sb, &tmB, &ctl->full[s], rs * p.cv.wcols + cc * 64, n0);
               }
             }
           }
@@ -541,7 +558,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       float acc_s = 0.f, acc_c = 0.f;
 
       if (EPI == EPI_PART) {
-        const int64_t row = static_cast<int64_t>(g.row0) + lane;
+        int64_t row = static_cast<int64_t>(g.row0) + lane;
+        if (p.cv.mode == 3) {
+          // tile row (tap, channel padded to 64) -> row of the weight matrix; padding rows are skipped
+          const int cpad = p.cv.cchunks * 64;
+          const int t = static_cast<int>(row) / cpad, c = static_cast<int>(row) - t * cpad;
+          row = (t < p.cv.ntaps && c < p.cv.C) ? static_cast<int64_t>(p.cv.tap_rs[t]) * p.cv.C + c : p.Mr;
+        }
         for (int jb = g.jb0; jb < g.jb1; ++jb) {
           const int c0 = jb * 32;
           uint32_t r[32];
@@ -779,13 +802,21 @@ static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows,
 }
 
 // 4-D NHWC tensor [B,H,W,C] (pitch C elements per pixel); box = row_bytes (128 or 64) of channels x bw x bh x bb pixels.
+// sw / sh / sb: distance in elements between neighbouring pixels along W, H and B (0: dense,
+// i.e. pitch, pitch * W, pitch * W * H).  A strided convolution addresses one of its
+// stride x stride interleaved pixel sub-grids this way: base moved to the sub-grid's first
+// pixel, W and H counted in sub-grid pixels, sw and sh multiplied by the stride.
 static int make_map_4d(CUtensorMap* m, const void* base, int is_bf16, int64_t B, int64_t H, int64_t W, int64_t C,
-                       int64_t pitch, int bw, int bh, int bb, int row_bytes = 128) {
+                       int64_t pitch, int bw, int bh, int bb, int row_bytes = 128, int64_t sw = 0, int64_t sh = 0,
+                       int64_t sb = 0) {
   const int es = is_bf16 ? 2 : 4;
+  if (!sw) sw = pitch;
+  if (!sh) sh = pitch * W;
+  if (!sb) sb = pitch * W * H;
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(W), static_cast<cuuint64_t>(H),
                               static_cast<cuuint64_t>(B)};
-  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(pitch) * es, static_cast<cuuint64_t>(pitch) * W * es,
-                                 static_cast<cuuint64_t>(pitch) * W * H * es};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(sw) * es, static_cast<cuuint64_t>(sh) * es,
+                                 static_cast<cuuint64_t>(sb) * es};
   const cuuint32_t box[4] = {static_cast<cuuint32_t>(row_bytes / es), static_cast<cuuint32_t>(bw),
                              static_cast<cuuint32_t>(bh), static_cast<cuuint32_t>(bb)};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
@@ -871,11 +902,11 @@ int gemm_choose_splits(int64_t Mr, int64_t Nc, int64_t Kc, int sm_count) {
 
 template <int A_MN, int B_MN, int EPI, int CTA2>
 static int launch(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to, const CUtensorMap& tx,
-                  const GemmParams& p, int grid, size_t smem, cudaStream_t st) {
+                  const CUtensorMap* tcls, const GemmParams& p, int grid, size_t smem, cudaStream_t st) {
   auto kern = gemm_kernel<A_MN, B_MN, EPI, CTA2>;
   count_launches(1);
-  if (launch_dependent(kern, static_cast<unsigned>(grid), GEMM_THREADS, smem, st, CTA2 ? 2 : 1, ta, tb, to, tx, p) !=
-      cudaSuccess)
+  if (launch_dependent(kern, static_cast<unsigned>(grid), GEMM_THREADS, smem, st, CTA2 ? 2 : 1, ta, tb, to, tx,
+                       tcls[0], tcls[1], tcls[2], p) != cudaSuccess)
     return EFQAT_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
@@ -916,10 +947,46 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   if (p.splits < 1 || p.splits > p.nkb) return EFQAT_ERR_SHAPE;
   p.BN = (a.epi == EPI_PART) ? part_bn(a.Nc) : choose_bn(a.Mr, a.Nc, sm_count);
   const ConvArgs* cv = a.conv;
+  const int cs = cv ? cv->stride : 1;           // convolution stride
+  int cWc = 0, cHc = 0;                         // grad-input: extent of this launch's pixel class
   if (cv) {
-    if (cv->mode < 1 || cv->mode > 3 || (cv->Cin & 63)) return EFQAT_ERR_UNIMPL;
+    if (cv->mode < 1 || cv->mode > 3 || cs < 1 || cs > 2 || cv->R * cv->S > MAX_TAPS) return EFQAT_ERR_UNIMPL;
     if (cv->mode == 2) {           // grad-input tiles must not straddle the end of Cin (B is not zero there)
       p.BN = (cv->Cin % 256 == 0) ? 256 : (cv->Cin % 192 == 0) ? 192 : (cv->Cin % 128 == 0) ? 128 : 64;
+      if (cv->cls_h < 0 || cv->cls_h >= cs || cv->cls_w < 0 || cv->cls_w >= cs) return EFQAT_ERR_SHAPE;
+      cWc = static_cast<int>(ceil_div(cv->W - cv->cls_w, cs));
+      cHc = static_cast<int>(ceil_div(cv->H - cv->cls_h, cs));
+    }
+    // filter taps of this launch
+    ConvP& c = p.cv;
+    c.ntaps = 0;
+    for (int r = 0; r < cv->R; ++r)
+      for (int sx = 0; sx < cv->S; ++sx) {
+        int dh, dw, mi = 0;
+        if (cv->mode == 2) {
+          // input pixel h = cls_h + stride * i receives tap r from output row (h + pad - r) / stride
+          const int nh = cv->cls_h + cv->pad - r, nw = cv->cls_w + cv->pad - sx;
+          if (nh % cs != 0 || nw % cs != 0) continue;
+          dh = nh / cs;
+          dw = nw / cs;
+        } else {
+          // output pixel ho reads input row stride * ho + r - pad = stride * (ho + dh) + class
+          const int oh = r - cv->pad, ow = sx - cv->pad;
+          const int ah = ((oh % cs) + cs) % cs, aw = ((ow % cs) + cs) % cs;
+          dh = (oh - ah) / cs;
+          dw = (ow - aw) / cs;
+          mi = ah * cs + aw;
+        }
+        c.tap_dh[c.ntaps] = static_cast<int8_t>(dh);
+        c.tap_dw[c.ntaps] = static_cast<int8_t>(dw);
+        c.tap_map[c.ntaps] = static_cast<uint8_t>(mi);
+        c.tap_rs[c.ntaps] = static_cast<uint8_t>(r * cv->S + sx);
+        ++c.ntaps;
+      }
+    if (c.ntaps == 0 || (cv->mode == 2 && (cWc < 1 || cHc < 1))) {     // nothing reaches this pixel class
+      if (tiles_out) *tiles_out = 0;
+      if (grid_out) *grid_out = 0;
+      return EFQAT_OK;
     }
   }
   // CTA pairs (256 x BN tiles, tiles full in N) halve the B traffic from L2 per FLOP; they are
@@ -956,9 +1023,9 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   if (cv) {
     ConvP& c = p.cv;
     c.mode = cv->mode;
-    c.R = cv->R; c.S = cv->S; c.pad = cv->pad;
-    // pixel space that is tiled: outputs for forward and grad-weight, inputs for grad-input
-    const int pW = (cv->mode == 2) ? cv->W : cv->Wo, pH = (cv->mode == 2) ? cv->H : cv->Ho;
+    // pixel space that is tiled: outputs for forward and grad-weight, the launch's class of
+    // input pixels for grad-input
+    const int pW = (cv->mode == 2) ? cWc : cv->Wo, pH = (cv->mode == 2) ? cHc : cv->Ho;
     conv_pixel_box(pW, pH, cv->B, cv->mode == 3 ? BK : BM, &c.tw, &c.th, &c.tb);
     c.tiles_w = static_cast<int>(ceil_div(pW, c.tw));
     c.tiles_h = static_cast<int>(ceil_div(pH, c.th));
@@ -966,12 +1033,14 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     c.dimH = pH; c.dimB = cv->B;
     c.C = (cv->mode == 2) ? cv->N : cv->Cin;
     c.cchunks = static_cast<int>(ceil_div(c.C, 64));
+    c.wcols = cv->Cin;
     if (cv->mode == 3) {
       p.nkb = c.tiles_w * c.tiles_h * tiles_b;                 // contraction over boxes of 64 output pixels
       if (p.splits > p.nkb) return EFQAT_ERR_SHAPE;
+      p.tiles_m = static_cast<int>(ceil_div(static_cast<int64_t>(c.ntaps) * c.cchunks * 64, BM));   // rows = (tap, padded channel)
     } else {
       p.tiles_m = c.tiles_w * c.tiles_h * tiles_b;             // one tile per box of 128 pixels
-      p.nkb = cv->R * cv->S * c.cchunks;
+      p.nkb = c.ntaps * c.cchunks;
     }
   }
   // Order of the work list.  One tile reads tile_rows x Kc of A and BN x Kc of B.  With the
@@ -997,6 +1066,13 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       const double t_m = b_all * static_cast<double>(ceil_div(p.tiles_m, gm)) + a_all;   // row panels
       if (t_n <= t_m) { p.panel_dir = 1; p.panel = gn; } else { p.panel_dir = 2; p.panel = gm; }
     }
+    // The panel's operand is asked to stay (L2 evict-last) while the other one streams past with
+    // the normal policy.  Measured on M = 16384, 8192 x 8192 and 4096 x 16384 (grad-input GEMM):
+    // 1.31 -> 1.32 PFLOP/s; marking the streamed operand evict-first costs 5-14 % (a row block is
+    // read by the `panel` tiles of its row at slightly different times), and panels of 16, 24 or
+    // 48 MB instead of 32 are 10-20 % slower.
+    if (p.panel_dir == 1) p.hint_b = 2;
+    else if (p.panel_dir == 2) p.hint_a = 2;
   }
   p.blk_cols = a.out_bf16 ? 32 : 16;
   p.b_stage_bytes = static_cast<int>(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2);
@@ -1035,7 +1111,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   p.status = a.status;
   p.defer_wait = a.defer_wait;
 
-  CUtensorMap ta, tb, to, tx;
+  CUtensorMap ta, tb, to, tx, tcls[3];
   if (a.epi == EPI_DX && (a.x_dtype == EFQAT_BF16) != (a.out_bf16 != 0)) return EFQAT_ERR_DTYPE;
   if (!cv) {
     // MN-major operands: one box = all kps k-blocks of a stage for one 64-wide chunk
@@ -1045,6 +1121,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     if (rc != EFQAT_OK) return rc;
     to = ta;
     tx = ta;
+    tcls[0] = tcls[1] = tcls[2] = ta;
     if (a.epi != EPI_PART) {
       rc = make_map(&to, a.out, a.out_bf16, a.Mr, a.Nc, a.ldo, 32, 64);
       if (rc != EFQAT_OK) return rc;
@@ -1059,21 +1136,36 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     // quarter of a 128-pixel box: the 32 rows one epilogue warp owns
     const int qh = (32 / c.tw < c.th) ? 32 / c.tw : c.th;
     const int qb = 32 / (c.tw * qh);
+    // The input activation tensor seen as stride x stride interleaved sub-grids of pixels: class
+    // (ah, aw) holds the pixels (ah + stride * i, aw + stride * j).
+    const int64_t Ci = cv->Cin, HW = static_cast<int64_t>(cv->H) * cv->W;
+    auto class_map = [&](CUtensorMap* m, const void* base, int is16, int ah, int aw, int bw_, int bh_, int bb_,
+                         int row_bytes) {
+      const int64_t Wc = ceil_div(cv->W - aw, cs), Hc = ceil_div(cv->H - ah, cs);
+      if (Wc < 1 || Hc < 1) return make_map_4d(m, base, is16, cv->B, 1, 1, Ci, Ci, bw_, bh_, bb_, row_bytes, 0, 0,
+                                               Ci * HW);     // empty class: never addressed by a tap
+      const char* b0 = static_cast<const char*>(base) + (static_cast<int64_t>(ah) * cv->W + aw) * Ci * (is16 ? 2 : 4);
+      return make_map_4d(m, b0, is16, cv->B, Hc, Wc, Ci, Ci, bw_, bh_, bb_, row_bytes, cs * Ci, cs * cv->W * Ci, Ci * HW);
+    };
+    if (cv->mode == 1 || cv->mode == 3) {
+      CUtensorMap* maps[4] = {&ta, &tcls[0], &tcls[1], &tcls[2]};
+      for (int i = 0; i < 4 && rc == EFQAT_OK; ++i) {
+        const int ah = (i < cs * cs) ? i / cs : 0, aw = (i < cs * cs) ? i % cs : 0;
+        rc = class_map(maps[i], a.A, 1, ah, aw, c.tw, c.th, c.tb, 128);
+      }
+    }
     if (cv->mode == 1) {
-      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, c.th, c.tb);
       if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, bn_cta);
       if (rc == EFQAT_OK)
         rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, qh, qb, 64);
       tx = ta;
     } else if (cv->mode == 2) {
       rc = make_map_4d(&ta, a.A, 1, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, c.th, c.tb);
+      tcls[0] = tcls[1] = tcls[2] = ta;
       if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, BK);
-      if (rc == EFQAT_OK)
-        rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb, 64);
-      if (rc == EFQAT_OK)
-        rc = make_map_4d(&tx, a.X, a.out_bf16, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, qh, qb, 64);
+      if (rc == EFQAT_OK) rc = class_map(&to, a.out, a.out_bf16, cv->cls_h, cv->cls_w, c.tw, qh, qb, 64);
+      if (rc == EFQAT_OK) rc = class_map(&tx, a.X, a.out_bf16, cv->cls_h, cv->cls_w, c.tw, qh, qb, 64);
     } else {
-      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->H, cv->W, cv->Cin, cv->Cin, c.tw, c.th, c.tb);
       if (rc == EFQAT_OK) rc = make_map_4d(&tb, a.B, 1, cv->B, cv->Ho, cv->Wo, a.Nc, a.ldb, c.tw, c.th, c.tb);
       to = ta;
       tx = ta;
@@ -1089,7 +1181,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * EPI_WARPS;
   if (grid_out) *grid_out = grid;
 
-#define EFQAT_LAUNCH(AM, BMj, E, P2) return launch<AM, BMj, E, P2>(ta, tb, to, tx, p, grid, smem, st)
+#define EFQAT_LAUNCH(AM, BMj, E, P2) return launch<AM, BMj, E, P2>(ta, tb, to, tx, tcls, p, grid, smem, st)
   if (a.epi == EPI_FWD && !a.a_mn && !a.b_mn) {
     if (i8) {
       if (pair) EFQAT_LAUNCH(0, 0, EPI_FWD_I8, 1);

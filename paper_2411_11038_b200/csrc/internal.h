@@ -121,9 +121,10 @@ int run_select(int mode, int L, const efqat_layer_desc* layers, const float* con
 // ---- gemm.cu ------------------------------------------------------------------------
 enum GemmEpi { EPI_FWD = 0, EPI_DX = 1, EPI_PART = 2, EPI_FWD_I8 = 3 };   // EPI_FWD_I8: chosen inside run_gemm
 
-// Implicit-GEMM convolution geometry (stride 1).  The activation operand is read through a
+// Implicit-GEMM convolution geometry (stride 1 or 2).  The activation operand is read through a
 // 4-D tensor map over its NHWC tensor with a box of pixels shifted by the filter tap; pixels
-// that fall into the padding come back as zeros from the TMA unit.
+// that fall into the padding come back as zeros from the TMA unit, and so do channels past the
+// tensor's last one (channel counts that are not multiples of 64).
 //   mode 1 forward : A = Xc [B,H,W,Cin] patches, B = weight codes [N, R*S*Cin], D = Y [B,Ho,Wo,N]
 //   mode 2 grad-in : A = dY [B,Ho,Wo,N] patches, B = W^ [N, R*S*Cin] (MN-major), D = dX [B,H,W,Cin]
 //   mode 3 grad-w  : A = Xc patches (MN-major), B = gathered dY [B,Ho,Wo,pitch] (MN-major),
@@ -133,6 +134,10 @@ struct ConvArgs {
   int B, H, W, Cin;     // input activation tensor
   int Ho, Wo, N;        // output activation tensor
   int R, S, pad;
+  int stride;           // 1 or 2
+  // mode 2 only: the class of input pixels (cls_h + stride * i, cls_w + stride * j) this launch
+  // computes; a strided grad-input is one launch per class, each with the taps that reach it
+  int cls_h, cls_w;
 };
 
 struct GemmArgs {

@@ -145,15 +145,15 @@ def conv_abs_bounds(case, T, s_w, s_x, z_x):
     N, R, S, C = W64.shape
     Bn, H, Wd, _ = X64.shape
     Ho, Wo = dY64.shape[1:3]
-    pad = case.pad
-    P = O._patches(np.abs(qx["deq"]), R, S, 1, pad).reshape(-1, R * S * C)
+    pad, st = case.pad, case.stride
+    P = O._patches(np.abs(qx["deq"]), R, S, st, pad).reshape(-1, R * S * C)
     Yabs = (P @ np.abs(qw["deq"]).reshape(N, -1).T).reshape(Bn, Ho, Wo, N)
     dY2 = np.abs(dY64).reshape(-1, N)
-    Pc = O._patches(np.abs(qx["c0"]), R, S, 1, pad).reshape(-1, R * S * C)
+    Pc = O._patches(np.abs(qx["c0"]), R, S, st, pad).reshape(-1, R * S * C)
     Gw_abs = (float(s_x) * (dY2.T @ Pc)).reshape(N, R, S, C)
     Gp = (dY2 @ np.abs(qw["deq"]).reshape(N, -1)).reshape(Bn, Ho, Wo, R, S, C)
-    Gxp = np.zeros((Bn, H + 2 * pad, Wd + 2 * pad, C))
+    Gxp = np.zeros((Bn, H + 2 * pad + st, Wd + 2 * pad + st, C))
     for r in range(R):
         for s in range(S):
-            Gxp[:, r:r + Ho, s:s + Wo, :] += Gp[:, :, :, r, s, :]
+            Gxp[:, r:r + st * Ho:st, s:s + st * Wo:st, :] += Gp[:, :, :, r, s, :]
     return Yabs, Gxp[:, pad:pad + H, pad:pad + Wd, :], Gw_abs

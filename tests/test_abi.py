@@ -58,7 +58,12 @@ def test_validate_layer_codes(lib):
     assert B.validate_layer(B.layer_desc(128, 32, 16, B.BF16, conv), spec) == 0
     assert B.validate_layer(B.layer_desc(127, 32, 16, B.BF16, conv), spec) == -2
     conv2 = B.ConvGeom(B=2, H=8, W=8, Cin=16, R=3, S=3, stride=2, pad=1)
-    assert B.validate_layer(B.layer_desc(32, 32, 144, B.BF16, conv2), spec) == -9
+    assert B.validate_layer(B.layer_desc(32, 32, 144, B.BF16, conv2), spec) == 0          # 8x8 -> 4x4
+    assert B.validate_layer(B.layer_desc(128, 32, 144, B.BF16, conv2), spec) == -2        # M of stride 1
+    conv3 = B.ConvGeom(B=2, H=8, W=8, Cin=16, R=3, S=3, stride=3, pad=1)
+    assert B.validate_layer(B.layer_desc(18, 32, 144, B.BF16, conv3), spec) == -9         # strides 1 and 2 only
+    conv4 = B.ConvGeom(B=1, H=16, W=16, Cin=8, R=9, S=9, stride=1, pad=4)
+    assert B.validate_layer(B.layer_desc(256, 32, 648, B.BF16, conv4), spec) == -9        # filters up to 7 x 7
 
 
 def test_workspace_queries(lib):

@@ -1,6 +1,10 @@
 """GPU parity of the convolution form of the layer step (implicit GEMM over NHWC tensors,
-stride 1) against the oracle: forward, grad-input with the STE mask and dS_x / dZ_x, and the
-partial grad-weight, including padded borders with a non-zero activation zero point."""
+strides 1 and 2, channel counts that are not multiples of 64, filters up to 7 x 7) against the
+oracle: forward, grad-input with the STE mask and dS_x / dZ_x, and the partial grad-weight,
+including padded borders with a non-zero activation zero point.  The stride-2 cases carry the
+shapes of ResNet-50's stem, of its three stride-2 3x3 convolutions and of its three stride-2
+1x1 shortcut convolutions (Section 4 "Setup": every convolution is quantized, "including the
+input, output, and shortcut layers")."""
 import numpy as np
 import pytest
 import torch
@@ -18,10 +22,10 @@ def ctx():
     return B.Context(0)
 
 
-def _case(name, Bn, H, Wd, Cin, N, R, pad, dtype=torch.bfloat16, w_bits=4, seed=0):
-    Ho, Wo = H + 2 * pad - R + 1, Wd + 2 * pad - R + 1
+def _case(name, Bn, H, Wd, Cin, N, R, pad, dtype=torch.bfloat16, w_bits=4, seed=0, stride=1):
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (Wd + 2 * pad - R) // stride + 1
     return I.LayerCase(name, Bn * Ho * Wo, R * R * Cin, N, act_dtype=dtype, w_bits=w_bits, x_bits=8, w_std=None,
-                       x_abs=True, seed=seed, conv=True, B=Bn, H=H, Wd=Wd, Cin=Cin, R=R, S=R, stride=1, pad=pad)
+                       x_abs=True, seed=seed, conv=True, B=Bn, H=H, Wd=Wd, Cin=Cin, R=R, S=R, stride=stride, pad=pad)
 
 
 CASES = [
@@ -31,6 +35,23 @@ CASES = [
     _case("c3x3_14", 4, 14, 14, 128, 256, 3, 1, seed=4),
     _case("c1x1", 2, 12, 12, 72, 64, 1, 0, seed=5),
     _case("resnet_56_64to256_3x3_b2", 2, 56, 56, 64, 256, 3, 1, seed=6),
+    # channel counts that are not multiples of 64 (zero-filled chunk tails)
+    _case("c3x3_cin72", 2, 10, 9, 72, 80, 3, 1, seed=7),
+    _case("c3x3_cin8_f32", 2, 12, 12, 8, 64, 3, 1, dtype=torch.float32, seed=8),
+    # stride 2: odd and even extents, padded and valid
+    _case("c3x3_s2_odd", 2, 9, 11, 64, 72, 3, 1, seed=9, stride=2),
+    _case("c3x3_s2_valid", 3, 10, 10, 64, 64, 3, 0, seed=10, stride=2),
+    _case("c5x5_s2", 2, 13, 12, 128, 64, 5, 2, w_bits=8, seed=11, stride=2),
+    _case("c1x1_s2", 2, 14, 14, 64, 128, 1, 0, seed=12, stride=2),
+    _case("c2x2_s2", 2, 8, 8, 64, 64, 2, 0, seed=13, stride=2),
+    # ResNet-50: stem (3 input channels padded to 8), stride-2 3x3 of stages 2-4, stride-2 shortcuts
+    _case("resnet_stem_7x7_s2", 1, 224, 224, 8, 64, 7, 3, w_bits=8, seed=14, stride=2),
+    _case("resnet_56_128_3x3_s2", 2, 56, 56, 128, 128, 3, 1, seed=15, stride=2),
+    _case("resnet_28_256_3x3_s2", 2, 28, 28, 256, 256, 3, 1, seed=16, stride=2),
+    _case("resnet_14_512_3x3_s2", 2, 14, 14, 512, 512, 3, 1, seed=17, stride=2),
+    _case("resnet_56_256to512_1x1_s2", 2, 56, 56, 256, 512, 1, 0, seed=18, stride=2),
+    _case("resnet_28_512to1024_1x1_s2", 2, 28, 28, 512, 1024, 1, 0, seed=19, stride=2),
+    _case("resnet_14_1024to2048_1x1_s2", 2, 14, 14, 1024, 2048, 1, 0, seed=20, stride=2),
 ]
 
 
@@ -44,7 +65,7 @@ def test_conv_forward_backward_parity(ctx, case):
     s_x = np.float32(s_x * np.float32(0.8))
     assert float(np.clip(np.rint(z_x), 0, 255)) > 0
     D = U.to_dev(T, s_w, s_x, z_x)
-    geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, 1, case.pad)
+    geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, case.stride, case.pad)
     is_bf16 = case.act_dtype == torch.bfloat16
     Yabs, Gx_abs, Gw_abs = U.conv_abs_bounds(case, T, s_w, s_x, z_x)
 
@@ -52,7 +73,7 @@ def test_conv_forward_backward_parity(ctx, case):
                         False, conv=geom)
     torch.cuda.synchronize()
     assert ctx.device_status() == 0
-    ref = O.conv_forward(X64, W64, s_w, s_x, z_x, b64, case.w_bits, case.x_bits, 1, case.pad)
+    ref = O.conv_forward(X64, W64, s_w, s_x, z_x, b64, case.w_bits, case.x_bits, case.stride, case.pad)
     got = U.np32(Y)
     U.assert_bf16_class(got, ref, case.name + " Y")
     U.assert_fp32_class(got, ref, Yabs + np.abs(b64), case.name + " Y", out_is_bf16=is_bf16)
@@ -69,7 +90,7 @@ def test_conv_forward_backward_parity(ctx, case):
         assert ctx.device_status() == 0
         g = {kk: (U.np32(v) if v is not None else None) for kk, v in out.items()}
         outs.append(g)
-        args = (dY64, X64, W64, s_w, s_x, z_x, idx, case.w_bits, case.x_bits, 1, case.pad)
+        args = (dY64, X64, W64, s_w, s_x, z_x, idx, case.w_bits, case.x_bits, case.stride, case.pad)
         ex = O.conv_backward_efqat(*args, operand_model="exact")
         bm = O.conv_backward_efqat(*args, operand_model="bf16")
         name = f"{case.name} k_sel={k}"

@@ -801,6 +801,12 @@ static int make_map(CUtensorMap* m, const void* base, int is_bf16, int64_t rows,
   return r == CUDA_SUCCESS ? EFQAT_OK : EFQAT_ERR_CUDA;
 }
 
+int tensor_map_2d(CUtensorMap* m, const void* base, int kind, int64_t rows, int64_t cols, int64_t ld, int box_rows,
+                  int row_bytes) {
+  if (!tensor_map_encoder()) return EFQAT_ERR_CUDA;
+  return make_map(m, base, kind, rows, cols, ld, box_rows, row_bytes);
+}
+
 // 4-D NHWC tensor [B,H,W,C] (pitch C elements per pixel); box = row_bytes (128 or 64) of channels x bw x bh x bb pixels.
 // sw / sh / sb: distance in elements between neighbouring pixels along W, H and B (0: dense,
 // i.e. pitch, pitch * W, pitch * W * H).  A strided convolution addresses one of its

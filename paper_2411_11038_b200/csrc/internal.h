@@ -112,6 +112,15 @@ struct CacheArgs {
 };
 void launch_weight_cache(const CacheArgs& a, cudaStream_t st);
 
+// ---- skinny.cu ----------------------------------------------------------------------
+// Forward of a plain layer with a contraction of 64 or 128 in one launch: fake-quant of X as the
+// operand producer, weight codes resident in shared memory, epilogue straight to global memory.
+// W (fp32, quantized in the kernel) or codes16 (the layer cache's bf16 codes) supplies the weights.
+bool skinny_fwd_applies(int64_t M, int64_t N, int64_t K);
+int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X, void* Y, const float* W,
+                   const bf16* codes16, const float* s_w, const float* s_x, const float* z_x, const float* bias,
+                   int w_bits, int x_bits, int x_sym, int* status, int sm_count, cudaStream_t st);
+
 // ---- select.cu ----------------------------------------------------------------------
 size_t select_workspace_bytes(int L, int64_t total_channels);
 int run_select(int mode, int L, const efqat_layer_desc* layers, const float* const* weights, const int64_t* k,
@@ -176,6 +185,10 @@ struct GemmArgs {
   // beside its predecessor (see gemm_kernel)
   int defer_wait;
 };
+// Tiled tensor map over a row-major matrix [rows, cols] with pitch ld (elements): box = row_bytes
+// (128 or 64: the swizzle span) of columns x box_rows rows.  kind: 0 fp32, 1 bf16, 2 8-bit.
+int tensor_map_2d(CUtensorMap* m, const void* base, int kind, int64_t rows, int64_t cols, int64_t ld, int box_rows,
+                  int row_bytes);
 // Number of (dS_x, dZ_x) partial pairs EPI_DX writes for this problem.
 int gemm_dx_num_partials(int64_t Mr, int64_t Nc);
 // Split count along the contraction for EPI_PART.

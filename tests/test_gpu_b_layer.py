@@ -33,6 +33,12 @@ SMALL = [
     _case("int8_asym_bf16", 333, 640, 96, torch.bfloat16, seed=8),
     _case("int8_asym_f32", 200, 512, 64, torch.float32, seed=9),
     _case("int8_sym_w4", 130, 1024, 160, torch.bfloat16, w_bits=4, x_bits=8, sym=True, seed=10),
+    # contractions of 64 / 128 with N % 64 == 0: the one-launch forward with the quantizer as operand producer
+    _case("short_k64_bf16", 1000, 64, 256, torch.bfloat16, w_bits=4, seed=11),
+    _case("short_k128_bf16", 700, 128, 512, torch.bfloat16, w_bits=4, seed=12),
+    _case("short_k64_f32", 300, 64, 64, torch.float32, seed=13),
+    _case("short_k128_ragged_n", 129, 128, 320, torch.bfloat16, seed=14),
+    _case("short_k64_wide", 260, 64, 832, torch.bfloat16, x_bits=4, sym=True, seed=15),
 ]
 
 

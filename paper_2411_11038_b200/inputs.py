@@ -113,6 +113,21 @@ def config3(batch: int = 64) -> List[LayerCase]:
     return out
 
 
+def config3_strided(batch: int = 64) -> List[LayerCase]:
+    """The stride-2 layers of ResNet-50: the 7x7 input layer (3 channels stored as 8), the 3x3
+    stride-2 convolution opening stages 2-4 and the 1x1 stride-2 shortcut beside each."""
+    specs = [("stem", 224, 8, 64, 7, 3), ("56_128_3x3", 56, 128, 128, 3, 1), ("28_256_3x3", 28, 256, 256, 3, 1),
+             ("14_512_3x3", 14, 512, 512, 3, 1), ("56_256to512_1x1", 56, 256, 512, 1, 0),
+             ("28_512to1024_1x1", 28, 512, 1024, 1, 0), ("14_1024to2048_1x1", 14, 1024, 2048, 1, 0)]
+    out = []
+    for i, (name, hw, cin, cout, r, pad) in enumerate(specs):
+        ho = (hw + 2 * pad - r) // 2 + 1
+        out.append(LayerCase(f"cfg3s_{name}_s2", batch * ho * ho, r * r * cin, cout, w_bits=4, x_bits=8, w_std=None,
+                             x_abs=True, seed=3100 + i, conv=True, B=batch, H=hw, Wd=hw, Cin=cin, R=r, S=r,
+                             stride=2, pad=pad))
+    return out
+
+
 def config4(layers: int = 24, M: int = 9216) -> List[LayerCase]:
     """BERT-large-shaped stack: per block Q,K,V,O 1024->1024, FFN 1024->4096->1024."""
     out = []

@@ -24,7 +24,32 @@ from . import inputs as I
 from .clocks import ClockSampler, physical_gpu_index
 
 FRACS = {1: (0.0, 26 / 512, 1.0), 2: (0.0, 0.05, 0.25, 1.0), 3: (0.0, 0.10, 1.0), 4: (0.0, 0.10, 1.0),
-         5: (0.0, 0.01, 0.05, 0.10, 0.25, 0.50, 1.0)}
+         5: (0.0, 0.01, 0.05, 0.10, 0.25, 0.50, 1.0), 6: (0.0, 0.10, 1.0)}
+SGD = (1e-9, 0.9, 1e-4)      # fused update of the unfrozen rows, as in bench.py (rate scaled for unit-variance dY)
+
+
+def load_peaks():
+    """Measured peaks of this machine (burst bf16 GEMM TFLOP/s, copy GB/s); the recipe's fallback otherwise."""
+    import os
+    p = os.path.join(os.path.dirname(os.path.abspath(__file__)), "..", "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["bf16_tflops"]), float(d["hbm_gbs"]), "measured"
+    return 1590.0, 6650.0, "fallback"
+
+
+def bounds(case, k, peaks, fwd_int8=False):
+    """Roofline time (ms) of the forward and of the backward with k unfrozen channels:
+    max(algorithmic flops / tensor peak, algorithmic bytes / copy bandwidth)."""
+    tf, gbs, _ = peaks
+    e = 2 if case.act_dtype == torch.bfloat16 else 4
+    g = 2.0 * case.M * case.N * case.K
+    x_elems = case.B * case.H * case.Wd * case.Cin if case.conv else case.M * case.K
+    fwd_bytes = x_elems * e + case.N * case.K * 4 + case.M * case.N * e
+    bwd_bytes = case.M * case.N * e + x_elems * e + case.N * case.K * 4 + x_elems * e + k * case.K * 4
+    fwd = max(g / (tf * (2.0 if fwd_int8 else 1.0) * 1e9), fwd_bytes / (gbs * 1e6))
+    bwd = max((g + 2.0 * case.M * k * case.K) / (tf * 1e9), bwd_bytes / (gbs * 1e6))
+    return fwd, bwd, fwd_bytes, bwd_bytes
 
 
 class Timer:
@@ -55,7 +80,8 @@ def layer_on_device(ctx, case: I.LayerCase, dev):
     D["s_x"], D["z_x"] = B.init_act_qparams(ctx, D["X"], case.x_bits, case.x_symmetric)
     conv = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, case.stride, case.pad) if case.conv else None
     if conv is not None:
-        Ho, Wo = case.H + 2 * case.pad - case.R + 1, case.Wd + 2 * case.pad - case.S + 1
+        Ho = (case.H + 2 * case.pad - case.R) // case.stride + 1
+        Wo = (case.Wd + 2 * case.pad - case.S) // case.stride + 1
         plan = B.LayerPlan(ctx, case.M, case.N, case.K, case.act_dtype, case.w_bits, case.x_bits, case.x_symmetric,
                            case.N, dev, conv, x_shape=D["X"].shape, y_shape=(case.B, Ho, Wo, case.N))
     else:
@@ -85,21 +111,31 @@ def sweep_layer(ctx, case, fracs, timer, dev, ks=None):
     D, plan = layer_on_device(ctx, case, dev)
     g = 2.0 * case.M * case.N * case.K
     rec = {"layer": case.name, "M": case.M, "N": case.N, "K": case.K, "w_bits": case.w_bits, "x_bits": case.x_bits}
+    peaks = load_peaks()
+    int8 = (not case.conv) and case.K >= 512 and case.K % 16 == 0 and case.N % 32 == 0
     t = timer.ms(lambda: plan.fwd(D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], D["bias"]))
-    rec["fwd_ms"], rec["fwd_tflops"] = t, g / t / 1e9
+    fb, _, fbytes, _ = bounds(case, 0, peaks, int8)
+    rec["fwd_ms"], rec["fwd_tflops"], rec["fwd_int8"] = t, g / t / 1e9, int8
+    rec["fwd_bound_ms"], rec["fwd_frac_of_bound"], rec["fwd_bytes"] = fb, fb / t, fbytes
+    rec["peaks"] = {"tflops": peaks[0], "hbm_gbs": peaks[1], "source": peaks[2]}
     rec["bwd"] = {}
     full_ms = None
+    mom = torch.zeros_like(D["W"])
+    sgd = B.make_sgd(SGD[0], SGD[1], SGD[2], D["W"], mom)
     for f in sorted(set(fracs), reverse=True):
         k = B.ratio_to_k(f, case.N) if ks is None else ks[f]
         sel = B.SelectPlan(ctx, B.CWPL, [D["W"]], [k])
         sel.run()
         idx = sel.idx[:k] if 0 < k < case.N else None
-        t = timer.ms(lambda: plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True))
+        t = timer.ms(lambda: plan.bwd(D["dY"], D["X"], D["W"], D["s_w"], D["s_x"], D["z_x"], idx, k, want_db=True,
+                                      sgd=sgd))
         if f == 1.0:
             full_ms = t
+        _, bb, _, bbytes = bounds(case, k, peaks)
         rec["bwd"][f"{f:.4g}"] = {"k_sel": k, "ms": t, "tflops": (g + 2.0 * case.M * k * case.K) / t / 1e9,
                                   "speedup_vs_full_qat": (full_ms / t) if full_ms else None,
-                                  "ideal": 2.0 / (1.0 + k / case.N)}
+                                  "ideal": 2.0 / (1.0 + k / case.N), "bound_ms": bb, "frac_of_bound": bb / t,
+                                  "bytes": bbytes}
     sel = B.SelectPlan(ctx, B.CWPL, [D["W"]], [B.ratio_to_k(0.05, case.N)])
     t = timer.ms(sel.run)
     rec["select_ms"], rec["select_gbs"] = t, case.N * case.K * 4 / t / 1e6
@@ -151,13 +187,44 @@ def sweep_layerwise(ctx, timer, dev):
             "layers": [c.name for c in cases], "unfrozen_layers": k_l, "channels_per_layer": counts}
 
 
+def print_markdown(path):
+    """Results table of a finished sweep: one row per layer, times in ms, fractions of the
+    roofline bound max(flops / tensor peak, bytes / copy bandwidth) of the measured peaks."""
+    recs = [json.loads(l) for l in open(path) if l.strip()]
+    print("| config | layer (M, N, K) | fwd ms (TFLOP/s; of bound) | bwd ms by unfrozen % (TFLOP/s; of bound) | "
+          "speed-up vs own full-QAT bwd (ideal) | SM MHz median (min); reasons |")
+    print("|---|---|---|---|---|---|")
+    for r in recs:
+        if "bwd" not in r:
+            continue
+        b = r["bwd"]
+        keys = sorted(b, key=float)
+        bw = " · ".join(f"{float(f) * 100:.3g}%: {b[f]['ms']:.3f} ({b[f]['tflops']:.0f}; {b[f]['frac_of_bound']:.2f})"
+                        for f in keys)
+        sp = " · ".join(f"{float(f) * 100:.3g}%: {b[f]['speedup_vs_full_qat']:.2f}x ({b[f]['ideal']:.2f})"
+                        for f in keys if float(f) < 1.0 and b[f]["speedup_vs_full_qat"])
+        c = r.get("clocks", {})
+        clk = f"{c.get('sm_mhz')} ({c.get('sm_min_mhz')}); {','.join(c.get('reasons', [])) or 'none'}"
+        tag = " int8" if r.get("fwd_int8") else ""
+        print(f"| {r['config']} | {r['layer']} ({r['M']}, {r['N']}, {r['K']}) | {r['fwd_ms']:.3f} ({r['fwd_tflops']:.0f}{tag}; "
+              f"{r['fwd_frac_of_bound']:.2f}) | {bw} | {sp} | {clk} |")
+    for r in recs:
+        if "bwd" not in r:
+            print()
+            print(json.dumps({k: v for k, v in r.items() if k != "clocks"}), "clocks:", json.dumps(r.get("clocks")))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--configs", default="1,2,3,4,5")
+    ap.add_argument("--configs", default="1,2,3,6,4,5", help="6 = the stride-2 layers of ResNet-50")
+    ap.add_argument("--markdown", default=None, help="print the results table of a finished sweep (JSONL file) and exit")
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--out", default=None)
     ap.add_argument("--only", default=None, help="run only layers whose name contains this string")
     args = ap.parse_args()
+    if args.markdown:
+        print_markdown(args.markdown)
+        return
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     ctx = B.Context(0)
@@ -167,7 +234,7 @@ def main():
         if cfg == 4:
             recs = sweep_network(ctx, timer, dev)
         else:
-            cases = {1: I.config1, 2: I.config2, 3: I.config3, 5: I.config5}[cfg]()
+            cases = {1: I.config1, 2: I.config2, 3: I.config3, 5: I.config5, 6: I.config3_strided}[cfg]()
             if cfg == 5:
                 cases = cases + I.config5(4, 4)
             recs = []

@@ -242,6 +242,11 @@ typedef struct {
 int efqat_qparam_adam(efqat_ctx* ctx, const efqat_adam* opt, const efqat_qparam_state* state, int64_t N,
                       const int32_t* idx, int64_t k_sel, const float* dS_w_sel, const float* dS_x,
                       const float* dZ_x, efqat_stream_t stream);
+/* efqat_qparam_adam over the layers of a network in one call (HOST arrays of length L: the
+ * per-layer states; layers[l] supplies N, idx, k_sel, dS_w_sel, dS_x, dZ_x; a layer with the
+ * symmetric activation quantizer leaves its zero point alone). */
+int efqat_network_qparam_adam(efqat_ctx* ctx, const efqat_adam* opt, int L, const efqat_net_layer* layers,
+                              const efqat_qparam_state* states, efqat_stream_t stream);
 /* theta[i] = log2(s[i]) for i < n (Appendix A.2). */
 int efqat_log2_scale_init(efqat_ctx* ctx, const float* s, float* theta, int64_t n, efqat_stream_t stream);
 

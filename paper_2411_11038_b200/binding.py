@@ -30,6 +30,7 @@ EXPORTS = [
     "efqat_selftest_bounded_wait", "efqat_qparam_adam", "efqat_log2_scale_init",
     "efqat_weight_cache_bytes", "efqat_weight_cache_update", "efqat_fq_linear_fwd_cached",
     "efqat_fq_linear_bwd_cached", "efqat_network_fwd", "efqat_network_bwd", "efqat_network_cache_update",
+    "efqat_network_qparam_adam",
 ]
 
 
@@ -126,6 +127,7 @@ def load() -> C.CDLL:
                                                vp, i64, vp, vp, vp, vp, vp, vp, C.POINTER(Sgd), vp, sz, vp, sz, vp]
     for nm in ("efqat_network_fwd", "efqat_network_bwd", "efqat_network_cache_update"):
         getattr(lib, nm).argtypes = [vp, i32, C.POINTER(NetLayer), vp]
+    lib.efqat_network_qparam_adam.argtypes = [vp, C.POINTER(Adam), i32, C.POINTER(NetLayer), C.POINTER(QParamState), vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("efqat_status_string", "efqat_ratio_to_k", "efqat_launch_count"):
@@ -447,6 +449,16 @@ class NetworkPlan:
     def cache_update(self):
         _check(load().efqat_network_cache_update(self.ctx.handle, self.L, self.arr, _stream()),
                "efqat_network_cache_update")
+
+    def qparam_adam(self, qopts: Sequence["QParamOptimizer"]):
+        """efqat_network_qparam_adam: one Adam step on every layer's quantization parameters (the
+        optimizers must share their hyper-parameters; their step counters advance together)."""
+        if not hasattr(self, "_states"):
+            self._states = (QParamState * self.L)(*[q.state for q in qopts])
+        for q in qopts:
+            q.opt.step += 1
+        _check(load().efqat_network_qparam_adam(self.ctx.handle, C.byref(qopts[0].opt), self.L, self.arr, self._states,
+                                                _stream()), "efqat_network_qparam_adam")
 
 
 def _plan_for(ctx, X, W, w_bits, x_bits, x_symmetric, k_sel_max, conv):

@@ -774,6 +774,19 @@ int efqat_qparam_adam(efqat_ctx* ctx, const efqat_adam* opt, const efqat_qparam_
   return last_error();
 }
 
+int efqat_network_qparam_adam(efqat_ctx* ctx, const efqat_adam* opt, int L, const efqat_net_layer* layers,
+                              const efqat_qparam_state* states, efqat_stream_t stream) {
+  if (!ctx || !opt || !layers || !states) return EFQAT_ERR_NULL;
+  if (L < 1) return EFQAT_ERR_SHAPE;
+  for (int l = 0; l < L; ++l) {
+    const efqat_net_layer& n = layers[l];
+    const int rc = efqat_qparam_adam(ctx, opt, &states[l], n.layer.N, n.idx, n.k_sel, n.dS_w_sel, n.dS_x,
+                                     n.q.x_symmetric ? nullptr : n.dZ_x, stream);
+    if (rc != EFQAT_OK) return rc;
+  }
+  return EFQAT_OK;
+}
+
 int efqat_log2_scale_init(efqat_ctx* ctx, const float* s, float* theta, int64_t n, efqat_stream_t stream) {
   if (!ctx || !s || !theta) return EFQAT_ERR_NULL;
   if (n < 1) return EFQAT_ERR_SHAPE;

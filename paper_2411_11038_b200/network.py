@@ -153,14 +153,7 @@ class EfqatNetwork:
         """Adam on the quantization parameters of every layer, then the cache rows of the channels
         whose weights or scales have just moved."""
         if self.qopts:
-            for l, (plan, q) in enumerate(zip(self.plans, self.qopts)):
-                e = self.net.arr[l]
-                k = int(e.k_sel)
-                idx = None
-                if 0 < k < self.N[l]:
-                    o = self.offsets_host[l]
-                    idx = self.net.idx[o:o + k]
-                q.step(idx, k, plan.dS_w_sel, plan.dS_x, plan.dZ_x if q.z_x is not None else None)
+            self.net.qparam_adam(self.qopts)
         if self.use_cache:
             self.net.cache_update()
 

@@ -39,17 +39,10 @@ __device__ __forceinline__ int layer_of_row(const LayerEntry* __restrict__ table
   return lo;
 }
 
-// |x| widened to fp64, exactly.  For normal numbers the widening is bit arithmetic (exponent
-// re-biased by 1023 - 127, mantissa moved up by 29 bits) on the integer pipes; the conversion
-// instruction, which issues at a fraction of their rate, is kept for zeros, denormals and
-// non-finite values.
-__device__ __forceinline__ double absd(float x) {
-  const uint32_t b = __float_as_uint(x) & 0x7fffffffu;
-  if (b - 0x00800000u < 0x7f000000u)
-    return __hiloint2double(static_cast<int>((b >> 3) + 0x38000000u), static_cast<int>(b << 29));
-  return static_cast<double>(__uint_as_float(b));
+__device__ __forceinline__ double abs4(const float4 a) {
+  return (static_cast<double>(fabsf(a.x)) + static_cast<double>(fabsf(a.y))) +
+         (static_cast<double>(fabsf(a.z)) + static_cast<double>(fabsf(a.w)));
 }
-__device__ __forceinline__ double abs4(const float4 a) { return (absd(a.x) + absd(a.y)) + (absd(a.z) + absd(a.w)); }
 
 // One warp per output channel: sum |w| over the row in fp64, key = fl32(sum / K).
 __global__ void __launch_bounds__(256) row_importance_kernel(const LayerEntry* __restrict__ table, int L,
@@ -85,7 +78,7 @@ __global__ void __launch_bounds__(256) row_importance_kernel(const LayerEntry* _
       }
       for (; i < n4; i += 32) acc += abs4(__ldg(w4 + i));
     } else {
-      for (int i = lane; i < e.K; i += 32) acc += absd(w[i]);
+      for (int i = lane; i < e.K; i += 32) acc += static_cast<double>(fabsf(w[i]));
     }
     acc = warp_sum(acc);
     if (lane == 0) {

@@ -16,7 +16,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libefqat.so")
-SOURCES = ["api.cu", "gemm.cu", "elementwise.cu", "select.cu", "noalloc.cu", "fused.cu", "selftest.cu", "optim.cu", "cache.cu", "skinny.cu"]
+SOURCES = ["api.cu", "gemm.cu", "elementwise.cu", "select.cu", "noalloc.cu", "fused.cu", "selftest.cu", "optim.cu", "cache.cu", "skinny.cu", "skinny_bwd.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 

@@ -129,6 +129,11 @@ int dx_partials(const efqat_layer_desc* l) {
   return static_cast<int>(n);
 }
 
+// Layers whose backward runs in one pass over dY and X (skinny_bwd.cu).
+bool one_pass_bwd(const efqat_layer_desc* l) {
+  return !spatial_conv(l) && skinny_bwd_applies(l->M, l->N, l->K, l->act_dtype == EFQAT_BF16);
+}
+
 LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, int64_t p_elems_override) {
   LayerWs w = {};
   char* base = ws ? reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 255) & ~uintptr_t(255)) : nullptr;
@@ -147,6 +152,7 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   w.pitch = gathered ? sel_pitch(k_sel) : N;
   w.dYsel = reinterpret_cast<bf16*>(take(gathered ? M * w.pitch * 2 : 0));
   w.splits = k_sel > 0 ? gemm_choose_splits(K, gathered ? round_up(k_sel, 16) : N, M, sm_count) : 1;
+  if (k_sel > 0 && one_pass_bwd(l)) w.splits = skinny_bwd_grid(M, sm_count);     // one partial product per CTA
   const int64_t p_elems = p_elems_override >= 0 ? p_elems_override : static_cast<int64_t>(w.splits) * k_sel * K;
   w.P = reinterpret_cast<float*>(take(p_elems * 4));
   w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(dx_partials(l)) * 8));
@@ -363,7 +369,8 @@ int efqat_workspace_bytes(const efqat_layer_desc* layer, const efqat_qspec* q, i
   int64_t p_max = 0;
   for (int64_t k = 1; k <= k_sel_max; ++k) {
     const int64_t nc = (k < layer->N) ? round_up(k, 16) : layer->N;
-    const int64_t e = static_cast<int64_t>(gemm_choose_splits(layer->K, nc, layer->M, sm)) * k * layer->K;
+    const int64_t sp = one_pass_bwd(layer) ? skinny_bwd_grid(layer->M, sm) : gemm_choose_splits(layer->K, nc, layer->M, sm);
+    const int64_t e = sp * k * layer->K;
     if (e > p_max) p_max = e;
   }
   // dYsel is largest for the largest gathered k
@@ -513,6 +520,27 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   const int act_bf16 = layer->act_dtype == EFQAT_BF16;
 
   const bool gathered = k_sel > 0 && k_sel < N;
+  if (one_pass_bwd(layer)) {
+    // short contraction: one launch reads dY and X once and leaves per-CTA partials for the finalize launch
+    const int grid = skinny_bwd_grid(M, ctx->sm_count);
+    rc = run_skinny_bwd(M, N, dY, X, dX, W, cache ? wc.what : nullptr, s_w, q->w_bits, s_x, z_x, q->x_bits,
+                        q->x_symmetric, gathered ? idx : nullptr, k_sel, w.P, db_or_null ? w.colsum : nullptr, w.dxpart,
+                        ctx->d_status, ctx->sm_count, st);
+    if (rc != EFQAT_OK) return rc;
+    FinArgs fa = {};
+    fa.N = N; fa.K = K; fa.k_sel = k_sel;
+    fa.P = w.P; fa.splits = grid; fa.split_stride = k_sel * K;
+    fa.W = W; fa.s_w = s_w; fa.s_x = s_x; fa.w_bits = q->w_bits;
+    fa.idx = gathered ? idx : nullptr;
+    fa.dW_sel = dW_sel; fa.dS_w_sel = dS_w_sel;
+    if (opt_or_null) fa.opt = *opt_or_null;
+    fa.has_opt = opt_or_null != nullptr;
+    fa.dx_partials = w.dxpart; fa.n_partials = grid * 8; fa.dS_x = dS_x; fa.dZ_x = dZ_x;
+    fa.colsum_ws = w.colsum; fa.slabs = grid; fa.db = db_or_null;
+    fa.status = ctx->d_status;
+    launch_finalize(fa, st);
+    return last_error();
+  }
   // a2: one launch: dequantised weight operand, activation codes (only when some channel is
   // unfrozen) and one pass over dY (column-sum partials, gathered columns, bf16 copy)
   const bf16* dYb = act_bf16 ? static_cast<const bf16*>(dY) : w.dYb;

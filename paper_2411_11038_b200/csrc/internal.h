@@ -121,6 +121,20 @@ int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X,
                    const bf16* codes16, const float* s_w, const float* s_x, const float* z_x, const float* bias,
                    int w_bits, int x_bits, int x_sym, int* status, int sm_count, cudaStream_t st);
 
+// ---- skinny_bwd.cu ------------------------------------------------------------------
+// Backward of a plain bf16 layer with K = 64 and N = 128 or 256 in one pass over dY and X: grad
+// input with the STE epilogue, the weight-gradient partial of every CTA (rows of the channels idx
+// only: P [grid][k_sel][64], raw sums) and the column sums of dY (colsum [grid][N], may be null),
+// dS_x / dZ_x partials (dxpart [grid * 8][2]); grid = skinny_bwd_grid().  The finalize launch
+// sums the per-CTA partials (splits = slabs = grid).  W (fp32) or what (cached bf16 W^) supplies
+// the weights.
+bool skinny_bwd_applies(int64_t M, int64_t N, int64_t K, int act_bf16);
+int skinny_bwd_grid(int64_t M, int sm_count);
+int run_skinny_bwd(int64_t M, int64_t N, const void* dY, const void* X, void* dX, const float* W, const bf16* what,
+                   const float* s_w, int w_bits, const float* s_x, const float* z_x, int x_bits, int x_sym,
+                   const int32_t* idx, int64_t k_sel, float* P, float* colsum, float* dxpart, int* status,
+                   int sm_count, cudaStream_t st);
+
 // ---- select.cu ----------------------------------------------------------------------
 size_t select_workspace_bytes(int L, int64_t total_channels);
 int run_select(int mode, int L, const efqat_layer_desc* layers, const float* const* weights, const int64_t* k,

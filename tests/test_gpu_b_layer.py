@@ -39,6 +39,10 @@ SMALL = [
     _case("short_k64_f32", 300, 64, 64, torch.float32, seed=13),
     _case("short_k128_ragged_n", 129, 128, 320, torch.bfloat16, seed=14),
     _case("short_k64_wide", 260, 64, 832, torch.bfloat16, x_bits=4, sym=True, seed=15),
+    # ... and with N = 128 / 256 the backward in one pass over dY and X
+    _case("short_k64_n128", 517, 64, 128, torch.bfloat16, seed=16),
+    _case("short_k64_n256_sym", 300, 64, 256, torch.bfloat16, w_bits=4, x_bits=4, sym=True, seed=17),
+    _case("short_k64_many_tiles", 40000, 64, 256, torch.bfloat16, w_bits=4, seed=18),
 ]
 
 

@@ -106,31 +106,51 @@ skinny_bwd_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constan
   }
   pdl_trigger();
   pdl_wait();
+  __syncthreads();                                       // barriers are initialised
+  const int my_tiles = (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  // The first tile's copies need nothing of the set-up below: they travel while it runs.
+  if (tid == 0 && my_tiles > 0) {
+    const int t = blockIdx.x;
+    mbar_arrive_expect_tx(&ctl->x_full, T16K);
+    tma_load_2d(xraw_t, &tmX, &ctl->x_full, 0, t * SB_ROWS);
+    for (int h = 0; h < a.nh; ++h) {
+      mbar_arrive_expect_tx(&ctl->full[h], HALF_BYTES);
+      tma_load_2d(ring + h * HALF_BYTES, &tmDY, &ctl->full[h], h * 128, t * SB_ROWS);
+      tma_load_2d(ring + h * HALF_BYTES + T16K, &tmDY, &ctl->full[h], h * 128 + 64, t * SB_ROWS);
+    }
+  }
 
-  // ---- resident operands: W^ = bf16(s_w q_w) (Eq. 3) and the ones tile
+  // ---- resident operands: W^ = bf16(s_w q_w) (Eq. 3), one thread per channel with the whole row's
+  // loads in flight at once (this phase is a chain of L2 round trips, not bandwidth), and the ones tile
   bool bad_scale = false;
-  for (int p = tid; p < a.N * 8; p += SB_THREADS) {
-    const int n = p >> 3, j = p & 7;
-    const int64_t g = static_cast<int64_t>(n) * 64 + j * 8;
-    uint4 o;
+  for (int n = tid - 32; n >= 0 && n < a.N; n += SB_THREADS - 32) {
     if (a.what) {
-      o = __ldg(reinterpret_cast<const uint4*>(a.what + g));
+      uint4 o[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o[j] = __ldg(reinterpret_cast<const uint4*>(a.what + static_cast<int64_t>(n) * 64) + j);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(what_t + sw128(n, j)) = o[j];
     } else {
+      float4 w4[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) w4[j] = __ldg(reinterpret_cast<const float4*>(a.W + static_cast<int64_t>(n) * 64) + j);
       float sw = __ldg(a.s_w + n);
       if (!scale_ok(sw)) {
         bad_scale = true;
         sw = 1.f;
       }
       const RowQ rq = make_rowq(sw, a.w_bits);
-      const float4 w0 = __ldg(reinterpret_cast<const float4*>(a.W + g));
-      const float4 w1 = __ldg(reinterpret_cast<const float4*>(a.W + g) + 1);
-      const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-      float d[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) d[i] = __fmul_rn(rq.s, quant_weight(w[i], rq).c0);
-      o = make_uint4(pk2b(d[0], d[1]), pk2b(d[2], d[3]), pk2b(d[4], d[5]), pk2b(d[6], d[7]));
+      for (int j = 0; j < 8; ++j) {
+        const float w[8] = {w4[2 * j].x, w4[2 * j].y, w4[2 * j].z, w4[2 * j].w,
+                            w4[2 * j + 1].x, w4[2 * j + 1].y, w4[2 * j + 1].z, w4[2 * j + 1].w};
+        float d[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) d[i] = __fmul_rn(rq.s, quant_weight(w[i], rq).c0);
+        *reinterpret_cast<uint4*>(what_t + sw128(n, j)) =
+            make_uint4(pk2b(d[0], d[1]), pk2b(d[2], d[3]), pk2b(d[4], d[5]), pk2b(d[6], d[7]));
+      }
     }
-    *reinterpret_cast<uint4*>(what_t + sw128(n, j)) = o;
   }
   for (int p = tid; p < SB_ROWS * 8; p += SB_THREADS) {
     const int r = p >> 3, j = p & 7;
@@ -151,14 +171,13 @@ skinny_bwd_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   volatile int* abort_flag = &ctl->abort_flag;
-  const int my_tiles = (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      int it = 0;
+      int it = a.nh;                                     // tile 0 was requested before the set-up
       bool live = true;
-      for (int n = 0; n < my_tiles && live; ++n) {
+      for (int n = 1; n < my_tiles && live; ++n) {
         const int t = blockIdx.x + n * gridDim.x;
         if (*abort_flag || !mbar_wait(&ctl->x_empty, (n & 1) ^ 1)) { live = false; break; }
         mbar_arrive_expect_tx(&ctl->x_full, T16K);

@@ -136,7 +136,8 @@ int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_des
  * s_w [N], s_x [1], z_x [1] (ignored when x_symmetric), bias [N] or NULL; Y in act_dtype.
  * Plain layers with 512 <= K <= 32768, K % 16 == 0 and N % 32 == 0 contract the 8-bit codes
  * on the integer tensor cores (int32 accumulation: the integer sum is exact); all others
- * contract the same integers held in bf16, with fp32 accumulation. */
+ * contract the same integers held in bf16, with fp32 accumulation.  Plain layers with K = 64
+ * and N % 64 == 0 run in a single launch that reads X and writes Y once. */
 int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
                         const float* W, const float* s_w, const float* s_x, const float* z_x,
                         const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream);
@@ -148,7 +149,9 @@ int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efq
  * or k_sel == N); dW_sel fp32 [k_sel, K] with row i <-> channel idx[i];
  * dS_w_sel fp32 [k_sel].  k_sel == N is the ordinary QAT backward; k_sel == 0 does no
  * weight-gradient work at all.  dW_sel carries the weight quantizer's clip mask.
- * opt_or_null != NULL applies the fused SGD-momentum update to rows idx of opt->W_inout. */
+ * opt_or_null != NULL applies the fused SGD-momentum update to rows idx of opt->W_inout.
+ * Plain bf16 layers with K = 64 and N = 128 or 256 take a one-pass form that reads dY and X
+ * once whatever k_sel is. */
 int efqat_fq_linear_bwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY,
                         const void* X, const float* W, const float* s_w, const float* s_x, const float* z_x,
                         const int32_t* idx, int64_t k_sel, void* dX, float* dW_sel, float* dS_w_sel,

@@ -269,6 +269,272 @@ __global__ void __launch_bounds__(SK_THREADS, 2) skinny_fwd_kernel(const __grid_
   if (warp == 0) tmem_dealloc(tmem_base, a.tmem_cols);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// The same forward as a persistent, warp-specialised kernel for bf16 activations and up to 256
+// output columns: one CTA per SM, warp 0 brings raw X tiles into a ring with TMA, warps 2..9 turn
+// each tile into centred codes (Eq. 1) in one of two operand buffers and run the epilogue of the
+// previous tile, warp 1 issues the MMAs into one of two TMEM accumulators.  Load, quantizer, MMA
+// and epilogue of neighbouring tiles overlap inside the CTA, so a tile costs what its bytes cost.
+const int WS_THREADS = 320;
+const int WS_STAGES = 3;
+const int WS_T16K = SK_ROWS * 128;
+
+struct __align__(16) WsCtl {
+  uint64_t full[WS_STAGES], empty[WS_STAGES];
+  uint64_t xc_full[2], xc_empty[2];
+  uint64_t acc_full[2], acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(WS_THREADS, 1)
+skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
+                     const SkinnyFwdArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* b_tile = smem;                                  // [BN rows][128 B] weight codes, K-major
+  uint8_t* xc_t = b_tile + a.BN * 128;                     // [2][128 rows][128 B] centred activation codes
+  uint8_t* ring = xc_t + 2 * WS_T16K;                      // [WS_STAGES][128 rows][128 B] raw X tiles
+  uint8_t* stage = ring + WS_STAGES * WS_T16K;             // [8 warps][2][32 rows][128 B] output staging
+  float* sc = reinterpret_cast<float*>(stage + 8 * 2 * 4096);   // [BN] s_x * s_w[n]
+  float* bi = sc + a.BN;                                   // [BN] bias[n]
+  WsCtl* ctl = reinterpret_cast<WsCtl*>(bi + a.BN);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n0 = blockIdx.y * a.BN;
+  int bn = static_cast<int>(a.N - n0);
+  if (bn > a.BN) bn = a.BN;
+  if (tid == 0) {
+    for (int s = 0; s < WS_STAGES; ++s) {
+      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->empty[s], 8);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&ctl->xc_full[b], 8);
+      mbar_init(&ctl->xc_empty[b], 1);
+      mbar_init(&ctl->acc_full[b], 1);
+      mbar_init(&ctl->acc_empty[b], 8);
+    }
+    mbar_init(&ctl->drain, 1);
+    ctl->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmX);
+    prefetch_tmap(&tmY);
+  }
+  if (warp == 1) {
+    tmem_alloc(&ctl->tmem_base, 512);
+    tmem_relinquish();
+  }
+  pdl_trigger();
+  pdl_wait();
+  __syncthreads();
+  const int my_tiles = (a.tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  // the first tiles travel while the weights are quantized
+  if (tid == 0) {
+    for (int n = 0; n < my_tiles && n < WS_STAGES; ++n) {
+      mbar_arrive_expect_tx(&ctl->full[n], WS_T16K);
+      tma_load_2d(ring + n * WS_T16K, &tmX, &ctl->full[n], 0, (blockIdx.x + n * gridDim.x) * SK_ROWS);
+    }
+  }
+  bool bad_scale = false;
+  for (int n = tid - 32; n >= 0 && n < a.BN; n += WS_THREADS - 32) {
+    if (n >= bn) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(b_tile + sw128_off(n, j)) = make_uint4(0u, 0u, 0u, 0u);
+      sc[n] = 0.f;
+      bi[n] = 0.f;
+      continue;
+    }
+    float sw = __ldg(a.s_w + n0 + n);
+    if (!scale_ok(sw)) {
+      bad_scale = true;
+      sw = 1.f;
+    }
+    if (a.codes16) {
+      uint4 o[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o[j] = __ldg(reinterpret_cast<const uint4*>(a.codes16 + static_cast<int64_t>(n0 + n) * 64) + j);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(b_tile + sw128_off(n, j)) = o[j];
+    } else {
+      float4 w4[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) w4[j] = __ldg(reinterpret_cast<const float4*>(a.W + static_cast<int64_t>(n0 + n) * 64) + j);
+      const RowQ rq = make_rowq(sw, a.w_bits);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float w[8] = {w4[2 * j].x, w4[2 * j].y, w4[2 * j].z, w4[2 * j].w,
+                            w4[2 * j + 1].x, w4[2 * j + 1].y, w4[2 * j + 1].z, w4[2 * j + 1].w};
+        float c[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) c[i] = quant_weight(w[i], rq).c0;
+        *reinterpret_cast<uint4*>(b_tile + sw128_off(n, j)) =
+            make_uint4(pk(c[0], c[1]), pk(c[2], c[3]), pk(c[4], c[5]), pk(c[6], c[7]));
+      }
+    }
+    sc[n] = sw;                        // s_x folded in below, once it is known
+    bi[n] = a.bias ? __ldg(a.bias + n0 + n) : 0.f;
+  }
+  bool bad_x;
+  const ActQ xq = make_actq(a.s_x, a.z_x, a.x_bits, a.x_sym, &bad_x);
+  if ((bad_scale || (bad_x && tid == 0)) && blockIdx.x == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
+  __syncthreads();
+  for (int n = tid; n < a.BN; n += WS_THREADS) sc[n] *= xq.s;
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool live = true;
+      int n = WS_STAGES;
+      for (; n < my_tiles && live; ++n) {
+        const int s = n % WS_STAGES;
+        if (*abort_flag || !mbar_wait(&ctl->empty[s], ((n / WS_STAGES) & 1) ^ 1)) { live = false; break; }
+        mbar_arrive_expect_tx(&ctl->full[s], WS_T16K);
+        tma_load_2d(ring + s * WS_T16K, &tmX, &ctl->full[s], 0, (blockIdx.x + n * gridDim.x) * SK_ROWS);
+      }
+      if (!live) {
+        record_status(a.status, EFQAT_DEV_WAIT_TIMEOUT);
+        *abort_flag = 1;
+        const int issued = n < my_tiles ? n : my_tiles;
+        for (int j = (issued > WS_STAGES ? issued - WS_STAGES : 0); j < issued; ++j)
+          mbar_wait(&ctl->full[j % WS_STAGES], (j / WS_STAGES) & 1, 20000000ull);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(SK_ROWS, bn, 0, 0);
+      const uint32_t b_addr = smem_u32(b_tile);
+      bool ok = true;
+      for (int n = 0; n < my_tiles && ok; ++n) {
+        const int b = n & 1;
+        if (*abort_flag || !mbar_wait(&ctl->acc_empty[b], ((n >> 1) & 1) ^ 1)) { ok = false; break; }
+        if (*abort_flag || !mbar_wait(&ctl->xc_full[b], (n >> 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(xc_t + b * WS_T16K);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16(tmem_base + b * 256, smem_desc_sw128(a_addr + k * 32, 16, 1024),
+                    smem_desc_sw128(b_addr + k * 32, 16, 1024), idesc, k ? 1u : 0u);
+        umma_commit(&ctl->acc_full[b]);
+        umma_commit(&ctl->xc_empty[b]);
+      }
+      if (!ok) {
+        record_status(a.status, EFQAT_DEV_WAIT_TIMEOUT);
+        *abort_flag = 1;
+        umma_commit(&ctl->drain);
+        mbar_wait(&ctl->drain, 0, 20000000ull);
+      }
+    }
+  } else {
+    const int e = warp - 2, q = warp & 3, h = e >> 2;
+    const int row = q * 32 + lane;
+    const float c_lo = xq.lo - xq.zr, c_hi = xq.hi - xq.zr;
+    int st_it = 0;
+    bool ok = true;
+    // Eq. 1 on this lane's 32 values (row `row`, 64-byte half h) of tile number n
+    auto quant_tile = [&](int n) -> bool {
+      const int s = n % WS_STAGES, b = n & 1;
+      bool g = *abort_flag ? false : mbar_wait(&ctl->full[s], (n / WS_STAGES) & 1);
+      if (!__all_sync(0xffffffffu, g)) return false;
+      uint4 xr[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const uint4*>(ring + s * WS_T16K + sw128_off(row, h * 4 + i));
+      fence_proxy_async();           // the bulk copy that refills the stage is ordered behind these reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctl->empty[s]);
+      g = *abort_flag ? false : mbar_wait(&ctl->xc_empty[b], ((n >> 1) & 1) ^ 1);
+      if (!__all_sync(0xffffffffu, g)) return false;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t wv[4] = {xr[i].x, xr[i].y, xr[i].z, xr[i].w};
+        float c[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          c[2 * j] = __uint_as_float(wv[j] << 16);
+          c[2 * j + 1] = __uint_as_float(wv[j] & 0xffff0000u);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c[j] = fminf(fmaxf(rne_small(__fmul_rn(c[j], xq.rinv)), c_lo), c_hi);
+        *reinterpret_cast<uint4*>(xc_t + b * WS_T16K + sw128_off(row, h * 4 + i)) =
+            make_uint4(pk(c[0], c[1]), pk(c[2], c[3]), pk(c[4], c[5]), pk(c[6], c[7]));
+      }
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctl->xc_full[b]);
+      return true;
+    };
+    if (my_tiles > 0) ok = quant_tile(0);
+    const int rounds = bn / 64;                              // 128-byte rounds of output columns
+    const int rd0 = h ? (rounds + 1) / 2 : 0, rd1 = h ? rounds : (rounds + 1) / 2;
+    for (int n = 0; n < my_tiles && ok; ++n) {
+      const int t = blockIdx.x + n * gridDim.x;
+      const int b = n & 1;
+      if (n + 1 < my_tiles) {
+        ok = quant_tile(n + 1);
+        if (!ok) break;
+      }
+      bool g = *abort_flag ? false : mbar_wait(&ctl->acc_full[b], (n >> 1) & 1);
+      if (!__all_sync(0xffffffffu, g)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256;
+      for (int rd = rd0; rd < rd1; ++rd, ++st_it) {
+        const int c0 = rd * 64;
+        uint8_t* stg = stage + (e * 2 + (st_it & 1)) * 4096;
+        uint32_t r[64];
+        tmem_ld_32x32(t_row + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld_32x32(t_row + c0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+        if (lane == 0) tma_store_wait_read1();
+        tmem_wait_ld();
+        if (rd + 1 == rd1) {                                  // the accumulator is in registers: hand it back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&ctl->acc_empty[b]);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int gi = 0; gi < 8; ++gi) {
+          const float4 s0 = *reinterpret_cast<const float4*>(sc + c0 + gi * 8);
+          const float4 s1 = *reinterpret_cast<const float4*>(sc + c0 + gi * 8 + 4);
+          const float4 b0 = *reinterpret_cast<const float4*>(bi + c0 + gi * 8);
+          const float4 b1 = *reinterpret_cast<const float4*>(bi + c0 + gi * 8 + 4);
+          const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+          const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+          float v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = fmaf(__uint_as_float(r[gi * 8 + j]), sv[j], bv[j]);
+          *reinterpret_cast<uint4*>(stg + sw128_off(lane, gi)) =
+              make_uint4(pk(v[0], v[1]), pk(v[2], v[3]), pk(v[4], v[5]), pk(v[6], v[7]));
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          if (static_cast<int64_t>(t) * SK_ROWS + q * 32 < a.M) tma_store_2d(&tmY, stg, n0 + c0, t * SK_ROWS + q * 32);
+          tma_store_commit();
+        }
+      }
+      if (rd0 >= rd1) {                                       // a warp without columns still returns the accumulator
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctl->acc_empty[b]);
+      }
+    }
+    if (!ok && lane == 0) {
+      record_status(a.status, EFQAT_DEV_WAIT_TIMEOUT);
+      *abort_flag = 1;
+    }
+    if (lane == 0) tma_store_wait_all();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
 }  // namespace
 
 // A contraction of 64: weight codes, operand tile and staging of two CTAs fit one SM.  At 128 the
@@ -293,6 +559,33 @@ int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X,
   a.s_w = s_w; a.s_x = s_x; a.z_x = z_x; a.bias = bias;
   a.w_bits = w_bits; a.x_bits = x_bits; a.x_sym = x_sym;
   a.status = status;
+  if (act_bf16 && K == 64) {
+    // persistent warp-specialised form: one CTA per SM and column chunk
+    CUtensorMap tmX, tmY;
+    if (tensor_map_2d(&tmX, X, 1, M, 64, 64, SK_ROWS, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
+    if (tensor_map_2d(&tmY, Y, 1, M, N, N, 32, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
+    const size_t smem = static_cast<size_t>(a.BN) * 128 + 2 * WS_T16K + WS_STAGES * WS_T16K + 8 * 2 * 4096 +
+                        2 * a.BN * sizeof(float) + sizeof(WsCtl);
+    if (cudaFuncSetAttribute(skinny_fwd_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+        cudaSuccess)
+      return EFQAT_ERR_CUDA;
+    int ctas = sm_count / chunks;
+    if (ctas < 1) ctas = 1;
+    if (ctas > a.tiles) ctas = a.tiles;
+    count_launches(1);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas), static_cast<unsigned>(chunks));
+    cfg.blockDim = dim3(WS_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, skinny_fwd_ws_kernel, tmX, tmY, a) != cudaSuccess) return EFQAT_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
+  }
   const int kb = a.K / 64;
   // CTAs per SM: as many as TMEM holds (512 columns); the shared-memory request is padded so that
   // no further CTA becomes resident and then waits for TMEM columns

@@ -92,3 +92,29 @@ def test_null_context_is_rejected_before_any_launch(lib):
     code = C.c_int(0)
     assert lib.efqat_device_status(None, C.byref(code)) == -1
     assert lib.efqat_destroy(None) == -1
+
+
+def test_weight_cache_and_network_queries(lib):
+    """Host-side behaviour of the cache / network entry points: sizes, and errors found before any launch."""
+    spec = B.QSpec(8, 8, 0)
+    big = B.layer_desc(4096, 768, 768, B.BF16)            # forward on 8-bit codes: 1 + 2 bytes per weight + row sums
+    small = B.layer_desc(4096, 520, 256, B.BF16)          # forward on bf16 codes: 2 + 2 bytes per weight
+    nb, ns = B.weight_cache_bytes(big, spec), B.weight_cache_bytes(small, spec)
+    assert 3 * 768 * 768 + 4 * 768 <= nb <= 3 * 768 * 768 + 4 * 768 + 4096
+    assert 4 * 520 * 256 <= ns <= 4 * 520 * 256 + 4096
+    out = C.c_size_t(0)
+    assert lib.efqat_weight_cache_bytes(C.byref(B.layer_desc(0, 8, 8, B.BF16)), C.byref(spec), C.byref(out)) == -2
+    assert lib.efqat_weight_cache_bytes(C.byref(big), C.byref(spec), None) == -1
+    assert lib.efqat_weight_cache_update(None, C.byref(big), C.byref(spec), None, None, None, 0, None, 0, None) == -1
+    assert lib.efqat_fq_linear_fwd_cached(None, C.byref(big), C.byref(spec), None, None, None, None, None, None,
+                                          None, 0, None, 0, None) == -1
+    assert lib.efqat_fq_linear_bwd_cached(None, C.byref(big), C.byref(spec), None, None, None, None, None, None,
+                                          None, 0, None, None, None, None, None, None, None, None, 0, None, 0,
+                                          None) == -1
+    for fn in (lib.efqat_network_fwd, lib.efqat_network_bwd, lib.efqat_network_cache_update):
+        assert fn(None, 1, None, None) == -1
+    adam = B.Adam(1e-6, 0.9, 0.999, 1e-8, 1, 0)
+    assert lib.efqat_network_qparam_adam(None, C.byref(adam), 1, None, None, None) == -1
+    # workspace of a layer that takes the one-pass backward: one partial product per CTA
+    skinny = B.layer_desc(200704, 256, 64, B.BF16)
+    assert B.workspace_bytes(skinny, spec, 256) >= 148 * 256 * 64 * 4

@@ -137,7 +137,8 @@ int efqat_select_channels(efqat_ctx* ctx, int mode, int L, const efqat_layer_des
  * Plain layers with 512 <= K <= 32768, K % 16 == 0 and N % 32 == 0 contract the 8-bit codes
  * on the integer tensor cores (int32 accumulation: the integer sum is exact); all others
  * contract the same integers held in bf16, with fp32 accumulation.  Plain layers with K = 64
- * and N % 64 == 0 run in a single launch that reads X and writes Y once. */
+ * (and, for bf16 activations, K = 128) and N % 64 == 0 run in a single launch that reads X
+ * and writes Y once. */
 int efqat_fq_linear_fwd(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* X,
                         const float* W, const float* s_w, const float* s_x, const float* z_x,
                         const float* bias_or_null, void* Y, void* ws, size_t ws_bytes, efqat_stream_t stream);

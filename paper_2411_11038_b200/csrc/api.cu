@@ -439,7 +439,7 @@ int fwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
 
   const int act_bf16 = layer->act_dtype == EFQAT_BF16;
   // short contractions (HBM-bound layers): one launch, X and Y touched once
-  if (!spatial_conv(layer) && skinny_fwd_applies(M, N, K)) {
+  if (!spatial_conv(layer) && skinny_fwd_applies(M, N, K, act_bf16)) {
     rc = run_skinny_fwd(M, N, K, act_bf16, X, Y, W, cache ? wc.codes16 : nullptr, s_w, s_x, z_x, bias_or_null,
                         q->w_bits, q->x_bits, q->x_symmetric, ctx->d_status, ctx->sm_count, st);
     return rc != EFQAT_OK ? rc : last_error();

@@ -116,7 +116,7 @@ void launch_weight_cache(const CacheArgs& a, cudaStream_t st);
 // Forward of a plain layer with a contraction of 64 or 128 in one launch: fake-quant of X as the
 // operand producer, weight codes resident in shared memory, epilogue straight to global memory.
 // W (fp32, quantized in the kernel) or codes16 (the layer cache's bf16 codes) supplies the weights.
-bool skinny_fwd_applies(int64_t M, int64_t N, int64_t K);
+bool skinny_fwd_applies(int64_t M, int64_t N, int64_t K, int act_bf16);
 int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X, void* Y, const float* W,
                    const bf16* codes16, const float* s_w, const float* s_x, const float* z_x, const float* bias,
                    int w_bits, int x_bits, int x_sym, int* status, int sm_count, cudaStream_t st);

@@ -38,6 +38,7 @@ struct SkinnyFwdArgs {
   const float* s_w; const float* s_x; const float* z_x; const float* bias;
   int w_bits, x_bits, x_sym;
   int* status;
+  int stages, stg_bufs;             // persistent form: X tiles in flight, staging buffers per epilogue warp
 };
 
 // 16-byte piece j (0..7) of row r inside a [rows x 64 bf16] tile in the canonical K-major
@@ -277,11 +278,11 @@ __global__ void __launch_bounds__(SK_THREADS, 2) skinny_fwd_kernel(const __grid_
 // previous tile, warp 1 issues the MMAs into one of two TMEM accumulators.  Load, quantizer, MMA
 // and epilogue of neighbouring tiles overlap inside the CTA, so a tile costs what its bytes cost.
 const int WS_THREADS = 320;
-const int WS_STAGES = 3;
+const int WS_MAX_STAGES = 3;
 const int WS_T16K = SK_ROWS * 128;
 
 struct __align__(16) WsCtl {
-  uint64_t full[WS_STAGES], empty[WS_STAGES];
+  uint64_t full[WS_MAX_STAGES], empty[WS_MAX_STAGES];
   uint64_t xc_full[2], xc_empty[2];
   uint64_t acc_full[2], acc_empty[2];
   uint64_t drain;
@@ -289,15 +290,18 @@ struct __align__(16) WsCtl {
   int abort_flag;
 };
 
+template <int KB /* 64-wide k-blocks of the contraction: 1 or 2 */>
 __global__ void __launch_bounds__(WS_THREADS, 1)
 skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
                      const SkinnyFwdArgs a) {
+  constexpr int TILE = KB * WS_T16K;                       // one X tile / one operand buffer
+  const int WS_STAGES = a.stages;
   extern __shared__ __align__(1024) uint8_t smem[];
-  uint8_t* b_tile = smem;                                  // [BN rows][128 B] weight codes, K-major
-  uint8_t* xc_t = b_tile + a.BN * 128;                     // [2][128 rows][128 B] centred activation codes
-  uint8_t* ring = xc_t + 2 * WS_T16K;                      // [WS_STAGES][128 rows][128 B] raw X tiles
-  uint8_t* stage = ring + WS_STAGES * WS_T16K;             // [8 warps][2][32 rows][128 B] output staging
-  float* sc = reinterpret_cast<float*>(stage + 8 * 2 * 4096);   // [BN] s_x * s_w[n]
+  uint8_t* b_tile = smem;                                  // [KB][BN rows][128 B] weight codes, K-major
+  uint8_t* xc_t = b_tile + KB * a.BN * 128;                // [2][KB][128 rows][128 B] centred activation codes
+  uint8_t* ring = xc_t + 2 * TILE;                         // [stages][KB][128 rows][128 B] raw X tiles
+  uint8_t* stage = ring + WS_STAGES * TILE;                // [8 warps][stg_bufs][32 rows][128 B] output staging
+  float* sc = reinterpret_cast<float*>(stage + 8 * a.stg_bufs * 4096);   // [BN] s_x * s_w[n]
   float* bi = sc + a.BN;                                   // [BN] bias[n]
   WsCtl* ctl = reinterpret_cast<WsCtl*>(bi + a.BN);
 
@@ -333,15 +337,17 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   // the first tiles travel while the weights are quantized
   if (tid == 0) {
     for (int n = 0; n < my_tiles && n < WS_STAGES; ++n) {
-      mbar_arrive_expect_tx(&ctl->full[n], WS_T16K);
-      tma_load_2d(ring + n * WS_T16K, &tmX, &ctl->full[n], 0, (blockIdx.x + n * gridDim.x) * SK_ROWS);
+      mbar_arrive_expect_tx(&ctl->full[n], TILE);
+      for (int kb = 0; kb < KB; ++kb)
+        tma_load_2d(ring + n * TILE + kb * WS_T16K, &tmX, &ctl->full[n], kb * 64, (blockIdx.x + n * gridDim.x) * SK_ROWS);
     }
   }
   bool bad_scale = false;
   for (int n = tid - 32; n >= 0 && n < a.BN; n += WS_THREADS - 32) {
     if (n >= bn) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(b_tile + sw128_off(n, j)) = make_uint4(0u, 0u, 0u, 0u);
+      for (int j = 0; j < 8 * KB; ++j)
+        *reinterpret_cast<uint4*>(b_tile + (j >> 3) * a.BN * 128 + sw128_off(n, j & 7)) = make_uint4(0u, 0u, 0u, 0u);
       sc[n] = 0.f;
       bi[n] = 0.f;
       continue;
@@ -352,24 +358,26 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       sw = 1.f;
     }
     if (a.codes16) {
-      uint4 o[8];
+      uint4 o[8 * KB];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) o[j] = __ldg(reinterpret_cast<const uint4*>(a.codes16 + static_cast<int64_t>(n0 + n) * 64) + j);
+      for (int j = 0; j < 8 * KB; ++j)
+        o[j] = __ldg(reinterpret_cast<const uint4*>(a.codes16 + static_cast<int64_t>(n0 + n) * (64 * KB)) + j);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4*>(b_tile + sw128_off(n, j)) = o[j];
+      for (int j = 0; j < 8 * KB; ++j) *reinterpret_cast<uint4*>(b_tile + (j >> 3) * a.BN * 128 + sw128_off(n, j & 7)) = o[j];
     } else {
-      float4 w4[16];
+      float4 w4[16 * KB];
 #pragma unroll
-      for (int j = 0; j < 16; ++j) w4[j] = __ldg(reinterpret_cast<const float4*>(a.W + static_cast<int64_t>(n0 + n) * 64) + j);
+      for (int j = 0; j < 16 * KB; ++j)
+        w4[j] = __ldg(reinterpret_cast<const float4*>(a.W + static_cast<int64_t>(n0 + n) * (64 * KB)) + j);
       const RowQ rq = make_rowq(sw, a.w_bits);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 8 * KB; ++j) {
         const float w[8] = {w4[2 * j].x, w4[2 * j].y, w4[2 * j].z, w4[2 * j].w,
                             w4[2 * j + 1].x, w4[2 * j + 1].y, w4[2 * j + 1].z, w4[2 * j + 1].w};
         float c[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) c[i] = quant_weight(w[i], rq).c0;
-        *reinterpret_cast<uint4*>(b_tile + sw128_off(n, j)) =
+        *reinterpret_cast<uint4*>(b_tile + (j >> 3) * a.BN * 128 + sw128_off(n, j & 7)) =
             make_uint4(pk(c[0], c[1]), pk(c[2], c[3]), pk(c[4], c[5]), pk(c[6], c[7]));
       }
     }
@@ -395,8 +403,9 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       for (; n < my_tiles && live; ++n) {
         const int s = n % WS_STAGES;
         if (*abort_flag || !mbar_wait(&ctl->empty[s], ((n / WS_STAGES) & 1) ^ 1)) { live = false; break; }
-        mbar_arrive_expect_tx(&ctl->full[s], WS_T16K);
-        tma_load_2d(ring + s * WS_T16K, &tmX, &ctl->full[s], 0, (blockIdx.x + n * gridDim.x) * SK_ROWS);
+        mbar_arrive_expect_tx(&ctl->full[s], TILE);
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_2d(ring + s * TILE + kb * WS_T16K, &tmX, &ctl->full[s], kb * 64, (blockIdx.x + n * gridDim.x) * SK_ROWS);
       }
       if (!live) {
         record_status(a.status, EFQAT_DEV_WAIT_TIMEOUT);
@@ -416,11 +425,13 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         if (*abort_flag || !mbar_wait(&ctl->acc_empty[b], ((n >> 1) & 1) ^ 1)) { ok = false; break; }
         if (*abort_flag || !mbar_wait(&ctl->xc_full[b], (n >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(xc_t + b * WS_T16K);
+        const uint32_t a_addr = smem_u32(xc_t + b * TILE);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_bf16(tmem_base + b * 256, smem_desc_sw128(a_addr + k * 32, 16, 1024),
-                    smem_desc_sw128(b_addr + k * 32, 16, 1024), idesc, k ? 1u : 0u);
+        for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16(tmem_base + b * 256, smem_desc_sw128(a_addr + kb * WS_T16K + k * 32, 16, 1024),
+                      smem_desc_sw128(b_addr + kb * a.BN * 128 + k * 32, 16, 1024), idesc, (kb | k) ? 1u : 0u);
         umma_commit(&ctl->acc_full[b]);
         umma_commit(&ctl->xc_empty[b]);
       }
@@ -437,21 +448,23 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const float c_lo = xq.lo - xq.zr, c_hi = xq.hi - xq.zr;
     int st_it = 0;
     bool ok = true;
-    // Eq. 1 on this lane's 32 values (row `row`, 64-byte half h) of tile number n
+    // Eq. 1 on this lane's 32 * KB values (row `row`, half h of its pieces) of tile number n
+    constexpr int NP = 4 * KB;                               // 16-byte pieces per lane
+    auto piece_off = [&](int i) { const int p = h * NP + i; return (p >> 3) * WS_T16K + sw128_off(row, p & 7); };
     auto quant_tile = [&](int n) -> bool {
       const int s = n % WS_STAGES, b = n & 1;
       bool g = *abort_flag ? false : mbar_wait(&ctl->full[s], (n / WS_STAGES) & 1);
       if (!__all_sync(0xffffffffu, g)) return false;
-      uint4 xr[4];
+      uint4 xr[NP];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) xr[i] = *reinterpret_cast<const uint4*>(ring + s * WS_T16K + sw128_off(row, h * 4 + i));
+      for (int i = 0; i < NP; ++i) xr[i] = *reinterpret_cast<const uint4*>(ring + s * TILE + piece_off(i));
       fence_proxy_async();           // the bulk copy that refills the stage is ordered behind these reads
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctl->empty[s]);
       g = *abort_flag ? false : mbar_wait(&ctl->xc_empty[b], ((n >> 1) & 1) ^ 1);
       if (!__all_sync(0xffffffffu, g)) return false;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < NP; ++i) {
         const uint32_t wv[4] = {xr[i].x, xr[i].y, xr[i].z, xr[i].w};
         float c[8];
 #pragma unroll
@@ -461,7 +474,7 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) c[j] = fminf(fmaxf(rne_small(__fmul_rn(c[j], xq.rinv)), c_lo), c_hi);
-        *reinterpret_cast<uint4*>(xc_t + b * WS_T16K + sw128_off(row, h * 4 + i)) =
+        *reinterpret_cast<uint4*>(xc_t + b * TILE + piece_off(i)) =
             make_uint4(pk(c[0], c[1]), pk(c[2], c[3]), pk(c[4], c[5]), pk(c[6], c[7]));
       }
       fence_proxy_async();
@@ -485,11 +498,13 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256;
       for (int rd = rd0; rd < rd1; ++rd, ++st_it) {
         const int c0 = rd * 64;
-        uint8_t* stg = stage + (e * 2 + (st_it & 1)) * 4096;
+        uint8_t* stg = stage + (e * a.stg_bufs + (a.stg_bufs == 2 ? (st_it & 1) : 0)) * 4096;
         uint32_t r[64];
         tmem_ld_32x32(t_row + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
         tmem_ld_32x32(t_row + c0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-        if (lane == 0) tma_store_wait_read1();
+        if (lane == 0) {
+          if (a.stg_bufs == 2) tma_store_wait_read1(); else tma_store_wait_read0();
+        }
         tmem_wait_ld();
         if (rd + 1 == rd1) {                                  // the accumulator is in registers: hand it back
           tc_fence_before();
@@ -537,11 +552,9 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 
 }  // namespace
 
-// A contraction of 64: weight codes, operand tile and staging of two CTAs fit one SM.  At 128 the
-// tiles double, one CTA per SM is left, and the general two-launch path measured faster
-// (28 x 28 x 128 -> 512 at batch 64: 46 us against 57 us); the kernel itself handles both.
-bool skinny_fwd_applies(int64_t M, int64_t N, int64_t K) {
-  return M >= 1 && K == 64 && N >= 64 && (N & 63) == 0;
+// Contractions of 64 and, for bf16 activations (the persistent form), 128.
+bool skinny_fwd_applies(int64_t M, int64_t N, int64_t K, int act_bf16) {
+  return M >= 1 && (K == 64 || (K == 128 && act_bf16)) && N >= 64 && (N & 63) == 0;
 }
 
 int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X, void* Y, const float* W,
@@ -559,15 +572,19 @@ int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X,
   a.s_w = s_w; a.s_x = s_x; a.z_x = z_x; a.bias = bias;
   a.w_bits = w_bits; a.x_bits = x_bits; a.x_sym = x_sym;
   a.status = status;
-  if (act_bf16 && K == 64) {
-    // persistent warp-specialised form: one CTA per SM and column chunk
+  if (act_bf16) {
+    // persistent warp-specialised form: one CTA per SM and column chunk.  K = 128 doubles the weight,
+    // operand and ring tiles: two X tiles in flight and one staging buffer per warp then fill the SM.
+    const int kbs = a.K / 64;
+    a.stages = kbs == 1 ? 3 : 2;
+    a.stg_bufs = kbs == 1 ? 2 : 1;
     CUtensorMap tmX, tmY;
-    if (tensor_map_2d(&tmX, X, 1, M, 64, 64, SK_ROWS, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
+    if (tensor_map_2d(&tmX, X, 1, M, K, K, SK_ROWS, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
     if (tensor_map_2d(&tmY, Y, 1, M, N, N, 32, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
-    const size_t smem = static_cast<size_t>(a.BN) * 128 + 2 * WS_T16K + WS_STAGES * WS_T16K + 8 * 2 * 4096 +
+    const size_t smem = static_cast<size_t>(kbs) * a.BN * 128 + (2 + a.stages) * kbs * WS_T16K + 8 * a.stg_bufs * 4096 +
                         2 * a.BN * sizeof(float) + sizeof(WsCtl);
-    if (cudaFuncSetAttribute(skinny_fwd_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
-        cudaSuccess)
+    auto kern = kbs == 1 ? skinny_fwd_ws_kernel<1> : skinny_fwd_ws_kernel<2>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
       return EFQAT_ERR_CUDA;
     int ctas = sm_count / chunks;
     if (ctas < 1) ctas = 1;
@@ -583,7 +600,7 @@ int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X,
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, skinny_fwd_ws_kernel, tmX, tmY, a) != cudaSuccess) return EFQAT_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tmX, tmY, a) != cudaSuccess) return EFQAT_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? EFQAT_OK : EFQAT_ERR_CUDA;
   }
   const int kb = a.K / 64;

@@ -113,6 +113,43 @@ int64_t x_elems(const efqat_layer_desc* l) {
   return spatial_conv(l) ? static_cast<int64_t>(l->B) * l->H * l->W * l->Cin : l->M * l->K;
 }
 
+// Convolutions with few input channels (the 7 x 7 input layer on 8 stored channels): one filter
+// row covers S * Cin <= 64 contiguous elements of an NHWC image row, so a whole filter row is one
+// 64-wide contraction block instead of S blocks that are mostly zero fill.  The forward and the
+// weight-gradient GEMMs then see an R x 1 convolution with S * Cin "channels" on a virtual image
+// whose pixel w starts at stored pixel w (pixels overlap: the pixel pitch stays Cin elements).
+// The horizontal padding cannot come from TMA's out-of-range fill in this view, so the
+// activation codes are written into a zero-framed image [B, H + 2 pad, W + 2 pad, Cin].
+bool narrow_conv(const efqat_layer_desc* l) {
+  return spatial_conv(l) && l->S > 1 && l->S * l->Cin <= 64;
+}
+
+ConvArgs conv_args_x(const efqat_layer_desc* l, int mode) {
+  ConvArgs c = conv_args(l, mode);
+  if (!narrow_conv(l)) return c;
+  const int64_t Hp = l->H + 2 * l->pad, Wp = l->W + 2 * l->pad;
+  c.H = static_cast<int>(Hp);
+  c.W = (c.Wo - 1) * l->stride + 1;          // virtual pixels 0, stride, ... are the first taps of the outputs
+  c.Cin = l->S * l->Cin;
+  c.S = 1;
+  c.pad = 0;
+  c.pix_pitch = l->Cin;
+  c.row_pitch = Wp * l->Cin;
+  c.img_pitch = Hp * Wp * l->Cin;
+  return c;
+}
+
+// elements of the activation-code buffer
+int64_t xc_elems(const efqat_layer_desc* l) {
+  if (!narrow_conv(l)) return x_elems(l);
+  return static_cast<int64_t>(l->B) * (l->H + 2 * l->pad) * (l->W + 2 * l->pad) * l->Cin;
+}
+
+void set_x_layout(PrepArgs* pa, const efqat_layer_desc* l) {
+  if (!narrow_conv(l)) return;
+  pa->xp_C8 = l->Cin / 8; pa->xp_H = l->H; pa->xp_W = l->W; pa->xp_pad = l->pad;
+}
+
 // (dS_x, dZ_x) partial pairs of the grad-input launches: for a convolution, one launch per class
 // of input pixels (stride x stride classes), each tiled by its own pixel box.
 int dx_partials(const efqat_layer_desc* l) {
@@ -145,7 +182,7 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   };
   const int64_t M = l->M, N = l->N, K = l->K;
   w.actq = reinterpret_cast<ActQ*>(take(sizeof(ActQ)));
-  w.Xc = reinterpret_cast<bf16*>(take(x_elems(l) * 2));
+  w.Xc = reinterpret_cast<bf16*>(take(xc_elems(l) * 2));
   w.Wq = reinterpret_cast<bf16*>(take(N * K * 2));
   w.dYb = reinterpret_cast<bf16*>(take(l->act_dtype == EFQAT_F32 ? M * N * 2 : 0));
   const bool gathered = k_sel > 0 && k_sel < N;
@@ -450,6 +487,7 @@ int fwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   pa.W = cache ? nullptr : W; pa.s_w = s_w; pa.w_bits = q->w_bits; pa.Wq = w.Wq;
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric; pa.Xc = w.Xc;
   pa.x_count = x_elems(layer);
+  set_x_layout(&pa, layer);
   pa.status = ctx->d_status;
   // integer forward: the code buffers of the bf16 path are reused, half filled
   const bool i8 = fwd_on_i8(layer);
@@ -475,7 +513,7 @@ int fwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   g.col_scale = s_w; g.col_bias = bias_or_null;
   g.s_x = s_x; g.z_x = z_x; g.x_bits = q->x_bits; g.x_sym = q->x_symmetric;
   if (spatial_conv(layer)) {
-    cva = conv_args(layer, 1);
+    cva = conv_args_x(layer, 1);
     g.conv = &cva;
   }
   g.status = ctx->d_status;
@@ -550,6 +588,7 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   pa.X = X; pa.s_x = s_x; pa.z_x = z_x; pa.x_bits = q->x_bits; pa.x_sym = q->x_symmetric;
   pa.Xc = k_sel > 0 ? w.Xc : nullptr;
   pa.x_count = x_elems(layer);
+  set_x_layout(&pa, layer);
   pa.dY = dY; pa.dYb = act_bf16 ? nullptr : w.dYb;
   pa.colsum_ws = db_or_null ? w.colsum : nullptr;
   pa.idx = idx; pa.k_sel = k_sel; pa.pitch = w.pitch; pa.dYsel = gathered ? w.dYsel : nullptr;
@@ -558,7 +597,7 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   // a4 + a5: dX = (dY W^) masked, with the dS_x / dZ_x partial sums in the epilogue
   int tiles = 0, dx_grid = 0, dw_splits = w.splits;
   const bool sconv = spatial_conv(layer);
-  ConvArgs cv_dx = conv_args(layer, 2), cv_dw = conv_args(layer, 3);
+  ConvArgs cv_dx = conv_args(layer, 2), cv_dw = conv_args_x(layer, 3);
   {
     GemmArgs g = {};
     if (sconv) g.conv = &cv_dx;

@@ -95,8 +95,40 @@ __device__ __forceinline__ void job_quant_x(const PrepArgs& a, int block, int nb
       if (i0 + u * stride < n8) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) v[u][j] = quant_act(v[u][j], p).c0;
-        st8(a.Xc + (i0 + u * stride) * 8, v[u]);
+        int64_t o = i0 + u * stride;
+        if (a.xp_C8) {                     // pixel (b, h, w) goes to (b, h + pad, w + pad) of the padded image
+          const int64_t px = o / a.xp_C8, c8 = o - px * a.xp_C8;
+          const int64_t t = px / a.xp_W, w = px - t * a.xp_W;
+          const int64_t b = t / a.xp_H, h = t - b * a.xp_H;
+          const int64_t Wp = a.xp_W + 2 * a.xp_pad, Hp = a.xp_H + 2 * a.xp_pad;
+          o = ((b * Hp + h + a.xp_pad) * Wp + w + a.xp_pad) * a.xp_C8 + c8;
+        }
+        st8(a.Xc + o * 8, v[u]);
       }
+    }
+  }
+  if (a.xp_C8 && a.xp_pad > 0) {
+    // the zero frame: 2 pad full rows, then 2 pad pixels at the ends of each of the H rows between
+    const int64_t Wp = a.xp_W + 2 * a.xp_pad, Hp = a.xp_H + 2 * a.xp_pad;
+    const int64_t full = 2 * a.xp_pad * Wp, side = 2 * a.xp_pad;
+    const int64_t per_img = full + a.xp_H * side;
+    const int64_t images = a.x_count / 8 / (static_cast<int64_t>(a.xp_C8) * a.xp_H * a.xp_W);
+    const int64_t total = images * per_img * a.xp_C8;
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (int64_t i = static_cast<int64_t>(block) * blockDim.x + threadIdx.x; i < total; i += stride) {
+      const int64_t fp = i / a.xp_C8, c8 = i - fp * a.xp_C8;
+      const int64_t b = fp / per_img, j = fp - b * per_img;
+      int64_t hp, wp;
+      if (j < full) {
+        const int64_t r = j / Wp;
+        hp = r < a.xp_pad ? r : Hp - 2 * a.xp_pad + r;
+        wp = j - r * Wp;
+      } else {
+        const int64_t h = (j - full) / side, k = (j - full) - h * side;
+        hp = h + a.xp_pad;
+        wp = k < a.xp_pad ? k : a.xp_W + k;
+      }
+      *reinterpret_cast<uint4*>(a.Xc + (((b * Hp + hp) * Wp + wp) * a.xp_C8 + c8) * 8) = z;
     }
   }
 }

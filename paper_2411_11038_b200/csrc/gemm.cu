@@ -1146,18 +1146,21 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     // (ah, aw) holds the pixels (ah + stride * i, aw + stride * j).
     const int64_t Ci = cv->Cin, HW = static_cast<int64_t>(cv->H) * cv->W;
     auto class_map = [&](CUtensorMap* m, const void* base, int is16, int ah, int aw, int bw_, int bh_, int bb_,
-                         int row_bytes) {
+                         int row_bytes, int64_t ppix = 0, int64_t prow = 0, int64_t pimg = 0) {
+      if (!ppix) ppix = Ci;
+      if (!prow) prow = cv->W * Ci;
+      if (!pimg) pimg = Ci * HW;
       const int64_t Wc = ceil_div(cv->W - aw, cs), Hc = ceil_div(cv->H - ah, cs);
-      if (Wc < 1 || Hc < 1) return make_map_4d(m, base, is16, cv->B, 1, 1, Ci, Ci, bw_, bh_, bb_, row_bytes, 0, 0,
-                                               Ci * HW);     // empty class: never addressed by a tap
-      const char* b0 = static_cast<const char*>(base) + (static_cast<int64_t>(ah) * cv->W + aw) * Ci * (is16 ? 2 : 4);
-      return make_map_4d(m, b0, is16, cv->B, Hc, Wc, Ci, Ci, bw_, bh_, bb_, row_bytes, cs * Ci, cs * cv->W * Ci, Ci * HW);
+      if (Wc < 1 || Hc < 1) return make_map_4d(m, base, is16, cv->B, 1, 1, Ci, Ci, bw_, bh_, bb_, row_bytes, ppix, prow,
+                                               pimg);        // empty class: never addressed by a tap
+      const char* b0 = static_cast<const char*>(base) + (static_cast<int64_t>(ah) * prow + aw * ppix) * (is16 ? 2 : 4);
+      return make_map_4d(m, b0, is16, cv->B, Hc, Wc, Ci, Ci, bw_, bh_, bb_, row_bytes, cs * ppix, cs * prow, pimg);
     };
     if (cv->mode == 1 || cv->mode == 3) {
       CUtensorMap* maps[4] = {&ta, &tcls[0], &tcls[1], &tcls[2]};
       for (int i = 0; i < 4 && rc == EFQAT_OK; ++i) {
         const int ah = (i < cs * cs) ? i / cs : 0, aw = (i < cs * cs) ? i % cs : 0;
-        rc = class_map(maps[i], a.A, 1, ah, aw, c.tw, c.th, c.tb, 128);
+        rc = class_map(maps[i], a.A, 1, ah, aw, c.tw, c.th, c.tb, 128, cv->pix_pitch, cv->row_pitch, cv->img_pitch);
       }
     }
     if (cv->mode == 1) {

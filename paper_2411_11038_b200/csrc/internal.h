@@ -68,6 +68,9 @@ struct PrepArgs {
   const float* W; const float* s_w; int w_bits; bf16* Wq;
   const void* X; const float* s_x; const float* z_x; int x_bits, x_sym; bf16* Xc;
   int64_t x_count;   // elements of X (B*H*W*Cin for convolutions, M*K otherwise)
+  // Padded code layout (convolutions with few input channels): Xc is [B, xp_H + 2 pad, xp_W + 2 pad, 8 xp_C8]
+  // with the quantized pixel (h, w) at (h + pad, w + pad) and zeros around it.  xp_C8 == 0: dense.
+  int xp_C8, xp_H, xp_W, xp_pad;
   const void* dY; bf16* dYb; float* colsum_ws;
   const int32_t* idx; int64_t k_sel, pitch; bf16* dYsel;
   int* status;
@@ -161,6 +164,9 @@ struct ConvArgs {
   // mode 2 only: the class of input pixels (cls_h + stride * i, cls_w + stride * j) this launch
   // computes; a strided grad-input is one launch per class, each with the taps that reach it
   int cls_h, cls_w;
+  // modes 1 and 3: distance in elements between neighbouring pixels, rows and images of the
+  // activation codes (0: dense NHWC, i.e. Cin, W * Cin, H * W * Cin)
+  int64_t pix_pitch, row_pitch, img_pitch;
 };
 
 struct GemmArgs {

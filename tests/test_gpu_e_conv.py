@@ -46,6 +46,10 @@ CASES = [
     _case("c2x2_s2", 2, 8, 8, 64, 64, 2, 0, seed=13, stride=2),
     # ResNet-50: stem (3 input channels padded to 8), stride-2 3x3 of stages 2-4, stride-2 shortcuts
     _case("resnet_stem_7x7_s2", 1, 224, 224, 8, 64, 7, 3, w_bits=8, seed=14, stride=2),
+    # few input channels: a whole filter row is one contraction block on a zero-framed copy of the codes
+    _case("c3x3_cin16_s2_odd", 2, 11, 13, 16, 72, 3, 1, seed=21, stride=2),
+    _case("c5x5_cin8_valid", 3, 12, 9, 8, 64, 5, 0, w_bits=8, seed=22),
+    _case("c3x3_cin16_pad2", 2, 9, 9, 16, 64, 3, 2, seed=23),
     _case("resnet_56_128_3x3_s2", 2, 56, 56, 128, 128, 3, 1, seed=15, stride=2),
     _case("resnet_28_256_3x3_s2", 2, 28, 28, 256, 256, 3, 1, seed=16, stride=2),
     _case("resnet_14_512_3x3_s2", 2, 14, 14, 512, 512, 3, 1, seed=17, stride=2),

@@ -479,6 +479,67 @@ def measure_network(ctx, dev, sync_all, max_over_ranks):
     return out
 
 
+def measure_resnet50(ctx, dev, sync_all, max_over_ranks, batch=64):
+    """Every quantized layer of ResNet-50 (53 convolutions and the classifier) at 224 x 224, batch 64,
+    W4A8, through the same network calls: forward and backward per unfrozen ratio, network-wide
+    (CWPN) and layer-wise (LWPN).  Each layer has its own input and output-gradient tensors
+    (2.8 GB together), so nothing a layer reads is left in L2 by the one before it."""
+    import math
+    from paper_2411_11038_b200 import binding as B
+    from paper_2411_11038_b200 import network as NW
+    cases = I.resnet50(batch)
+    gen = torch.Generator(device=dev)
+    states = []
+    for c in cases:
+        gen.manual_seed(c.seed)
+        wshape = (c.N, c.R, c.S, c.Cin) if c.conv else (c.N, c.K)
+        xshape = (c.B, c.H, c.Wd, c.Cin) if c.conv else (c.M, c.K)
+        ho = (c.H + 2 * c.pad - c.R) // c.stride + 1
+        yshape = (c.B, ho, ho, c.N) if c.conv else (c.M, c.N)
+        W = torch.randn(wshape, generator=gen, device=dev) * math.sqrt(2.0 / c.K)
+        X = torch.randn(xshape, generator=gen, device=dev).abs().to(torch.bfloat16)
+        dY = torch.randn(yshape, generator=gen, device=dev).to(torch.bfloat16)
+        states.append(NW.LayerState(c, W, X, dY, None))
+    total = sum(c.N for c in cases)
+    net = NW.EfqatNetwork(ctx, states, B.CWPN, B.ratio_to_k(0.1, total), f_samples=batch, batch_samples=batch,
+                          use_cache=True, sgd=(SGD_LR, 0.9, 1e-4), adam=dict(lr=1e-6), share_outputs=False)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def t(fn, steps=8, warm=3):
+        return max_over_ranks(timed(fn, steps, warm, flush, sync_all) / steps)
+
+    gemm = sum(2.0 * c.M * c.N * c.K for c in cases)
+    out = {"workload": f"ResNet-50 at 224x224, batch {batch}: 53 convolutions (7x7 stride-2 input layer on 8 stored "
+                       "channels, bottleneck blocks 3-4-6-3, stride on the 3x3, shortcuts) + classifier, W4A8, NHWC "
+                       "bf16, synthetic |N(0,1)| activations, one tensor pair per layer",
+           "layers": len(cases), "channels": total, "fwd_gflop": gemm / 1e9}
+    rows = {}
+    for mode, name, ratios in ((B.CWPN, "CWPN", (0.0, 0.05, 0.10, 0.25, 1.0)), (B.LWPN, "LWPN", (0.05, 0.10, 0.25))):
+        for r in ratios:
+            budget = B.ratio_to_k(r, total) if mode == B.CWPN else int(r * len(cases))
+            net.use_selection(mode, budget)
+            net.reselect()
+            ks = net.counts()
+            fl = sum(2.0 * c.M * c.K * (c.N + k) for c, k in zip(cases, ks))
+            ms = t(net.backward)
+            rows[f"{name} {int(round(r * 100))}%"] = {
+                "bwd_ms": ms, "tflops": fl / (ms * 1e-3) / 1e12, "unfrozen_channels": int(sum(ks)),
+                "layers_with_unfrozen_channels": int(sum(1 for k in ks if k))}
+    full = rows["CWPN 100%"]["bwd_ms"]
+    for v in rows.values():
+        v["speedup_vs_full_qat"] = full / v["bwd_ms"]
+    out["backward"] = rows
+    net.use_selection(B.CWPN, B.ratio_to_k(0.1, total))
+    out["select_ms"] = t(net.reselect)
+    net.reselect()
+    out["fwd_ms"] = t(net.forward)
+    out["fwd_tflops"] = gemm / (out["fwd_ms"] * 1e-3) / 1e12
+    out["adam_and_cache_refresh_ms"] = t(net.optimizer_tail)
+    out["paper_context"] = ("Table 5 (A100, ResNet-50, f=12288): CWPN backward 0.87x / 0.86x / 0.80x of QAT speed at "
+                            "5 / 10 / 25 % (slower than QAT), LWPN 1.55x / 1.49x / 1.36x, 0 % 1.56x")
+    return out
+
+
 def run_capture(args):
     """Short run for a profiler: the first layer of the headline workload alone, a few steps."""
     from paper_2411_11038_b200 import binding as B
@@ -548,6 +609,12 @@ def run_ours(args):
         network = measure_network(ctx, dev, sync_all, max_over_ranks)
         status = status or ctx.device_status()
         torch.cuda.empty_cache()
+    # ---- ResNet-50, every quantized layer: the convolutional counterpart
+    resnet = None
+    if not args.skip_extras and not args.no_network:
+        resnet = measure_resnet50(ctx, dev, sync_all, max_over_ranks)
+        status = status or ctx.device_status()
+        torch.cuda.empty_cache()
     all_clock.stop_flag = True
     all_clock.join(timeout=2)
 
@@ -577,6 +644,7 @@ def run_ours(args):
             "select_ms": head["select_ms"],
             "bert_base": bert,
             "network": network,
+            "resnet50": resnet,
             "device_status": status,
             "paper_context": "paper reports 1.44-1.64x backward speed-up on A10/A100 (whole network)",
         }))
@@ -593,7 +661,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the headline timed steps and a 3-step end-to-end leg")
-    ap.add_argument("--no-network", action="store_true", help="skip the 144-layer stack")
+    ap.add_argument("--no-network", action="store_true", help="skip the 144-layer stack and the ResNet-50 stack")
     ap.add_argument("--capture", action="store_true",
                     help="three steps of the first headline layer alone (small run for a profiler)")
     args = ap.parse_args()

@@ -161,7 +161,14 @@ int dx_partials(const efqat_layer_desc* l) {
       if (Wc < 1 || Hc < 1) continue;
       int tw, th, tb;
       conv_pixel_box(static_cast<int>(Wc), static_cast<int>(Hc), l->B, 128, &tw, &th, &tb);
-      n += ceil_div(Wc, tw) * ceil_div(Hc, th) * ceil_div(l->B, tb) * ceil_div(l->Cin, 64) * 8;
+      int64_t boxes = ceil_div(Wc, tw) * ceil_div(Hc, th) * ceil_div(l->B, tb);
+      // the launch may tile the class with one-image boxes instead (taps sharing a box per filter column)
+      const int cand[2][2] = {{8, 16}, {16, 8}};
+      for (int i = 0; i < 2; ++i) {
+        const int64_t b2 = ceil_div(Wc, cand[i][0]) * ceil_div(Hc, cand[i][1]) * l->B;
+        if (b2 <= (23 * Wc * Hc * l->B) / (20 * 128) + 1 && b2 > boxes) boxes = b2;
+      }
+      n += boxes * ceil_div(l->Cin, 64) * 8;
     }
   return static_cast<int>(n);
 }

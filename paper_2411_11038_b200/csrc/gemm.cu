@@ -70,6 +70,18 @@ struct GemmParams {
   int kps;            // k-blocks per stage: one barrier round trip covers kps * 64 contraction elements
   int merged;         // MN-major operands arrive as one TMA box per 64-wide chunk and stage (plain matrices only)
   int b_stage_bytes;
+  // One stage of the ring = a_region_bytes of A operand + b_region_bytes of B operand; k-block u of
+  // the stage has its A operand a_sub_off * u bytes into the A region.
+  int a_region_bytes, b_region_bytes, a_sub_off;
+  // Convolutions whose taps form a grid (filter rows x filter columns, consecutive row shifts):
+  // the taps of one filter column differ only by a shift of whole pixel rows, so ONE box of
+  // th + colshare - 1 pixel rows serves all `colshare` of them (each tap's operand starts
+  // tw pixels = tw * 128 bytes further on, a multiple of the 1024-byte swizzle atom because tw is a
+  // multiple of 8).  0: every tap loads a box of its own.  a_tx: bytes of that shared box.
+  int colshare, a_tx;
+  // The whole B operand (all taps and channel chunks) stays in shared memory for the life of the
+  // CTA: nkb blocks of b_stage_bytes behind the ring (tiles_n == 1 only).
+  int bres;
   int splits;
   int tiles_m, tiles_n;
   int panel_dir, panel;   // order of the tiles in the work list (see tile_coords)
@@ -95,6 +107,7 @@ struct __align__(16) SmemCtl {
   uint64_t acc_empty[2];
   uint64_t xbar[EPI_WARPS];
   uint64_t drain;           // abort path only: completion of the MMAs issued before the abort
+  uint64_t bres_full;       // resident B operand has landed
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -127,6 +140,21 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int t, int& tm,
   }
 }
 
+// Contraction block kb of a convolution (modes 1, 2) -> filter tap t and 64-channel chunk cc.  Plain
+// order: chunks inside taps.  Column-sharing order: the taps of one filter column are the k-blocks
+// of one stage, so blocks run (column, chunk, tap of the column).
+__device__ __forceinline__ void conv_block(const GemmParams& p, int kb, int& t, int& cc) {
+  if (p.colshare) {
+    const int per_col = p.colshare * p.cv.cchunks;
+    const int col = kb / per_col, r = kb - col * per_col;
+    cc = r / p.colshare;
+    t = col * p.colshare + (r - cc * p.colshare);
+  } else {
+    t = kb / p.cv.cchunks;
+    cc = kb - t * p.cv.cchunks;
+  }
+}
+
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -148,9 +176,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms of TMA and UMMA
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;     // one k-block of A and B
-  const int stage_bytes = p.kps * sub_bytes;
-  uint8_t* out_stg = smem + p.stages * stage_bytes;          // [8 warps][out_bufs][HB_BYTES]
+  const int stage_bytes = p.a_region_bytes + p.b_region_bytes;
+  uint8_t* bres_reg = smem + p.stages * stage_bytes;         // [nkb][b_stage_bytes] resident B operand (bres)
+  uint8_t* out_stg = bres_reg + (p.bres ? p.nkb * p.b_stage_bytes : 0);   // [8 warps][out_bufs][HB_BYTES]
   uint8_t* x_stg = out_stg + (EPI == EPI_PART ? 0 : EPI_WARPS * p.out_bufs * HB_BYTES);   // [8 warps][HB_BYTES] (EPI_DX)
   SmemCtl* ctl = reinterpret_cast<SmemCtl*>(x_stg + (EPI == EPI_DX ? EPI_WARPS * HB_BYTES : 0));
   float* s_scale = reinterpret_cast<float*>(ctl + 1);        // [8 warps][128 scales, 128 biases, 128 zero-point terms] (EPI_FWD), warp-private
@@ -176,6 +204,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&ctl->xbar[w], 1);
     mbar_init(&ctl->drain, 1);
+    mbar_init(&ctl->bres_full, 1);
     ctl->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmA);
@@ -222,6 +251,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int it = 0;
       bool live = true;
       const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
+      if (p.bres && unit < total_items) {
+        // resident B operand: every (tap, chunk) block once, all on one barrier
+        const int bch = (((static_cast<int>(p.Nc) + 15) & ~15) + 63) >> 6;
+        const uint32_t tx_b1 = B_MN ? bch * CHUNK_BYTES : bn_cta * BK * 2;
+        if (lane == 0) mbar_arrive_expect_tx(&ctl->bres_full, tx_b1 * p.nkb);
+        __syncwarp();
+        for (int kb = lane; kb < p.nkb; kb += 32) {
+          int t, cc;
+          conv_block(p, kb, t, cc);
+          const int rs = p.cv.tap_rs[t];
+          uint8_t* sb = bres_reg + kb * p.b_stage_bytes;
+          if (B_MN) {
+            for (int c = 0; c < bch; ++c)
+              tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->bres_full, rs * p.cv.wcols + 64 * c, cc * 64);
+          } else {
+            tma_load_2d(sb, &tmB, &ctl->bres_full, rs * p.cv.wcols + cc * 64, 0);
+          }
+        }
+      }
       for (int w = unit; w < total_items && live; w += num_units) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
         int tm, tn;
@@ -234,12 +282,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int b_chunks = (n_eff + 63) >> 6;
         // bytes credited to the (leader's) full barrier per stage: both CTAs' copies in pair mode
         // (a merged MN-major box always brings all kps k-blocks of its chunk, used or not)
-        const uint32_t tx_a = A_STAGE_BYTES, tx_b = B_MN ? b_chunks * CHUNK_BYTES : bn_cta * BK * 2;
+        const uint32_t tx_a = A_STAGE_BYTES, tx_b = p.bres ? 0u : (B_MN ? b_chunks * CHUNK_BYTES : bn_cta * BK * 2);
         const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
         const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
         const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
         // One barrier round trip costs ~0.3 us whatever it carries, so a stage holds several
         // k-blocks: all of them land on the same full barrier and are released by one commit.
+        // convolution (modes 1, 2): filter tap and channel chunk of this lane's k-block, kept by
+        // increments from stage to stage (an integer division per copy sat on the issue path)
+        int ct = 0, ccc = 0, tw0 = 0, th0 = 0, tb0 = 0;     // ... and the origin of the tile's pixel box
+        if ((p.cv.mode == 1 || p.cv.mode == 2) && lane >= 8) {
+          conv_block(p, kb_begin + ((lane - 8) >> 1), ct, ccc);
+          const int bw = tm % p.cv.tiles_w, bh = (tm / p.cv.tiles_w) % p.cv.tiles_h;
+          const int bb = tm / (p.cv.tiles_w * p.cv.tiles_h);
+          tw0 = bw * p.cv.tw; th0 = bh * p.cv.th; tb0 = bb * p.cv.tb;
+        }
         for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it) {
           const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
           const int s = it % p.stages;
@@ -252,7 +309,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               ok_stage = 0;
             } else if (rank == 0) {
               // the leader's barrier collects the bytes of both CTAs of a pair; only the leader arrives on it
-              mbar_arrive_expect_tx(&ctl->full[s], (CTA2 ? 2u : 1u) * (tx_a * (a_mrg ? p.kps : nsub) +
+              mbar_arrive_expect_tx(&ctl->full[s], (CTA2 ? 2u : 1u) * ((p.colshare ? static_cast<uint32_t>(p.a_tx)
+                                                                                   : tx_a * (a_mrg ? p.kps : nsub)) +
                                                                       tx_b * (b_mrg ? p.kps : nsub)));
             }
           }
@@ -262,7 +320,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           uint8_t* a_reg = smem + s * stage_bytes;               // [kps k-blocks of A][kps k-blocks of B]
-          uint8_t* b_reg = a_reg + p.kps * A_STAGE_BYTES;
+          uint8_t* b_reg = a_reg + p.a_region_bytes;
           const uint32_t fb = CTA2 ? mapa_u32(smem_u32(&ctl->full[s]), 0) : 0u;
           if (lane < 6) {
             // one box of kps * 64 contraction rows per 64-wide chunk: chunk c sits at c * kps * 8 KiB
@@ -338,16 +396,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             } else {
               // forward / grad-input: tile rows = one box of 128 pixels; contraction block kb = (tap, 64 channels)
-              const int tmi = tm;
-              const int bw = tmi % p.cv.tiles_w, bh = (tmi / p.cv.tiles_w) % p.cv.tiles_h;
-              const int bb = tmi / (p.cv.tiles_w * p.cv.tiles_h);
-              const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
-              const int t = kb / p.cv.cchunks, cc = kb - t * p.cv.cchunks;
+              const int w0 = tw0, h0 = th0, b0 = tb0;
+              const int t = ct, cc = ccc;
               const int rs = p.cv.tap_rs[t];
               if (do_a) {
-                const int mi = p.cv.tap_map[t];
-                const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
-                tma_load_4d(sa, ma, &ctl->full[s], cc * 64, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
+                if (p.colshare) {
+                  // the first tap of the filter column (smallest row shift) brings the box of all of them
+                  if (u == 0) tma_load_4d(a_reg, &tmA, &ctl->full[s], cc * 64, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
+                } else {
+                  const int mi = p.cv.tap_map[t];
+                  const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
+                  tma_load_4d(sa, ma, &ctl->full[s], cc * 64, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
+                }
+              } else if (p.bres) {
+                // B operand already resident
               } else if (B_MN) {     // W^ viewed as [N rows, R*S*Cin columns]: rows = contraction
                 for (int c = 0; c < b_chunks; ++c)
                   tma_load_2d(sb + c * CHUNK_BYTES, &tmB, &ctl->full[s], rs * p.cv.wcols + n0 + 64 * c, cc * 64);
@@ -356,15 +418,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             }
           }
+          if (p.colshare) {
+            if (++ccc == p.cv.cchunks) { ccc = 0; ct += p.colshare; }
+          } else {
+            ccc += p.kps;
+            while (ccc >= p.cv.cchunks && p.cv.cchunks > 0) { ccc -= p.cv.cchunks; ++ct; }
+          }
           __syncwarp();
         }
       }
       // Make sure none of this CTA's bulk copies is still in flight when it exits (only
       // relevant after an abort: otherwise the MMA warp has consumed every stage).
       const int issued = it;
-      if (lane == 0 && rank == 0)
+      if (lane == 0 && rank == 0) {
         for (int j = (issued > p.stages ? issued - p.stages : 0); j < issued; ++j)
           mbar_wait(&ctl->full[j % p.stages], (j / p.stages) & 1, 20000000ull);
+        if (p.bres && unit < total_items) mbar_wait(&ctl->bres_full, 0, 20000000ull);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
@@ -393,6 +463,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_STRIDE;
+        if (p.bres && acc_it == 0) {
+          if (*abort_flag || !mbar_wait(&ctl->bres_full, 0)) {
+            record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
+            *abort_flag = 1;
+            ok = false;
+            break;
+          }
+        }
         for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it) {
           const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
           const int s = it % p.stages;
@@ -409,9 +487,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           // k-block u of the stage: merged MN-major operands keep their chunks kps * 8 KiB apart
           const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
           const uint32_t a_base = smem_u32(smem + s * stage_bytes);
-          const uint32_t b_base = a_base + p.kps * A_STAGE_BYTES;
-          const uint32_t a_addr = a_base + u * (a_mrg ? CHUNK_BYTES : A_STAGE_BYTES);
-          const uint32_t b_addr = b_base + u * (b_mrg ? CHUNK_BYTES : p.b_stage_bytes);
+          const uint32_t b_base = a_base + p.a_region_bytes;
+          const uint32_t a_addr = a_base + u * (a_mrg ? CHUNK_BYTES : p.a_sub_off);
+          const uint32_t b_addr = p.bres ? smem_u32(bres_reg) + kb * p.b_stage_bytes
+                                         : b_base + u * (b_mrg ? CHUNK_BYTES : p.b_stage_bytes);
           const uint32_t a_lbo = a_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
           const uint32_t b_lbo = b_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
 #pragma unroll
@@ -853,6 +932,37 @@ void conv_pixel_box(int W, int H, int B, int target, int* tw, int* th, int* tb) 
     }
 }
 
+// Shared memory left for the operand ring after the epilogue's staging blocks and the control block.
+static int ring_budget(int epi) {
+  const int out_stg_bytes = (epi == EPI_PART) ? 0 : EPI_WARPS * HB_BYTES;
+  const int fixed = out_stg_bytes + (epi == EPI_DX ? EPI_WARPS * HB_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
+                    (epi == EPI_FWD ? EPI_WARPS * 384 * 4 : 0);
+  return 227 * 1024 - 1024 - fixed;
+}
+
+// Column-sharing tiles (see GemmParams::colshare): one image per box and a box width that is a
+// multiple of 8 pixels, so that a shift by one pixel row moves the operand by whole swizzle
+// atoms.  Returns false when every such box wastes more than 15 % of its pixels on this extent.
+bool conv_colshare_box(int W, int H, int rows_extra, int* tw, int* th) {
+  double best = 1e300;
+  bool found = false;
+  // (32 x 4 boxes were measured too: with so few rows per box the shared box saves too little)
+  const int cand[2][2] = {{8, 16}, {16, 8}};
+  for (int i = 0; i < 2; ++i) {
+    const int a = cand[i][0], b = cand[i][1];
+    const double vol = static_cast<double>(ceil_div(W, a) * a) * static_cast<double>(ceil_div(H, b) * b);
+    if (vol > 1.15 * W * H) continue;
+    // at equal waste, the box that loads the fewest halo rows
+    const double score = vol * (1.0 + 1e-3 * (b + rows_extra) / b);
+    if (score < best) {
+      best = score;
+      *tw = a; *th = b;
+      found = true;
+    }
+  }
+  return found;
+}
+
 // Tile width for the forward / grad-input GEMMs: multiples of 64 so that every 128-byte
 // staging row of the epilogue lies inside one tile.
 static int choose_bn(int64_t Mr, int64_t Nc, int sm_count) {
@@ -955,6 +1065,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   const ConvArgs* cv = a.conv;
   const int cs = cv ? cv->stride : 1;           // convolution stride
   int cWc = 0, cHc = 0;                         // grad-input: extent of this launch's pixel class
+  int col_order[MAX_TAPS];                      // taps column by column (column sharing)
   if (cv) {
     if (cv->mode < 1 || cv->mode > 3 || cs < 1 || cs > 2 || cv->R * cv->S > MAX_TAPS) return EFQAT_ERR_UNIMPL;
     if (cv->mode == 2) {           // grad-input tiles must not straddle the end of Cin (B is not zero there)
@@ -993,6 +1104,34 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       if (tiles_out) *tiles_out = 0;
       if (grid_out) *grid_out = 0;
       return EFQAT_OK;
+    }
+    // Column sharing: the taps must form a grid of filter columns (one dw each) x rows with
+    // consecutive dh, all through one tensor map; they are then re-ordered column by column,
+    // smallest row shift first.
+    if ((cv->mode == 2 || (cv->mode == 1 && cs == 1)) && c.ntaps >= 2) {
+      int order[MAX_TAPS], n = c.ntaps, per_col = 0;
+      for (int j = 0; j < n; ++j) order[j] = j;
+      for (int i = 1; i < n; ++i)                         // insertion sort by (dw, dh)
+        for (int j = i; j > 0; --j) {
+          const int x = order[j - 1], y = order[j];
+          if (c.tap_dw[x] < c.tap_dw[y] || (c.tap_dw[x] == c.tap_dw[y] && c.tap_dh[x] <= c.tap_dh[y])) break;
+          order[j - 1] = y; order[j] = x;
+        }
+      bool grid = true;
+      for (int first = 0; first < n && grid;) {
+        int last = first + 1;
+        while (last < n && c.tap_dw[order[last]] == c.tap_dw[order[first]]) ++last;
+        const int cnt = last - first;
+        if (per_col == 0) per_col = cnt;
+        if (cnt != per_col || c.tap_map[order[first]] != 0) grid = false;
+        for (int j = first + 1; j < last && grid; ++j)
+          if (c.tap_dh[order[j]] != c.tap_dh[order[j - 1]] + 1 || c.tap_map[order[j]] != 0) grid = false;
+        first = last;
+      }
+      if (grid && n == c.ntaps && per_col >= 2 && per_col <= 4) {
+        p.colshare = per_col;
+        for (int j = 0; j < n; ++j) col_order[j] = order[j];
+      }
     }
   }
   // CTA pairs (256 x BN tiles, tiles full in N) halve the B traffic from L2 per FLOP; they are
@@ -1033,6 +1172,31 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     // input pixels for grad-input
     const int pW = (cv->mode == 2) ? cWc : cv->Wo, pH = (cv->mode == 2) ? cHc : cv->Ho;
     conv_pixel_box(pW, pH, cv->B, cv->mode == 3 ? BK : BM, &c.tw, &c.th, &c.tb);
+    if (p.colshare) {
+      // taken when a suitable box exists and two stages (with the B operand resident or staged) fit
+      int tw2 = 0, th2 = 0;
+      bool fits = conv_colshare_box(pW, pH, p.colshare - 1, &tw2, &th2);
+      if (fits) {
+        const int a_reg = static_cast<int>(round_up((th2 + p.colshare - 1) * tw2 * 128, 1024));
+        const int b_st = static_cast<int>(round_up(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2, 1024));
+        const int nkb2 = c.ntaps * static_cast<int>(ceil_div((cv->mode == 2) ? cv->N : cv->Cin, 64));
+        const int ring = ring_budget(a.epi);
+        const bool res = p.tiles_n == 1 && static_cast<int64_t>(nkb2) * b_st + 2 * a_reg <= ring;
+        fits = res || ring / (a_reg + p.colshare * b_st) >= 2;
+        if (fits) {
+          c.tw = tw2; c.th = th2; c.tb = 1;
+          p.bres = res ? 1 : 0;
+          p.a_region_bytes = a_reg;
+          p.a_tx = (th2 + p.colshare - 1) * tw2 * 128;
+          const ConvP o = c;
+          for (int j = 0; j < c.ntaps; ++j) {
+            c.tap_dh[j] = o.tap_dh[col_order[j]]; c.tap_dw[j] = o.tap_dw[col_order[j]];
+            c.tap_map[j] = o.tap_map[col_order[j]]; c.tap_rs[j] = o.tap_rs[col_order[j]];
+          }
+        }
+      }
+      if (!fits) p.colshare = 0;
+    }
     c.tiles_w = static_cast<int>(ceil_div(pW, c.tw));
     c.tiles_h = static_cast<int>(ceil_div(pH, c.th));
     const int tiles_b = static_cast<int>(ceil_div(cv->B, c.tb));
@@ -1085,17 +1249,28 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   p.b_stage_bytes = static_cast<int>(round_up(p.b_stage_bytes, 1024));
   const int sub_bytes = A_STAGE_BYTES + p.b_stage_bytes;
   const int out_stg_bytes = (a.epi == EPI_PART) ? 0 : EPI_WARPS * HB_BYTES;     // one staging buffer per warp
-  int fixed_bytes = out_stg_bytes + (a.epi == EPI_DX ? EPI_WARPS * HB_BYTES : 0) + static_cast<int>(sizeof(SmemCtl)) +
-                    (a.epi == EPI_FWD ? EPI_WARPS * 384 * 4 : 0);
-  const int ring_bytes = 227 * 1024 - 1024 - fixed_bytes;
+  int fixed_bytes = 227 * 1024 - 1024 - ring_budget(a.epi);
+  int ring_bytes = ring_budget(a.epi);
   // k-blocks per stage: as many as still leave three stages (two for the widest tiles), at most 4
   int kps = ring_bytes / (3 * sub_bytes);
   if (kps <= 1) kps = (ring_bytes / (2 * sub_bytes) >= 2) ? 2 : 1;
   if (kps > 4) kps = 4;
   if (kps > p.nkb) kps = p.nkb;
+  int bres_bytes = 0;
+  if (p.colshare) {
+    kps = p.colshare;
+    p.a_sub_off = p.cv.tw * 128;
+    p.b_region_bytes = p.bres ? 0 : kps * p.b_stage_bytes;
+    bres_bytes = p.bres ? p.nkb * p.b_stage_bytes : 0;
+    ring_bytes -= bres_bytes;
+  } else {
+    p.a_region_bytes = kps * A_STAGE_BYTES;
+    p.b_region_bytes = kps * p.b_stage_bytes;
+    p.a_sub_off = A_STAGE_BYTES;
+  }
   p.kps = kps;
   p.merged = cv ? 0 : 1;
-  const int stage_bytes = kps * sub_bytes;
+  const int stage_bytes = p.a_region_bytes + p.b_region_bytes;
   int stages = ring_bytes / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return EFQAT_ERR_SHAPE;
@@ -1160,7 +1335,8 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       CUtensorMap* maps[4] = {&ta, &tcls[0], &tcls[1], &tcls[2]};
       for (int i = 0; i < 4 && rc == EFQAT_OK; ++i) {
         const int ah = (i < cs * cs) ? i / cs : 0, aw = (i < cs * cs) ? i % cs : 0;
-        rc = class_map(maps[i], a.A, 1, ah, aw, c.tw, c.th, c.tb, 128, cv->pix_pitch, cv->row_pitch, cv->img_pitch);
+        rc = class_map(maps[i], a.A, 1, ah, aw, c.tw, c.th + (p.colshare ? p.colshare - 1 : 0), c.tb, 128, cv->pix_pitch,
+                       cv->row_pitch, cv->img_pitch);
       }
     }
     if (cv->mode == 1) {
@@ -1169,7 +1345,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
         rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, qh, qb, 64);
       tx = ta;
     } else if (cv->mode == 2) {
-      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, c.th, c.tb);
+      rc = make_map_4d(&ta, a.A, 1, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, c.th + (p.colshare ? p.colshare - 1 : 0), c.tb);
       tcls[0] = tcls[1] = tcls[2] = ta;
       if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, BK);
       if (rc == EFQAT_OK) rc = class_map(&to, a.out, a.out_bf16, cv->cls_h, cv->cls_w, c.tw, qh, qb, 64);
@@ -1186,7 +1362,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   const int max_units = pair ? sm_count / 2 : sm_count;
   const int units = static_cast<int>(items < max_units ? items : max_units);
   const int grid = pair ? 2 * units : units;
-  const size_t smem = static_cast<size_t>(stages) * stage_bytes + fixed_bytes + 1024;
+  const size_t smem = static_cast<size_t>(stages) * stage_bytes + bres_bytes + fixed_bytes + 1024;
   if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * EPI_WARPS;
   if (grid_out) *grid_out = grid;
 

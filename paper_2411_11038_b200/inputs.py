@@ -128,6 +128,38 @@ def config3_strided(batch: int = 64) -> List[LayerCase]:
     return out
 
 
+def resnet50(batch: int = 64) -> List[LayerCase]:
+    """Every convolution of ResNet-50 at 224 x 224 (bottleneck blocks 3-4-6-3, stride on the 3x3
+    convolution, input stored with 8 channels) and the classifier: 54 quantized layers, W4A8,
+    |N(0,1)| activations.  Section 4 "Setup" quantizes all of them, input, output and shortcut
+    layers included."""
+    out = []
+
+    def conv(name, hw, cin, cout, r, stride):
+        pad = r // 2
+        ho = (hw + 2 * pad - r) // stride + 1
+        out.append(LayerCase(f"rn50_{name}", batch * ho * ho, r * r * cin, cout, w_bits=4, x_bits=8, w_std=None,
+                             x_abs=True, seed=3200 + len(out), conv=True, B=batch, H=hw, Wd=hw, Cin=cin, R=r, S=r,
+                             stride=stride, pad=pad))
+        return ho
+
+    conv("stem", 224, 8, 64, 7, 2)
+    hw, cin = 56, 64                                    # after the 3x3 stride-2 max-pool
+    for stage, (width, blocks) in enumerate(((64, 3), (128, 4), (256, 6), (512, 3))):
+        for b in range(blocks):
+            stride = 2 if (b == 0 and stage > 0) else 1
+            tag = f"s{stage + 1}b{b + 1}"
+            if b == 0:
+                conv(tag + "_shortcut", hw, cin, 4 * width, 1, stride)
+            conv(tag + "_a", hw, cin, width, 1, 1)
+            ho = conv(tag + "_b", hw, width, width, 3, stride)
+            conv(tag + "_c", ho, width, 4 * width, 1, 1)
+            hw, cin = ho, 4 * width
+    out.append(LayerCase("rn50_fc", batch, 2048, 1000, w_bits=4, x_bits=8, w_std=None, x_abs=True,
+                         seed=3200 + len(out)))
+    return out
+
+
 def config4(layers: int = 24, M: int = 9216) -> List[LayerCase]:
     """BERT-large-shaped stack: per block Q,K,V,O 1024->1024, FFN 1024->4096->1024."""
     out = []

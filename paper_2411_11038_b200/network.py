@@ -88,9 +88,13 @@ class EfqatNetwork:
         k_max = [n for n in self.N]          # any layer may end up fully unfrozen (LWPN, CWPN)
         descs = []
         ws_need = 0
+
+        def geom(c):
+            return B.ConvGeom(c.B, c.H, c.Wd, c.Cin, c.R, c.S, c.stride, c.pad) if c.conv else None
+
         for st, km in zip(self.layers, k_max):
             c = st.case
-            d = B.layer_desc(c.M, c.N, c.K, B.F32 if c.act_dtype == torch.float32 else B.BF16)
+            d = B.layer_desc(c.M, c.N, c.K, B.F32 if c.act_dtype == torch.float32 else B.BF16, geom(c))
             spec = B.QSpec(c.w_bits, c.x_bits, 1 if c.x_symmetric else 0)
             ws_need = max(ws_need, B.workspace_bytes(d, spec, km))
             descs.append((d, spec))
@@ -102,8 +106,9 @@ class EfqatNetwork:
         self.qopts = []
         for st, km in zip(self.layers, k_max):
             c = st.case
-            key = (c.M, c.N, c.K, c.act_dtype)
+            key = (c.M, c.N, c.K, c.act_dtype, c.conv, c.R, c.stride)
             plan = B.LayerPlan(ctx, c.M, c.N, c.K, c.act_dtype, c.w_bits, c.x_bits, c.x_symmetric, km, dev,
+                               conv=geom(c), x_shape=tuple(st.X.shape), y_shape=tuple(st.dY.shape),
                                with_cache=use_cache, ws=self.ws,
                                outputs=by_shape.get(key) if share_outputs else None)
             by_shape.setdefault(key, plan)

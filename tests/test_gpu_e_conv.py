@@ -50,6 +50,12 @@ CASES = [
     _case("c3x3_cin16_s2_odd", 2, 11, 13, 16, 72, 3, 1, seed=21, stride=2),
     _case("c5x5_cin8_valid", 3, 12, 9, 8, 64, 5, 0, w_bits=8, seed=22),
     _case("c3x3_cin16_pad2", 2, 9, 9, 16, 64, 3, 2, seed=23),
+    # extents that 8-, 16- or 32-pixel-wide one-image boxes tile well: the taps of a filter column share one box
+    _case("c3x3_shared_30x15", 2, 15, 30, 64, 72, 3, 1, seed=24),
+    _case("c3x3_shared_cin128", 2, 16, 24, 128, 136, 3, 1, seed=25),
+    _case("c3x3_shared_valid_f32", 1, 16, 24, 64, 64, 3, 0, dtype=torch.float32, seed=26),
+    _case("c4x4_shared_s2", 2, 32, 48, 64, 64, 4, 1, seed=27, stride=2),
+    _case("resnet_56_64to64_3x3_b2", 2, 56, 56, 64, 64, 3, 1, seed=28),
     _case("resnet_56_128_3x3_s2", 2, 56, 56, 128, 128, 3, 1, seed=15, stride=2),
     _case("resnet_28_256_3x3_s2", 2, 28, 28, 256, 256, 3, 1, seed=16, stride=2),
     _case("resnet_14_512_3x3_s2", 2, 14, 14, 512, 512, 3, 1, seed=17, stride=2),

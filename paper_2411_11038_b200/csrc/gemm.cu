@@ -248,7 +248,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // Lanes 0..5 take the merged MN-major boxes (A chunks 0-1, B chunks 0-3); lanes 8.. take
     // the per-k-block copies, two lanes per k-block (A operand, B operand).
     {
-      int it = 0;
+      int it = 0, ring_s = 0;
+      uint32_t ring_ph = 0;
       bool live = true;
       const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
       if (p.bres && unit < total_items) {
@@ -297,10 +298,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int bb = tm / (p.cv.tiles_w * p.cv.tiles_h);
           tw0 = bw * p.cv.tw; th0 = bh * p.cv.th; tb0 = bb * p.cv.tb;
         }
-        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it) {
+        // grad-weight: contraction block -> box of 64 output pixels, and the (tap, first channel) of
+        // the two 64-row halves of this tile
+        int kbw = 0, kbh = 0, kbb = 0, at[2] = {0, 0}, ac[2] = {0, 0};
+        if (p.cv.mode == 3 && lane >= 8) {
+          const int kb = kb_begin + ((lane - 8) >> 1);
+          kbw = kb % p.cv.tiles_w; kbh = (kb / p.cv.tiles_w) % p.cv.tiles_h;
+          kbb = kb / (p.cv.tiles_w * p.cv.tiles_h);
+          const int cpad = p.cv.cchunks * 64;       // tile rows per tap (channels padded to 64)
+          for (int j = 0; j < 2; ++j) {
+            const int k = m0 + 64 * j;
+            at[j] = k / cpad; ac[j] = k - at[j] * cpad;
+            if (at[j] >= p.cv.ntaps) { at[j] = 0; ac[j] = p.cv.C; }     // past the last tap: all zeros
+          }
+        }
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it, ring_s = (ring_s + 1 == p.stages) ? 0 : ring_s + 1,
+                 ring_ph ^= (ring_s == 0) ? 1u : 0u) {
           const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1;
+          const int s = ring_s;               // it % stages and (it / stages) & 1, kept by increments
+          const uint32_t ph = ring_ph;
           int ok_stage = 1;
           if (lane == 0) {
             if (*abort_flag || !mbar_wait(&ctl->empty[s], ph ^ 1)) {
@@ -377,15 +393,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             } else if (p.cv.mode == 3) {
               // grad-weight: contraction block kb = one box of 64 output pixels; tile rows = (tap, channel)
-              const int bw = kb % p.cv.tiles_w, bh = (kb / p.cv.tiles_w) % p.cv.tiles_h;
-              const int bb = kb / (p.cv.tiles_w * p.cv.tiles_h);
-              const int w0 = bw * p.cv.tw, h0 = bh * p.cv.th, b0 = bb * p.cv.tb;
+              const int w0 = kbw * p.cv.tw, h0 = kbh * p.cv.th, b0 = kbb * p.cv.tb;
               if (do_a) {
-                const int cpad = p.cv.cchunks * 64;       // tile rows per tap (channels padded to 64)
                 for (int j = 0; j < 2; ++j) {
-                  const int k = m0 + 64 * j;
-                  int t = k / cpad, c = k - t * cpad;
-                  if (t >= p.cv.ntaps) { t = 0; c = p.cv.C; }     // past the last tap: all zeros
+                  const int t = at[j], c = ac[j];
                   const int mi = p.cv.tap_map[t];
                   const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
                   tma_load_4d(sa + j * CHUNK_BYTES, ma, &ctl->full[s], c, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
@@ -418,7 +429,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             }
           }
-          if (p.colshare) {
+          if (p.cv.mode == 3) {
+            kbw += p.kps;
+            while (kbw >= p.cv.tiles_w) {
+              kbw -= p.cv.tiles_w;
+              if (++kbh == p.cv.tiles_h) { kbh = 0; ++kbb; }
+            }
+          } else if (p.colshare) {
             if (++ccc == p.cv.cchunks) { ccc = 0; ct += p.colshare; }
           } else {
             ccc += p.kps;
@@ -439,7 +456,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
     if (lane == 0 && rank == 0) {
-      int it = 0, acc_it = 0;
+      int it = 0, acc_it = 0, ring_s = 0;
+      uint32_t ring_ph = 0;
       bool ok = true;
       for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
         const int split = w / tiles_mn, t = w - split * tiles_mn;
@@ -471,10 +489,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
         }
-        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it) {
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += p.kps, ++it, ring_s = (ring_s + 1 == p.stages) ? 0 : ring_s + 1,
+                 ring_ph ^= (ring_s == 0) ? 1u : 0u) {
           const int nsub = (kb_end - kb0 < p.kps) ? kb_end - kb0 : p.kps;
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1;
+          const int s = ring_s;               // it % stages and (it / stages) & 1, kept by increments
+          const uint32_t ph = ring_ph;
           if (*abort_flag || !mbar_wait(&ctl->full[s], ph)) {
             record_status(p.status, EFQAT_DEV_WAIT_TIMEOUT);
             *abort_flag = 1;

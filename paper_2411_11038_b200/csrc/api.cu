@@ -85,6 +85,7 @@ struct LayerWs {
   float* dxpart;   // [tiles][2]
   float* colsum;   // [COLSUM_SLABS][N]
   int32_t* wsum;   // [N] row sums of the 8-bit weight codes (integer forward)
+  bf16* strip;     // [N, R * nP * 64] banded weights of the strip-form grad-input (few input channels)
   int64_t pitch;
   int splits;
   size_t bytes;
@@ -145,6 +146,33 @@ int64_t xc_elems(const efqat_layer_desc* l) {
   return static_cast<int64_t>(l->B) * (l->H + 2 * l->pad) * (l->W + 2 * l->pad) * l->Cin;
 }
 
+// Strip form of the grad-input of such a layer.  With Cin stored channels, P = 64 / Cin input pixels
+// of one image row are 64 contiguous elements of dX: they become ONE output row of the GEMM (64
+// columns instead of Cin), fed by the nP output columns that reach the strip, through a banded
+// copy of the weights (StripArgs).  One launch per class of input ROWS (stride classes); along W
+// the stride is absorbed by the band.  dY is read through up to four views whose pixel pitch is
+// Q = P / stride output pixels (one per residue of the output column modulo Q).
+struct StripGeo {
+  bool ok;
+  int P, Q, p_min, nP;
+};
+
+StripGeo strip_geo(const efqat_layer_desc* l) {
+  StripGeo g = {};
+  if (!narrow_conv(l) || 64 % l->Cin != 0) return g;
+  g.P = 64 / l->Cin;
+  if (l->W % g.P != 0 || g.P % l->stride != 0) return g;
+  g.Q = g.P / l->stride;
+  if (g.Q > 4) return g;
+  const int lo = l->pad - (l->S - 1);                       // smallest stride * p that still reaches pixel q = 0
+  g.p_min = lo >= 0 ? (lo + l->stride - 1) / l->stride : -((-lo) / l->stride);
+  const int p_max = (g.P - 1 + l->pad) / l->stride;
+  g.nP = p_max - g.p_min + 1;
+  if (g.nP < 1 || (l->R + l->stride - 1) / l->stride * g.nP > 49 || l->R * g.nP > 255) return g;
+  g.ok = true;
+  return g;
+}
+
 void set_x_layout(PrepArgs* pa, const efqat_layer_desc* l) {
   if (!narrow_conv(l)) return;
   pa->xp_C8 = l->Cin / 8; pa->xp_H = l->H; pa->xp_W = l->W; pa->xp_pad = l->pad;
@@ -155,6 +183,17 @@ void set_x_layout(PrepArgs* pa, const efqat_layer_desc* l) {
 int dx_partials(const efqat_layer_desc* l) {
   if (!spatial_conv(l)) return gemm_dx_num_partials(l->M, l->K);
   int64_t n = 0;
+  const StripGeo sg = strip_geo(l);
+  if (sg.ok) {
+    for (int ah = 0; ah < l->stride; ++ah) {
+      const int64_t Hc = ceil_div(l->H - ah, l->stride);
+      if (Hc < 1) continue;
+      int tw, th, tb;
+      conv_pixel_box(l->W / sg.P, static_cast<int>(Hc), l->B, 128, &tw, &th, &tb);
+      n += ceil_div(l->W / sg.P, tw) * ceil_div(Hc, th) * ceil_div(l->B, tb) * 8;
+    }
+    return static_cast<int>(n);
+  }
   for (int ah = 0; ah < l->stride; ++ah)
     for (int aw = 0; aw < l->stride; ++aw) {
       const int64_t Wc = ceil_div(l->W - aw, l->stride), Hc = ceil_div(l->H - ah, l->stride);
@@ -202,6 +241,8 @@ LayerWs carve(void* ws, const efqat_layer_desc* l, int64_t k_sel, int sm_count, 
   w.dxpart = reinterpret_cast<float*>(take(static_cast<int64_t>(dx_partials(l)) * 8));
   w.colsum = reinterpret_cast<float*>(take(static_cast<int64_t>(prepare_slabs(M, N)) * N * 4));
   w.wsum = reinterpret_cast<int32_t*>(take(N * 4));
+  const StripGeo sg = strip_geo(l);
+  w.strip = reinterpret_cast<bf16*>(take(sg.ok ? N * l->R * sg.nP * 64 * 2 : 0));
   w.bytes = off + 256;
   return w;
 }
@@ -624,6 +665,70 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
     if (!sconv) {
       rc = timed_gemm(ctx, 1, g, st, &tiles, &dx_grid);
       if (rc != EFQAT_OK) return rc;
+    } else if (strip_geo(layer).ok) {
+      // few input channels: strips of P pixels as GEMM rows, one launch per class of input rows
+      const StripGeo sg = strip_geo(layer);
+      StripArgs sa = {};
+      sa.what = cache ? wc.what : w.Wq; sa.T = w.strip; sa.N = N;
+      sa.R = layer->R; sa.S = layer->S; sa.Cin = layer->Cin; sa.pad = layer->pad; sa.stride = layer->stride;
+      sa.p_min = sg.p_min; sa.nP = sg.nP;
+      launch_strip_weights(sa, st);
+      const int es = act_bf16 ? 2 : 4;
+      const int64_t Ho = cv_dx.Ho, Wo = cv_dx.Wo, Cin = layer->Cin, Wd = layer->W, Hd = layer->H;
+      g.B = w.strip;
+      g.Nc = 64;
+      g.Kc = static_cast<int64_t>(layer->R) * sg.nP * N;
+      g.ldo = 64;
+      for (int ah = 0; ah < layer->stride; ++ah) {
+        const int64_t Hc = ceil_div(Hd - ah, static_cast<int64_t>(layer->stride));
+        if (Hc < 1) continue;
+        ConvExplicit ex = {};
+        ex.pW = static_cast<int>(Wd / sg.P);
+        ex.pH = static_cast<int>(Hc);
+        for (int r = 0; r < layer->R; ++r) {
+          const int nh = ah + layer->pad - r;
+          if (nh % layer->stride != 0) continue;
+          for (int pi = 0; pi < sg.nP; ++pi) {
+            const int p = sg.p_min + pi;
+            const int dwv = p >= 0 ? p / sg.Q : -((-p + sg.Q - 1) / sg.Q);     // floor(p / Q)
+            const int t = ex.ntaps++;
+            ex.tap_dh[t] = static_cast<int8_t>(nh / layer->stride);
+            ex.tap_dw[t] = static_cast<int8_t>(dwv);
+            ex.tap_map[t] = static_cast<uint8_t>(p - dwv * sg.Q);
+            ex.tap_rs[t] = static_cast<uint8_t>(r * sg.nP + pi);
+          }
+        }
+        for (int pm = 0; pm < sg.Q; ++pm) {
+          ConvView& v = ex.a_view[pm];
+          v.base = reinterpret_cast<const char*>(dYb) + static_cast<int64_t>(pm) * N * 2;
+          v.W = Wo > pm ? ceil_div(Wo - pm, static_cast<int64_t>(sg.Q)) : 1;
+          v.H = Ho;
+          v.pix = static_cast<int64_t>(sg.Q) * N; v.row = Wo * N; v.img = Ho * Wo * N;
+        }
+        ex.o_view.base = static_cast<char*>(dX) + static_cast<int64_t>(ah) * Wd * Cin * es;
+        ex.x_base = static_cast<const char*>(X) + static_cast<int64_t>(ah) * Wd * Cin * es;
+        ex.o_view.W = Wd / sg.P; ex.o_view.H = Hc;
+        ex.o_view.pix = 64; ex.o_view.row = static_cast<int64_t>(layer->stride) * Wd * Cin; ex.o_view.img = Hd * Wd * Cin;
+        ex.b_cols = static_cast<int64_t>(layer->R) * sg.nP * 64;
+        cv_dx.ex = &ex;
+        if (ex.ntaps == 0) {
+          // no filter row reaches this class of input rows: its gradient is zero
+          for (int b = 0; b < layer->B; ++b)
+            if (cudaMemset2DAsync(static_cast<char*>(dX) + (static_cast<int64_t>(b) * Hd + ah) * Wd * Cin * es,
+                                  static_cast<size_t>(layer->stride) * Wd * Cin * es, 0,
+                                  static_cast<size_t>(Wd) * Cin * es, static_cast<size_t>(Hc), st) != cudaSuccess)
+              return EFQAT_ERR_CUDA;
+          continue;
+        }
+        g.Mr = static_cast<int64_t>(layer->B) * Hc * (Wd / sg.P);
+        g.partials = w.dxpart + 2 * static_cast<int64_t>(tiles);
+        int t1 = 0, g1 = 0;
+        rc = timed_gemm(ctx, 1, g, st, &t1, &g1);
+        cv_dx.ex = nullptr;
+        if (rc != EFQAT_OK) return rc;
+        tiles += t1;
+        if (g1 > dx_grid) dx_grid = g1;
+      }
     } else {
       // One launch per class of input pixels (a single class for stride 1).  Classes that no
       // filter tap reaches (a 1x1 filter with stride 2 reads one pixel in four) get no launch:

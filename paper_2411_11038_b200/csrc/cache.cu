@@ -87,6 +87,37 @@ __global__ void __launch_bounds__(256) weight_cache_kernel(const CacheArgs a) {
 
 }  // namespace
 
+// Banded weight matrix of the strip form of a grad-input (see StripArgs): column block (r, p) holds,
+// for the P pixels q of a strip and the Cin channels c, the filter coefficient that connects output
+// column strip * P / stride + p with input column strip * P + q, i.e. filter column
+// s = q + pad - stride * p, or zero when that lies outside the filter.
+__global__ void __launch_bounds__(256) strip_weights_kernel(const StripArgs a) {
+  pdl_trigger();
+  pdl_wait();
+  const int64_t cols = static_cast<int64_t>(a.R) * a.nP * 64;
+  const int64_t total = a.N * cols;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t n = i / cols;
+    const int col = static_cast<int>(i - n * cols);
+    const int blk = col >> 6, j = col & 63;
+    const int r = blk / a.nP, p = a.p_min + (blk - r * a.nP);
+    const int q = j / a.Cin, c = j - q * a.Cin;
+    const int s = q + a.pad - a.stride * p;
+    bf16 v = __float2bfloat16(0.f);
+    if (s >= 0 && s < a.S) v = a.what[n * (static_cast<int64_t>(a.R) * a.S * a.Cin) + (static_cast<int64_t>(r) * a.S + s) * a.Cin + c];
+    a.T[i] = v;
+  }
+}
+
+void launch_strip_weights(const StripArgs& a, cudaStream_t st) {
+  const int64_t total = a.N * a.R * a.nP * 64;
+  int64_t grid = ceil_div(total, 256 * 4);
+  if (grid > 148 * 8) grid = 148 * 8;
+  count_launches(1);
+  launch_dependent(strip_weights_kernel, static_cast<unsigned>(grid), 256, 0, st, 1, a);
+}
+
 void launch_weight_cache(const CacheArgs& a, cudaStream_t st) {
   if (a.rows < 1) return;
   int64_t grid = ceil_div(a.rows, 8);

@@ -1088,14 +1088,29 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   if (cv) {
     if (cv->mode < 1 || cv->mode > 3 || cs < 1 || cs > 2 || cv->R * cv->S > MAX_TAPS) return EFQAT_ERR_UNIMPL;
     if (cv->mode == 2) {           // grad-input tiles must not straddle the end of Cin (B is not zero there)
-      p.BN = (cv->Cin % 256 == 0) ? 256 : (cv->Cin % 192 == 0) ? 192 : (cv->Cin % 128 == 0) ? 128 : 64;
-      if (cv->cls_h < 0 || cv->cls_h >= cs || cv->cls_w < 0 || cv->cls_w >= cs) return EFQAT_ERR_SHAPE;
-      cWc = static_cast<int>(ceil_div(cv->W - cv->cls_w, cs));
-      cHc = static_cast<int>(ceil_div(cv->H - cv->cls_h, cs));
+      const int64_t ncols = cv->ex ? a.Nc : cv->Cin;
+      p.BN = (ncols % 256 == 0) ? 256 : (ncols % 192 == 0) ? 192 : (ncols % 128 == 0) ? 128 : 64;
+      if (cv->ex) {
+        cWc = cv->ex->pW;
+        cHc = cv->ex->pH;
+      } else {
+        if (cv->cls_h < 0 || cv->cls_h >= cs || cv->cls_w < 0 || cv->cls_w >= cs) return EFQAT_ERR_SHAPE;
+        cWc = static_cast<int>(ceil_div(cv->W - cv->cls_w, cs));
+        cHc = static_cast<int>(ceil_div(cv->H - cv->cls_h, cs));
+      }
     }
     // filter taps of this launch
     ConvP& c = p.cv;
     c.ntaps = 0;
+    if (cv->mode == 2 && cv->ex) {
+      const ConvExplicit& ex = *cv->ex;
+      if (ex.ntaps < 0 || ex.ntaps > MAX_TAPS) return EFQAT_ERR_SHAPE;
+      c.ntaps = ex.ntaps;
+      for (int t = 0; t < ex.ntaps; ++t) {
+        c.tap_dh[t] = ex.tap_dh[t]; c.tap_dw[t] = ex.tap_dw[t];
+        c.tap_map[t] = ex.tap_map[t]; c.tap_rs[t] = ex.tap_rs[t];
+      }
+    } else
     for (int r = 0; r < cv->R; ++r)
       for (int sx = 0; sx < cv->S; ++sx) {
         int dh, dw, mi = 0;
@@ -1222,7 +1237,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     c.dimH = pH; c.dimB = cv->B;
     c.C = (cv->mode == 2) ? cv->N : cv->Cin;
     c.cchunks = static_cast<int>(ceil_div(c.C, 64));
-    c.wcols = cv->Cin;
+    c.wcols = (cv->mode == 2 && cv->ex) ? 64 : cv->Cin;
     if (cv->mode == 3) {
       p.nkb = c.tiles_w * c.tiles_h * tiles_b;                 // contraction over boxes of 64 output pixels
       if (p.splits > p.nkb) return EFQAT_ERR_SHAPE;
@@ -1332,7 +1347,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
     }
   } else {
     const ConvP& c = p.cv;
-    const int64_t KK = static_cast<int64_t>(cv->R) * cv->S * cv->Cin;
+    const int64_t KK = (cv->mode == 2 && cv->ex) ? cv->ex->b_cols : static_cast<int64_t>(cv->R) * cv->S * cv->Cin;
     // quarter of a 128-pixel box: the 32 rows one epilogue warp owns
     const int qh = (32 / c.tw < c.th) ? 32 / c.tw : c.th;
     const int qb = 32 / (c.tw * qh);
@@ -1363,6 +1378,19 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       if (rc == EFQAT_OK)
         rc = make_map_4d(&to, a.out, a.out_bf16, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, qh, qb, 64);
       tx = ta;
+    } else if (cv->mode == 2 && cv->ex) {
+      const ConvExplicit& ex = *cv->ex;
+      CUtensorMap* maps[4] = {&ta, &tcls[0], &tcls[1], &tcls[2]};
+      for (int i = 0; i < 4 && rc == EFQAT_OK; ++i) {
+        const ConvView& v = ex.a_view[ex.a_view[i].base ? i : 0];
+        rc = make_map_4d(maps[i], v.base, 1, cv->B, v.H, v.W, cv->N, cv->N, c.tw, c.th, c.tb, 128, v.pix, v.row, v.img);
+      }
+      if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, BK);
+      const ConvView& o = ex.o_view;
+      if (rc == EFQAT_OK)
+        rc = make_map_4d(&to, o.base, a.out_bf16, cv->B, o.H, o.W, a.Nc, a.Nc, c.tw, qh, qb, 64, o.pix, o.row, o.img);
+      if (rc == EFQAT_OK)
+        rc = make_map_4d(&tx, ex.x_base, a.out_bf16, cv->B, o.H, o.W, a.Nc, a.Nc, c.tw, qh, qb, 64, o.pix, o.row, o.img);
     } else if (cv->mode == 2) {
       rc = make_map_4d(&ta, a.A, 1, cv->B, cv->Ho, cv->Wo, cv->N, cv->N, c.tw, c.th + (p.colshare ? p.colshare - 1 : 0), c.tb);
       tcls[0] = tcls[1] = tcls[2] = ta;

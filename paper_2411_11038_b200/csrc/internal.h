@@ -155,7 +155,34 @@ enum GemmEpi { EPI_FWD = 0, EPI_DX = 1, EPI_PART = 2, EPI_FWD_I8 = 3 };   // EPI
 //   mode 2 grad-in : A = dY [B,Ho,Wo,N] patches, B = W^ [N, R*S*Cin] (MN-major), D = dX [B,H,W,Cin]
 //   mode 3 grad-w  : A = Xc patches (MN-major), B = gathered dY [B,Ho,Wo,pitch] (MN-major),
 //                    D[(r,s,c), i] partial products, contraction over output pixels
+// A view of an NHWC tensor as W x H pixels per image with explicit pitches (elements).
+struct ConvView { const void* base; int64_t W, H, pix, row, img; };
+// A grad-input launch (mode 2) described directly instead of through (R, S, pad, stride, class):
+// the pixel space it tiles, its filter taps and the views of dY (by tap_map), of dX and of X.
+struct ConvExplicit {
+  int pW, pH;                       // pixel space of the launch (images: ConvArgs::B); columns of D: GemmArgs::Nc
+  int ntaps;
+  int8_t tap_dh[49], tap_dw[49];    // tap t reads the dY view tap_map[t] shifted by (tap_dw, tap_dh) pixels
+  uint8_t tap_map[49], tap_rs[49];  // ... against columns [64 tap_rs[t], 64 tap_rs[t] + Nc) of the B matrix
+  ConvView a_view[4];
+  const void* x_base;               // dX (GemmArgs::out) and X share the pitches of o_view; X starts here
+  ConvView o_view;
+  int64_t b_cols;                   // columns (row pitch) of the B matrix [N, b_cols]
+};
+
+// Strip form of the grad-input of a convolution with few input channels (P = 64 / Cin input pixels
+// of one row are one output row of the GEMM): the banded weight matrix T [N, R * nP * 64] built
+// from the dequantised weights what [N, R * S * Cin]; nP = number of output columns p_min .. that
+// reach a strip.
+struct StripArgs {
+  const bf16* what; bf16* T;
+  int64_t N;
+  int R, S, Cin, pad, stride, p_min, nP;
+};
+void launch_strip_weights(const StripArgs& a, cudaStream_t st);
+
 struct ConvArgs {
+  const ConvExplicit* ex;           // null: derived from the fields below
   int mode;
   int B, H, W, Cin;     // input activation tensor
   int Ho, Wo, N;        // output activation tensor

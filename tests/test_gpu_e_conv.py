@@ -50,6 +50,12 @@ CASES = [
     _case("c3x3_cin16_s2_odd", 2, 11, 13, 16, 72, 3, 1, seed=21, stride=2),
     _case("c5x5_cin8_valid", 3, 12, 9, 8, 64, 5, 0, w_bits=8, seed=22),
     _case("c3x3_cin16_pad2", 2, 9, 9, 16, 64, 3, 2, seed=23),
+    # ... and grad-input on strips of 64 / Cin pixels where the width allows it
+    _case("c3x3_cin16_strip", 2, 9, 12, 16, 72, 3, 1, seed=29),
+    _case("c2x2_cin32_s2_strip", 2, 8, 16, 32, 64, 2, 0, seed=30, stride=2),
+    _case("c5x5_cin8_s2_strip", 2, 10, 16, 8, 64, 5, 2, w_bits=8, seed=31, stride=2),
+    _case("c7x7_cin8_s2_strip_b2", 2, 30, 32, 8, 72, 7, 3, seed=32, stride=2),
+    _case("c3x3_cin16_strip_f32", 1, 8, 8, 16, 64, 3, 1, dtype=torch.float32, seed=33),
     # extents that 8-, 16- or 32-pixel-wide one-image boxes tile well: the taps of a filter column share one box
     _case("c3x3_shared_30x15", 2, 15, 30, 64, 72, 3, 1, seed=24),
     _case("c3x3_shared_cin128", 2, 16, 24, 128, 136, 3, 1, seed=25),

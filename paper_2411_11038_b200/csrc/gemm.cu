@@ -211,7 +211,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     prefetch_tmap(&tmB);
     if (EPI != EPI_PART) prefetch_tmap(&tmOut);
     if (EPI == EPI_DX) prefetch_tmap(&tmX);
-    if (p.cv.mode == 1 || p.cv.mode == 3) {
+    if (p.cv.mode != 0) {
       prefetch_tmap(&tmA1);
       prefetch_tmap(&tmA2);
       prefetch_tmap(&tmA3);
@@ -413,7 +413,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               if (do_a) {
                 if (p.colshare) {
                   // the first tap of the filter column (smallest row shift) brings the box of all of them
-                  if (u == 0) tma_load_4d(a_reg, &tmA, &ctl->full[s], cc * 64, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
+                  if (u == 0) {
+                    const int mi = p.cv.tap_map[t];
+                    const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
+                    tma_load_4d(a_reg, ma, &ctl->full[s], cc * 64, w0 + p.cv.tap_dw[t], h0 + p.cv.tap_dh[t], b0);
+                  }
                 } else {
                   const int mi = p.cv.tap_map[t];
                   const CUtensorMap* ma = mi == 0 ? &tmA : (mi == 1 ? &tmA1 : (mi == 2 ? &tmA2 : &tmA3));
@@ -1139,27 +1143,29 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       if (grid_out) *grid_out = 0;
       return EFQAT_OK;
     }
-    // Column sharing: the taps must form a grid of filter columns (one dw each) x rows with
-    // consecutive dh, all through one tensor map; they are then re-ordered column by column,
+    // Column sharing: the taps must form groups of equal size, each with one tensor map, one dw and
+    // consecutive dh (the rows of one filter column); they are then re-ordered group by group,
     // smallest row shift first.
     if ((cv->mode == 2 || (cv->mode == 1 && cs == 1)) && c.ntaps >= 2) {
       int order[MAX_TAPS], n = c.ntaps, per_col = 0;
       for (int j = 0; j < n; ++j) order[j] = j;
-      for (int i = 1; i < n; ++i)                         // insertion sort by (dw, dh)
+      for (int i = 1; i < n; ++i)                         // insertion sort by (map, dw, dh)
         for (int j = i; j > 0; --j) {
           const int x = order[j - 1], y = order[j];
-          if (c.tap_dw[x] < c.tap_dw[y] || (c.tap_dw[x] == c.tap_dw[y] && c.tap_dh[x] <= c.tap_dh[y])) break;
+          const int kx = c.tap_map[x] * 256 + c.tap_dw[x], ky = c.tap_map[y] * 256 + c.tap_dw[y];
+          if (kx < ky || (kx == ky && c.tap_dh[x] <= c.tap_dh[y])) break;
           order[j - 1] = y; order[j] = x;
         }
       bool grid = true;
       for (int first = 0; first < n && grid;) {
         int last = first + 1;
-        while (last < n && c.tap_dw[order[last]] == c.tap_dw[order[first]]) ++last;
+        while (last < n && c.tap_dw[order[last]] == c.tap_dw[order[first]] &&
+               c.tap_map[order[last]] == c.tap_map[order[first]]) ++last;
         const int cnt = last - first;
         if (per_col == 0) per_col = cnt;
-        if (cnt != per_col || c.tap_map[order[first]] != 0) grid = false;
+        if (cnt != per_col) grid = false;
         for (int j = first + 1; j < last && grid; ++j)
-          if (c.tap_dh[order[j]] != c.tap_dh[order[j - 1]] + 1 || c.tap_map[order[j]] != 0) grid = false;
+          if (c.tap_dh[order[j]] != c.tap_dh[order[j - 1]] + 1) grid = false;
         first = last;
       }
       if (grid && n == c.ntaps && per_col >= 2 && per_col <= 4) {
@@ -1383,7 +1389,8 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       CUtensorMap* maps[4] = {&ta, &tcls[0], &tcls[1], &tcls[2]};
       for (int i = 0; i < 4 && rc == EFQAT_OK; ++i) {
         const ConvView& v = ex.a_view[ex.a_view[i].base ? i : 0];
-        rc = make_map_4d(maps[i], v.base, 1, cv->B, v.H, v.W, cv->N, cv->N, c.tw, c.th, c.tb, 128, v.pix, v.row, v.img);
+        rc = make_map_4d(maps[i], v.base, 1, cv->B, v.H, v.W, cv->N, cv->N, c.tw, c.th + (p.colshare ? p.colshare - 1 : 0),
+                         c.tb, 128, v.pix, v.row, v.img);
       }
       if (rc == EFQAT_OK) rc = make_map(&tb, a.B, 1, cv->N, KK, KK, BK);
       const ConvView& o = ex.o_view;

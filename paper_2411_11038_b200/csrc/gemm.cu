@@ -1088,7 +1088,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   const ConvArgs* cv = a.conv;
   const int cs = cv ? cv->stride : 1;           // convolution stride
   int cWc = 0, cHc = 0;                         // grad-input: extent of this launch's pixel class
-  int col_order[MAX_TAPS];                      // taps column by column (column sharing)
+  ConvP col_taps = {};                          // the taps re-ordered (and filled up) for column sharing
   if (cv) {
     if (cv->mode < 1 || cv->mode > 3 || cs < 1 || cs > 2 || cv->R * cv->S > MAX_TAPS) return EFQAT_ERR_UNIMPL;
     if (cv->mode == 2) {           // grad-input tiles must not straddle the end of Cin (B is not zero there)
@@ -1143,11 +1143,13 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       if (grid_out) *grid_out = 0;
       return EFQAT_OK;
     }
-    // Column sharing: the taps must form groups of equal size, each with one tensor map, one dw and
-    // consecutive dh (the rows of one filter column); they are then re-ordered group by group,
-    // smallest row shift first.
-    if ((cv->mode == 2 || (cv->mode == 1 && cs == 1)) && c.ntaps >= 2) {
-      int order[MAX_TAPS], n = c.ntaps, per_col = 0;
+    // Column sharing: the taps must form groups, each with one tensor map, one dw and consecutive
+    // dh (the rows of one filter column); they are then re-ordered group by group, smallest row
+    // shift first.  Groups of unequal size (a strided forward reads even and odd filter rows
+    // through different maps) are filled up with taps whose weight columns lie past the end of the
+    // weight matrix, i.e. read as zeros, as long as that adds at most 15 % of blocks.
+    if ((cv->mode == 2 || cv->mode == 1) && c.ntaps >= 2) {
+      int order[MAX_TAPS], n = c.ntaps, gmax = 0, groups = 0;
       for (int j = 0; j < n; ++j) order[j] = j;
       for (int i = 1; i < n; ++i)                         // insertion sort by (map, dw, dh)
         for (int j = i; j > 0; --j) {
@@ -1161,16 +1163,33 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
         int last = first + 1;
         while (last < n && c.tap_dw[order[last]] == c.tap_dw[order[first]] &&
                c.tap_map[order[last]] == c.tap_map[order[first]]) ++last;
-        const int cnt = last - first;
-        if (per_col == 0) per_col = cnt;
-        if (cnt != per_col) grid = false;
+        if (last - first > gmax) gmax = last - first;
+        ++groups;
         for (int j = first + 1; j < last && grid; ++j)
           if (c.tap_dh[order[j]] != c.tap_dh[order[j - 1]] + 1) grid = false;
         first = last;
       }
-      if (grid && n == c.ntaps && per_col >= 2 && per_col <= 4) {
-        p.colshare = per_col;
-        for (int j = 0; j < n; ++j) col_order[j] = order[j];
+      const int padded = groups * gmax;
+      const bool may_pad = cv->mode == 1 && !a.b_mn && cv->R * cv->S < 255;
+      if (grid && gmax >= 2 && gmax <= 4 && padded <= MAX_TAPS &&
+          (padded == n || (may_pad && padded * 20 <= n * 23))) {
+        p.colshare = gmax;
+        col_taps = c;
+        int m = 0;
+        for (int first = 0; first < n;) {
+          int last = first + 1;
+          while (last < n && c.tap_dw[order[last]] == c.tap_dw[order[first]] &&
+                 c.tap_map[order[last]] == c.tap_map[order[first]]) ++last;
+          for (int j = 0; j < gmax; ++j, ++m) {
+            const int src = order[first + j < last ? first + j : last - 1];
+            col_taps.tap_dh[m] = static_cast<int8_t>(c.tap_dh[order[first]] + j);
+            col_taps.tap_dw[m] = c.tap_dw[src];
+            col_taps.tap_map[m] = c.tap_map[src];
+            col_taps.tap_rs[m] = first + j < last ? c.tap_rs[src] : static_cast<uint8_t>(cv->R * cv->S);
+          }
+          first = last;
+        }
+        col_taps.ntaps = m;
       }
     }
   }
@@ -1219,7 +1238,7 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
       if (fits) {
         const int a_reg = static_cast<int>(round_up((th2 + p.colshare - 1) * tw2 * 128, 1024));
         const int b_st = static_cast<int>(round_up(a.b_mn ? ceil_div(bn_cta, 64) * CHUNK_BYTES : bn_cta * BK * 2, 1024));
-        const int nkb2 = c.ntaps * static_cast<int>(ceil_div((cv->mode == 2) ? cv->N : cv->Cin, 64));
+        const int nkb2 = col_taps.ntaps * static_cast<int>(ceil_div((cv->mode == 2) ? cv->N : cv->Cin, 64));
         const int ring = ring_budget(a.epi);
         const bool res = p.tiles_n == 1 && static_cast<int64_t>(nkb2) * b_st + 2 * a_reg <= ring;
         fits = res || ring / (a_reg + p.colshare * b_st) >= 2;
@@ -1228,10 +1247,10 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
           p.bres = res ? 1 : 0;
           p.a_region_bytes = a_reg;
           p.a_tx = (th2 + p.colshare - 1) * tw2 * 128;
-          const ConvP o = c;
+          c.ntaps = col_taps.ntaps;
           for (int j = 0; j < c.ntaps; ++j) {
-            c.tap_dh[j] = o.tap_dh[col_order[j]]; c.tap_dw[j] = o.tap_dw[col_order[j]];
-            c.tap_map[j] = o.tap_map[col_order[j]]; c.tap_rs[j] = o.tap_rs[col_order[j]];
+            c.tap_dh[j] = col_taps.tap_dh[j]; c.tap_dw[j] = col_taps.tap_dw[j];
+            c.tap_map[j] = col_taps.tap_map[j]; c.tap_rs[j] = col_taps.tap_rs[j];
           }
         }
       }

@@ -180,35 +180,37 @@ void set_x_layout(PrepArgs* pa, const efqat_layer_desc* l) {
 
 // (dS_x, dZ_x) partial pairs of the grad-input launches: for a convolution, one launch per class
 // of input pixels (stride x stride classes), each tiled by its own pixel box.
+// Upper bound of the 128-pixel boxes a grad-input launch may cut a W x H x B pixel space into: the
+// least-waste box, or one of the one-image boxes of a launch whose taps share boxes per filter column.
+int64_t dx_boxes(int64_t Wc, int64_t Hc, int64_t Bn) {
+  int tw, th, tb;
+  conv_pixel_box(static_cast<int>(Wc), static_cast<int>(Hc), static_cast<int>(Bn), 128, &tw, &th, &tb);
+  int64_t boxes = ceil_div(Wc, tw) * ceil_div(Hc, th) * ceil_div(Bn, tb);
+  const int cand[2][2] = {{8, 16}, {16, 8}};
+  for (int i = 0; i < 2; ++i) {
+    const int64_t b2 = ceil_div(Wc, cand[i][0]) * ceil_div(Hc, cand[i][1]) * Bn;
+    if (b2 * 128 <= (23 * Wc * Hc * Bn) / 20 + 128 && b2 > boxes) boxes = b2;
+  }
+  return boxes;
+}
+
 int dx_partials(const efqat_layer_desc* l) {
   if (!spatial_conv(l)) return gemm_dx_num_partials(l->M, l->K);
   int64_t n = 0;
   const StripGeo sg = strip_geo(l);
-  if (sg.ok) {
-    for (int ah = 0; ah < l->stride; ++ah) {
-      const int64_t Hc = ceil_div(l->H - ah, l->stride);
-      if (Hc < 1) continue;
-      int tw, th, tb;
-      conv_pixel_box(l->W / sg.P, static_cast<int>(Hc), l->B, 128, &tw, &th, &tb);
-      n += ceil_div(l->W / sg.P, tw) * ceil_div(Hc, th) * ceil_div(l->B, tb) * 8;
+  for (int ah = 0; ah < l->stride; ++ah) {
+    const int64_t Hc = ceil_div(l->H - ah, l->stride);
+    if (Hc < 1) continue;
+    if (sg.ok) {                      // strips of P pixels: one launch per class of input rows, 64 columns
+      n += dx_boxes(l->W / sg.P, Hc, l->B) * 8;
+      continue;
     }
-    return static_cast<int>(n);
-  }
-  for (int ah = 0; ah < l->stride; ++ah)
     for (int aw = 0; aw < l->stride; ++aw) {
-      const int64_t Wc = ceil_div(l->W - aw, l->stride), Hc = ceil_div(l->H - ah, l->stride);
-      if (Wc < 1 || Hc < 1) continue;
-      int tw, th, tb;
-      conv_pixel_box(static_cast<int>(Wc), static_cast<int>(Hc), l->B, 128, &tw, &th, &tb);
-      int64_t boxes = ceil_div(Wc, tw) * ceil_div(Hc, th) * ceil_div(l->B, tb);
-      // the launch may tile the class with one-image boxes instead (taps sharing a box per filter column)
-      const int cand[2][2] = {{8, 16}, {16, 8}};
-      for (int i = 0; i < 2; ++i) {
-        const int64_t b2 = ceil_div(Wc, cand[i][0]) * ceil_div(Hc, cand[i][1]) * l->B;
-        if (b2 <= (23 * Wc * Hc * l->B) / (20 * 128) + 1 && b2 > boxes) boxes = b2;
-      }
-      n += boxes * ceil_div(l->Cin, 64) * 8;
+      const int64_t Wc = ceil_div(l->W - aw, l->stride);
+      if (Wc < 1) continue;
+      n += dx_boxes(Wc, Hc, l->B) * ceil_div(l->Cin, 64) * 8;
     }
+  }
   return static_cast<int>(n);
 }
 
@@ -661,6 +663,7 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
     g.s_x = s_x; g.z_x = z_x; g.x_bits = q->x_bits; g.x_sym = q->x_symmetric;
     g.X = X; g.x_dtype = layer->act_dtype;
     g.partials = w.dxpart;
+    g.partials_cap = dx_partials(layer);
     g.status = ctx->d_status;
     if (!sconv) {
       rc = timed_gemm(ctx, 1, g, st, &tiles, &dx_grid);
@@ -722,6 +725,7 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
         }
         g.Mr = static_cast<int64_t>(layer->B) * Hc * (Wd / sg.P);
         g.partials = w.dxpart + 2 * static_cast<int64_t>(tiles);
+        g.partials_cap = dx_partials(layer) - tiles;
         int t1 = 0, g1 = 0;
         rc = timed_gemm(ctx, 1, g, st, &t1, &g1);
         cv_dx.ex = nullptr;
@@ -742,6 +746,8 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
           cv_dx.cls_h = ah;
           cv_dx.cls_w = aw;
           g.partials = w.dxpart + 2 * static_cast<int64_t>(tiles);
+          g.partials_cap = dx_partials(layer) - tiles;
+        g.partials_cap = dx_partials(layer) - tiles;
           int t1 = 0, g1 = 0;
           rc = timed_gemm(ctx, 1, g, st, &t1, &g1);
           if (rc != EFQAT_OK) return rc;

@@ -1436,6 +1436,10 @@ int run_gemm(const GemmArgs& a, int sm_count, cudaStream_t st, int* tiles_out, i
   const int units = static_cast<int>(items < max_units ? items : max_units);
   const int grid = pair ? 2 * units : units;
   const size_t smem = static_cast<size_t>(stages) * stage_bytes + bres_bytes + fixed_bytes + 1024;
+  // the (dS_x, dZ_x) pairs this launch writes must fit what the caller set aside for them
+  if (a.epi == EPI_DX && a.partials_cap > 0 &&
+      static_cast<int64_t>(p.tiles_m) * p.tiles_n * (pair ? 2 : 1) * EPI_WARPS > a.partials_cap)
+    return EFQAT_ERR_WORKSPACE;
   if (tiles_out) *tiles_out = p.tiles_m * p.tiles_n * (pair ? 2 : 1) * EPI_WARPS;
   if (grid_out) *grid_out = grid;
 

@@ -222,6 +222,7 @@ struct GemmArgs {
   const void* X;     // raw activations [Mr,Nc] in x_dtype
   int x_dtype;
   float* partials;   // [gemm_dx_num_partials][2]
+  int64_t partials_cap;   // EPI_DX: pairs available at `partials` (0: not checked)
   // EPI_PART: out[split*split_stride + col*ldo + row], col < part_cols only
   int splits;
   int64_t split_stride;

@@ -45,13 +45,23 @@ def _conv_sub(case, T, images):
     return c, dict(X=T["X"][images].contiguous(), W=T["W"], dY=T["dY"][images].contiguous(), bias=T["bias"])
 
 
-@pytest.mark.parametrize("li", range(8))
+def _batch64_cases():
+    """The eight ResNet-50-shaped layers of configs[2], then layers of the real network that take
+    other launch forms: the 7x7 stride-2 input layer on 8 stored channels (filter rows as
+    contraction blocks, grad-input on strips of 8 pixels), the first stage's 3x3 64 -> 64 (taps of a
+    filter column sharing one box, weights resident in shared memory) and the stride-2 3x3 that
+    opens the second stage."""
+    rn = {c.name: c for c in I.resnet50(64)}
+    return I.config3() + [rn["rn50_stem"], rn["rn50_s1b1_b"], rn["rn50_s2b1_b"]]
+
+
+@pytest.mark.parametrize("li", range(11))
 def test_config3_layer_batch64(ctx, li):
-    case = I.config3()[li]
+    case = _batch64_cases()[li]
     T = I.make_tensors(case)
     s_w, s_x, z_x = U.oracle_qparams(case, T, (0.6, 0.9, 0.0))       # shrunk scales: both tensors clip
     D = U.to_dev(T, s_w, s_x, z_x)
-    geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, 1, case.pad)
+    geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, case.stride, case.pad)
     N, K = case.N, case.K
     k = B.ratio_to_k(0.10, N)
     W64 = I.as_f64(T["W"])
@@ -73,12 +83,12 @@ def test_config3_layer_batch64(ctx, li):
     torch.cuda.synchronize()
     assert ctx.device_status() == 0
     name = case.name
-    ref = O.conv_forward(Xs, W64, s_w, s_x, z_x, b64, case.w_bits, case.x_bits, 1, case.pad)
+    ref = O.conv_forward(Xs, W64, s_w, s_x, z_x, b64, case.w_bits, case.x_bits, case.stride, case.pad)
     got = _np(Y[images])
     U.assert_bf16_class(got, ref, name + " Y")
     U.assert_fp32_class(got, ref, Yabs + np.abs(b64), name + " Y", out_is_bf16=True)
 
-    args = (dYs, Xs, W64, s_w, s_x, z_x, idx, case.w_bits, case.x_bits, 1, case.pad)
+    args = (dYs, Xs, W64, s_w, s_x, z_x, idx, case.w_bits, case.x_bits, case.stride, case.pad)
     ex = O.conv_backward_efqat(*args, operand_model="exact")
     bm = O.conv_backward_efqat(*args, operand_model="bf16")
     dX = _np(out["dX"][images])
@@ -103,7 +113,7 @@ def test_config3_layer_batch64(ctx, li):
     rng = np.random.default_rng(li)
     pick = np.unique(np.concatenate([[0, k - 1], rng.choice(k, 6, replace=False)]))
     d = O.conv_backward_efqat_direct(I.as_f64(T["dY"]), I.as_f64(T["X"]), W64, s_w, s_x, z_x, idx[pick],
-                                     case.w_bits, case.x_bits, 1, case.pad, operand_model="bf16")
+                                     case.w_bits, case.x_bits, case.stride, case.pad, operand_model="bf16")
     U.assert_bf16_class(dW[pick], d["dW_sel"], name + " dW_sel sampled channels")
     U.assert_fp32_class(dW[pick], d["dW_sel"], d["G_w_sel_abs"], name + " dW_sel sampled channels")
     U.assert_fp32_class(dSw[pick], d["dS_w_sel"], d["dS_w_sel_abs"], name + " dS_w sampled channels", atol=1e-30)

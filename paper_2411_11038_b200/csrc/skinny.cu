@@ -295,13 +295,14 @@ __global__ void __launch_bounds__(WS_THREADS, 1)
 skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
                      const SkinnyFwdArgs a) {
   constexpr int TILE = KB * WS_T16K;                       // one X tile / one operand buffer
-  const int WS_STAGES = a.stages;
+  constexpr int WS_STAGES = KB == 1 ? 3 : 2;               // X tiles in flight (compile time: the stage index is n % WS_STAGES)
+  constexpr int STG_BUFS = KB == 1 ? 2 : 1;                // staging buffers per epilogue warp
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* b_tile = smem;                                  // [KB][BN rows][128 B] weight codes, K-major
   uint8_t* xc_t = b_tile + KB * a.BN * 128;                // [2][KB][128 rows][128 B] centred activation codes
   uint8_t* ring = xc_t + 2 * TILE;                         // [stages][KB][128 rows][128 B] raw X tiles
   uint8_t* stage = ring + WS_STAGES * TILE;                // [8 warps][stg_bufs][32 rows][128 B] output staging
-  float* sc = reinterpret_cast<float*>(stage + 8 * a.stg_bufs * 4096);   // [BN] s_x * s_w[n]
+  float* sc = reinterpret_cast<float*>(stage + 8 * STG_BUFS * 4096);   // [BN] s_x * s_w[n]
   float* bi = sc + a.BN;                                   // [BN] bias[n]
   WsCtl* ctl = reinterpret_cast<WsCtl*>(bi + a.BN);
 
@@ -498,12 +499,12 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256;
       for (int rd = rd0; rd < rd1; ++rd, ++st_it) {
         const int c0 = rd * 64;
-        uint8_t* stg = stage + (e * a.stg_bufs + (a.stg_bufs == 2 ? (st_it & 1) : 0)) * 4096;
+        uint8_t* stg = stage + (e * STG_BUFS + (STG_BUFS == 2 ? (st_it & 1) : 0)) * 4096;
         uint32_t r[64];
         tmem_ld_32x32(t_row + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
         tmem_ld_32x32(t_row + c0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
         if (lane == 0) {
-          if (a.stg_bufs == 2) tma_store_wait_read1(); else tma_store_wait_read0();
+          if (STG_BUFS == 2) tma_store_wait_read1(); else tma_store_wait_read0();
         }
         tmem_wait_ld();
         if (rd + 1 == rd1) {                                  // the accumulator is in registers: hand it back

@@ -479,15 +479,13 @@ def measure_network(ctx, dev, sync_all, max_over_ranks):
     return out
 
 
-def measure_resnet50(ctx, dev, sync_all, max_over_ranks, batch=64):
-    """Every quantized layer of ResNet-50 (53 convolutions and the classifier) at 224 x 224, batch 64,
-    W4A8, through the same network calls: forward and backward per unfrozen ratio, network-wide
-    (CWPN) and layer-wise (LWPN).  Each layer has its own input and output-gradient tensors
-    (2.8 GB together), so nothing a layer reads is left in L2 by the one before it."""
+def measure_convnet(ctx, dev, sync_all, max_over_ranks, cases, workload, paper_context):
+    """A convolutional network's quantized layers through the network calls: forward and backward per
+    unfrozen ratio, network-wide (CWPN) and layer-wise (LWPN).  Each layer has its own input and
+    output-gradient tensors, so nothing a layer reads is left in L2 by the one before it."""
     import math
     from paper_2411_11038_b200 import binding as B
     from paper_2411_11038_b200 import network as NW
-    cases = I.resnet50(batch)
     gen = torch.Generator(device=dev)
     states = []
     for c in cases:
@@ -501,6 +499,7 @@ def measure_resnet50(ctx, dev, sync_all, max_over_ranks, batch=64):
         dY = torch.randn(yshape, generator=gen, device=dev).to(torch.bfloat16)
         states.append(NW.LayerState(c, W, X, dY, None))
     total = sum(c.N for c in cases)
+    batch = cases[0].B
     net = NW.EfqatNetwork(ctx, states, B.CWPN, B.ratio_to_k(0.1, total), f_samples=batch, batch_samples=batch,
                           use_cache=True, sgd=(SGD_LR, 0.9, 1e-4), adam=dict(lr=1e-6), share_outputs=False)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
@@ -509,10 +508,7 @@ def measure_resnet50(ctx, dev, sync_all, max_over_ranks, batch=64):
         return max_over_ranks(timed(fn, steps, warm, flush, sync_all) / steps)
 
     gemm = sum(2.0 * c.M * c.N * c.K for c in cases)
-    out = {"workload": f"ResNet-50 at 224x224, batch {batch}: 53 convolutions (7x7 stride-2 input layer on 8 stored "
-                       "channels, bottleneck blocks 3-4-6-3, stride on the 3x3, shortcuts) + classifier, W4A8, NHWC "
-                       "bf16, synthetic |N(0,1)| activations, one tensor pair per layer",
-           "layers": len(cases), "channels": total, "fwd_gflop": gemm / 1e9}
+    out = {"workload": workload, "layers": len(cases), "channels": total, "fwd_gflop": gemm / 1e9}
     rows = {}
     for mode, name, ratios in ((B.CWPN, "CWPN", (0.0, 0.05, 0.10, 0.25, 1.0)), (B.LWPN, "LWPN", (0.05, 0.10, 0.25))):
         for r in ratios:
@@ -535,9 +531,32 @@ def measure_resnet50(ctx, dev, sync_all, max_over_ranks, batch=64):
     out["fwd_ms"] = t(net.forward)
     out["fwd_tflops"] = gemm / (out["fwd_ms"] * 1e-3) / 1e12
     out["adam_and_cache_refresh_ms"] = t(net.optimizer_tail)
-    out["paper_context"] = ("Table 5 (A100, ResNet-50, f=12288): CWPN backward 0.87x / 0.86x / 0.80x of QAT speed at "
-                            "5 / 10 / 25 % (slower than QAT), LWPN 1.55x / 1.49x / 1.36x, 0 % 1.56x")
+    out["paper_context"] = paper_context
     return out
+
+
+def measure_resnet50(ctx, dev, sync_all, max_over_ranks, batch=64):
+    """Every quantized layer of ResNet-50 (53 convolutions and the classifier) at 224 x 224, batch 64,
+    W4A8 (2.8 GB of activations and gradients, one pair per layer)."""
+    return measure_convnet(
+        ctx, dev, sync_all, max_over_ranks, I.resnet50(batch),
+        f"ResNet-50 at 224x224, batch {batch}: 53 convolutions (7x7 stride-2 input layer on 8 stored channels, "
+        "bottleneck blocks 3-4-6-3, stride on the 3x3, shortcuts) + classifier, W4A8, NHWC bf16, synthetic |N(0,1)| "
+        "activations, one tensor pair per layer",
+        "Table 5 (A100, ResNet-50, f=12288): CWPN backward 0.87x / 0.86x / 0.80x of QAT speed at 5 / 10 / 25 % (slower "
+        "than QAT), LWPN 1.55x / 1.49x / 1.36x, 0 % 1.56x")
+
+
+def measure_resnet20(ctx, dev, sync_all, max_over_ranks, batch=128):
+    """The CIFAR-10 ResNet-20 (19 convolutions of 16 / 32 / 64 channels and the classifier) at 32 x 32,
+    batch 128, W4A8."""
+    return measure_convnet(
+        ctx, dev, sync_all, max_over_ranks, I.resnet20(batch),
+        f"ResNet-20 at 32x32, batch {batch}: 3x3 input layer on 8 stored channels, 3 stages x 3 basic blocks with 16 / 32 "
+        "/ 64 channels, parameter-free shortcuts, classifier stored with 16 outputs; W4A8, NHWC bf16, synthetic "
+        "|N(0,1)| activations, one tensor pair per layer",
+        "Table 5 (A100, ResNet-20, f=16384): CWPN backward 1.09x / 0.88x / 0.62x of QAT speed at 5 / 10 / 25 %, LWPN "
+        "1.55x / 1.52x / 1.28x, 0 % 1.67x")
 
 
 def run_capture(args):
@@ -610,9 +629,12 @@ def run_ours(args):
         status = status or ctx.device_status()
         torch.cuda.empty_cache()
     # ---- ResNet-50, every quantized layer: the convolutional counterpart
-    resnet = None
+    resnet = resnet20 = None
     if not args.skip_extras and not args.no_network:
         resnet = measure_resnet50(ctx, dev, sync_all, max_over_ranks)
+        status = status or ctx.device_status()
+        torch.cuda.empty_cache()
+        resnet20 = measure_resnet20(ctx, dev, sync_all, max_over_ranks)
         status = status or ctx.device_status()
         torch.cuda.empty_cache()
     all_clock.stop_flag = True
@@ -645,6 +667,7 @@ def run_ours(args):
             "bert_base": bert,
             "network": network,
             "resnet50": resnet,
+            "resnet20": resnet20,
             "device_status": status,
             "paper_context": "paper reports 1.44-1.64x backward speed-up on A10/A100 (whole network)",
         }))

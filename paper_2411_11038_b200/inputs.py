@@ -160,6 +160,32 @@ def resnet50(batch: int = 64) -> List[LayerCase]:
     return out
 
 
+def resnet20(batch: int = 128) -> List[LayerCase]:
+    """The 20 quantized layers of the CIFAR-10 ResNet-20 at 32 x 32: a 3x3 input layer (3 channels
+    stored as 8), three stages of three basic blocks (two 3x3 convolutions each) with 16, 32 and
+    64 channels, the first convolution of stages 2 and 3 with stride 2, parameter-free shortcuts,
+    and the classifier.  W4A8, |N(0,1)| activations."""
+    out = []
+
+    def conv(name, hw, cin, cout, stride):
+        ho = (hw + 2 - 3) // stride + 1
+        out.append(LayerCase(f"rn20_{name}", batch * ho * ho, 9 * cin, cout, w_bits=4, x_bits=8, w_std=None,
+                             x_abs=True, seed=3300 + len(out), conv=True, B=batch, H=hw, Wd=hw, Cin=cin, R=3, S=3,
+                             stride=stride, pad=1))
+        return ho
+
+    conv("stem", 32, 8, 16, 1)
+    hw, cin = 32, 16
+    for stage, width in enumerate((16, 32, 64)):
+        for b in range(3):
+            stride = 2 if (b == 0 and stage > 0) else 1
+            ho = conv(f"s{stage + 1}b{b + 1}_a", hw, cin, width, stride)
+            conv(f"s{stage + 1}b{b + 1}_b", ho, width, width, 1)
+            hw, cin = ho, width
+    out.append(LayerCase("rn20_fc", batch, 64, 16, w_bits=4, x_bits=8, w_std=None, x_abs=True, seed=3300 + len(out)))
+    return out
+
+
 def config4(layers: int = 24, M: int = 9216) -> List[LayerCase]:
     """BERT-large-shaped stack: per block Q,K,V,O 1024->1024, FFN 1024->4096->1024."""
     out = []

@@ -62,6 +62,13 @@ CASES = [
     _case("c3x3_shared_valid_f32", 1, 16, 24, 64, 64, 3, 0, dtype=torch.float32, seed=26),
     _case("c4x4_shared_s2", 2, 32, 48, 64, 64, 4, 1, seed=27, stride=2),
     _case("resnet_56_64to64_3x3_b2", 2, 56, 56, 64, 64, 3, 1, seed=28),
+    # the CIFAR-10 ResNet-20's layer shapes (16 / 32 / 64 channels on 32 x 32, 16 x 16 and 8 x 8 maps)
+    _case("resnet20_stem", 2, 32, 32, 8, 16, 3, 1, seed=34),
+    _case("resnet20_stage1", 2, 32, 32, 16, 16, 3, 1, seed=35),
+    _case("resnet20_stage2_first_s2", 2, 32, 32, 16, 32, 3, 1, seed=36, stride=2),
+    _case("resnet20_stage2", 2, 16, 16, 32, 32, 3, 1, seed=37),
+    _case("resnet20_stage3_first_s2", 3, 16, 16, 32, 64, 3, 1, seed=38, stride=2),
+    _case("resnet20_stage3", 4, 8, 8, 64, 64, 3, 1, seed=39),
     _case("resnet_56_128_3x3_s2", 2, 56, 56, 128, 128, 3, 1, seed=15, stride=2),
     _case("resnet_28_256_3x3_s2", 2, 28, 28, 256, 256, 3, 1, seed=16, stride=2),
     _case("resnet_14_512_3x3_s2", 2, 14, 14, 512, 512, 3, 1, seed=17, stride=2),

@@ -173,3 +173,56 @@ def test_training_steps_with_freezing_frequency(ctx):
     b.forward()
     for pa, pb in zip(a.plans, b.plans):
         assert torch.equal(pa.Y, pb.Y)
+
+
+def test_network_calls_on_convolutions_equal_layer_calls(ctx):
+    """A small convolutional stack through the network calls (cache on): an input layer on 8 stored
+    channels (filter rows as contraction blocks, strip-form grad-input), a 3x3 whose taps share
+    boxes per filter column, a stride-2 3x3 and a 1x1: bit-identical to the per-layer calls, and one
+    layer against the oracle."""
+    def conv_case(name, Bn, H, Wd, Cin, N, R, pad, stride, seed):
+        Ho, Wo = (H + 2 * pad - R) // stride + 1, (Wd + 2 * pad - R) // stride + 1
+        return I.LayerCase(name, Bn * Ho * Wo, R * R * Cin, N, act_dtype=torch.bfloat16, w_bits=4, x_bits=8, w_std=None,
+                           x_abs=True, seed=seed, conv=True, B=Bn, H=H, Wd=Wd, Cin=Cin, R=R, S=R, stride=stride, pad=pad)
+
+    cases = [conv_case("in7x7", 2, 32, 32, 8, 64, 7, 3, 2, 1301), conv_case("c3x3", 2, 16, 24, 64, 64, 3, 1, 1, 1302),
+             conv_case("c3x3s2", 2, 16, 24, 64, 128, 3, 1, 2, 1303), conv_case("c1x1", 2, 8, 12, 128, 64, 1, 0, 1, 1304)]
+    stack = [(c, I.make_tensors(c)) for c in cases]
+    states = [NW.LayerState(c, T["W"].cuda(), T["X"].cuda(), T["dY"].cuda(), T["bias"].cuda()) for c, T in stack]
+    total = sum(c.N for c in cases)
+    net = NW.EfqatNetwork(ctx, states, B.CWPN, B.ratio_to_k(0.25, total), f_samples=1, batch_samples=1,
+                          use_cache=True, sgd=None, adam=None, share_outputs=False)
+    net.reselect()
+    ref = O.select_cwpn([I.as_f64(T["W"]).reshape(c.N, -1) for c, T in stack], B.ratio_to_k(0.25, total))
+    assert net.counts() == [len(r) for r in ref]
+    net.forward()
+    net.backward()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for l, ((case, T), st, plan) in enumerate(zip(stack, states, net.plans)):
+        k = net.counts()[l]
+        idx = net.net.idx[net.offsets_host[l]:net.offsets_host[l] + k] if k else None
+        geom = B.ConvGeom(case.B, case.H, case.Wd, case.Cin, case.R, case.S, case.stride, case.pad)
+        Y = B.fq_linear_fwd(ctx, st.X, st.W, st.s_w, st.s_x, st.z_x, st.bias, case.w_bits, case.x_bits, False, conv=geom)
+        assert torch.equal(Y, plan.Y), f"layer {l}: network forward differs from the layer call"
+        out = B.fq_linear_bwd(ctx, st.dY, st.X, st.W, st.s_w, st.s_x, st.z_x, idx, k, case.w_bits, case.x_bits,
+                              False, want_db=True, conv=geom)
+        assert torch.equal(out["dX"], plan.dX), f"layer {l}: dX"
+        assert torch.equal(out["dW_sel"].reshape(k, case.K), plan.dW_sel[:k].reshape(k, case.K)), f"layer {l}: dW"
+        assert torch.equal(out["dS_w_sel"], plan.dS_w_sel[:k])
+        assert torch.equal(out["dS_x"], plan.dS_x) and torch.equal(out["dZ_x"], plan.dZ_x)
+        assert torch.equal(out["db"], plan.db)
+    # the input layer against the oracle (selection from the network-wide ranking)
+    case, T = stack[0]
+    st = states[0]
+    s_w, s_x, z_x = st.s_w.cpu().numpy(), np.float32(st.s_x.item()), np.float32(st.z_x.item())
+    X64, W64, dY64, b64 = (I.as_f64(T[kk]) for kk in ("X", "W", "dY", "bias"))
+    refY = O.conv_forward(X64, W64, s_w, s_x, z_x, b64, case.w_bits, case.x_bits, case.stride, case.pad)
+    U.assert_bf16_class(net.plans[0].Y.float().cpu().numpy(), refY, "input layer Y through the network call")
+    ex = O.conv_backward_efqat(dY64, X64, W64, s_w, s_x, z_x, ref[0], case.w_bits, case.x_bits, case.stride, case.pad,
+                               operand_model="exact")
+    U.assert_bf16_class(net.plans[0].dX.float().cpu().numpy(), ex["dX"], "input layer dX through the network call")
+    k0 = net.counts()[0]
+    if k0:
+        U.assert_bf16_class(net.plans[0].dW_sel[:k0].cpu().numpy().reshape(ex["dW_sel"].shape), ex["dW_sel"],
+                            "input layer dW_sel through the network call")

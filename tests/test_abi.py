@@ -118,3 +118,39 @@ def test_weight_cache_and_network_queries(lib):
     # workspace of a layer that takes the one-pass backward: one partial product per CTA
     skinny = B.layer_desc(200704, 256, 64, B.BF16)
     assert B.workspace_bytes(skinny, spec, 256) >= 148 * 256 * 64 * 4
+
+
+def test_workspace_of_the_input_layer_forms(lib):
+    """Convolutions with few input channels keep a zero-framed copy of the activation codes and the
+    banded weights of the strip-form grad-input in the workspace: the query must cover both."""
+    spec = B.QSpec(4, 8, 0)
+    conv = B.ConvGeom(B=4, H=224, W=224, Cin=8, R=7, S=7, stride=2, pad=3)
+    d = B.layer_desc(4 * 112 * 112, 64, 392, B.BF16, conv)
+    assert B.validate_layer(d, spec) == 0
+    need = 4 * 230 * 230 * 8 * 2 + 64 * 7 * 7 * 64 * 2            # framed codes + banded weights [N, R * nP * 64]
+    assert B.workspace_bytes(d, spec, 64) >= need
+    # a wide layer of the same extent keeps the dense code layout
+    conv2 = B.ConvGeom(B=4, H=56, W=56, Cin=64, R=3, S=3, stride=1, pad=1)
+    d2 = B.layer_desc(4 * 56 * 56, 64, 576, B.BF16, conv2)
+    assert B.workspace_bytes(d2, spec, 0) < 4 * 56 * 56 * 64 * 2 + 64 * 576 * 2 + (1 << 20)
+
+
+def test_network_layer_lists():
+    """The layer lists of the two convolutional networks the bench runs: counts, channels and work
+    as the architectures fix them (ResNet-50: 4.1 G multiply-adds per 224 x 224 image with the input
+    layer on 8 stored channels; ResNet-20: 41 M per 32 x 32 image)."""
+    from paper_2411_11038_b200 import inputs as I
+    r50, r20 = I.resnet50(2), I.resnet20(2)
+    assert len(r50) == 54 and sum(c.conv for c in r50) == 53 and sum(c.N for c in r50) == 26560 + 1000
+    assert len(r20) == 20 and sum(c.conv for c in r20) == 19 and sum(c.N for c in r20) == 16 + 6 * 16 + 6 * 32 + 6 * 64 + 16
+    macs50 = sum(c.M * c.N * c.K for c in r50) / 2
+    macs20 = sum(c.M * c.N * c.K for c in r20) / 2
+    assert 4.0e9 < macs50 < 4.4e9 and 40e6 < macs20 < 43e6
+    for c in r50 + r20:
+        if c.conv:
+            ho = (c.H + 2 * c.pad - c.R) // c.stride + 1
+            assert c.M == c.B * ho * ho and c.K == c.R * c.S * c.Cin
+    # consecutive layers of a stage agree in their map size: the 3x3 of a ResNet-50 block reads what its 1x1 wrote
+    by = {c.name: c for c in r50}
+    assert by["rn50_s2b1_b"].H == 56 and by["rn50_s2b1_b"].stride == 2 and by["rn50_s2b1_c"].H == 28
+    assert by["rn50_s4b3_c"].H == 7 and by["rn50_s4b3_c"].N == 2048

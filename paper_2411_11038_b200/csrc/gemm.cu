@@ -463,18 +463,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int it = 0, acc_it = 0, ring_s = 0;
       uint32_t ring_ph = 0;
       bool ok = true;
+      // This one thread is the critical path of tiles with few or narrow MMAs, so nothing it does per
+      // tile or per instruction is more than it must be: the tile's position is only computed when
+      // tiles differ in width (a ragged last tile column), the k-range only for split contractions
+      // (both need integer divisions), and the operand descriptors of a k-block are built once and
+      // advanced by adding to their address field.
+      const bool ragged_n = (p.Nc % p.BN) != 0;
+      const uint32_t idesc_full = I8 ? instr_desc_i8(TILE_M, p.BN, p.a_signed, 1) : instr_desc_bf16(TILE_M, p.BN, A_MN, B_MN);
+      const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
+      const uint32_t a_lbo = a_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
+      const uint32_t b_lbo = b_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
+      const uint32_t a_step = a_mrg ? CHUNK_BYTES : p.a_sub_off;
+      const uint32_t b_step = b_mrg ? CHUNK_BYTES : p.b_stage_bytes;
+      const uint32_t bres_base = smem_u32(bres_reg);
+      const uint32_t ring_base = smem_u32(smem);
       for (int w = unit; w < total_items && ok; w += num_units, ++acc_it) {
-        const int split = w / tiles_mn, t = w - split * tiles_mn;
-        int tm, tn;
-        tile_coords(p, t, tm, tn);
-        const int n0 = tn * p.BN;
-        int n_eff = static_cast<int>(p.Nc - n0);
-        if (n_eff > p.BN) n_eff = p.BN;
-        n_eff = (n_eff + 15) & ~15;
-        const uint32_t idesc = I8 ? instr_desc_i8(TILE_M, n_eff, p.a_signed, 1)
-                                                        : instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
-        const int kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
-        const int kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
+        uint32_t idesc = idesc_full;
+        int kb_begin = 0, kb_end = p.nkb;
+        if (ragged_n || p.splits > 1) {
+          const int split = w / tiles_mn, t = w - split * tiles_mn;
+          int tm, tn;
+          tile_coords(p, t, tm, tn);
+          const int n0 = tn * p.BN;
+          int n_eff = static_cast<int>(p.Nc - n0);
+          if (n_eff > p.BN) n_eff = p.BN;
+          n_eff = (n_eff + 15) & ~15;
+          idesc = I8 ? instr_desc_i8(TILE_M, n_eff, p.a_signed, 1) : instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
+          kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
+          kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
+        }
         const int buf = acc_it & 1;
         // wait until the epilogue has drained this accumulator (two tiles ago)
         if (*abort_flag || !mbar_wait(&ctl->acc_empty[buf], ((acc_it >> 1) & 1) ^ 1)) {
@@ -505,25 +522,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           tc_fence_after();
+          const uint32_t a_base = ring_base + s * stage_bytes;
+          const uint32_t b_base = p.bres ? bres_base + kb0 * p.b_stage_bytes : a_base + p.a_region_bytes;
          for (int u = 0; u < nsub; ++u) {
           const int kb = kb0 + u;
           // k-block u of the stage: merged MN-major operands keep their chunks kps * 8 KiB apart
-          const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
-          const uint32_t a_base = smem_u32(smem + s * stage_bytes);
-          const uint32_t b_base = a_base + p.a_region_bytes;
-          const uint32_t a_addr = a_base + u * (a_mrg ? CHUNK_BYTES : p.a_sub_off);
-          const uint32_t b_addr = p.bres ? smem_u32(bres_reg) + kb * p.b_stage_bytes
-                                         : b_base + u * (b_mrg ? CHUNK_BYTES : p.b_stage_bytes);
-          const uint32_t a_lbo = a_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
-          const uint32_t b_lbo = b_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
+          const uint32_t a_addr = a_base + u * a_step;
+          const uint32_t b_addr = b_base + u * b_step;
+          // K-major: 16 contraction elements = 32 bytes inside the swizzled 128-byte row.
+          // MN-major: 16 contraction elements = 16 rows of 128 bytes = two 8-row groups.
+          // The address field counts 16-byte units and cannot carry out of its 14 bits (shared
+          // memory ends below 256 KiB), so a k-step is an addition to the whole descriptor.
+          const uint64_t adesc0 = A_MN ? smem_desc_sw128(a_addr, a_lbo, 1024) : smem_desc_sw128(a_addr, 16, 1024);
+          const uint64_t bdesc0 = B_MN ? smem_desc_sw128(b_addr, b_lbo, 1024) : smem_desc_sw128(b_addr, 16, 1024);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
-            // K-major: 16 contraction elements = 32 bytes inside the swizzled 128-byte row.
-            // MN-major: 16 contraction elements = 16 rows of 128 bytes = two 8-row groups.
-            const uint64_t adesc = A_MN ? smem_desc_sw128(a_addr + k * 2048, a_lbo, 1024)
-                                        : smem_desc_sw128(a_addr + k * 32, 16, 1024);
-            const uint64_t bdesc = B_MN ? smem_desc_sw128(b_addr + k * 2048, b_lbo, 1024)
-                                        : smem_desc_sw128(b_addr + k * 32, 16, 1024);
+            const uint64_t adesc = adesc0 + static_cast<uint64_t>(k * (A_MN ? 2048 / 16 : 32 / 16));
+            const uint64_t bdesc = bdesc0 + static_cast<uint64_t>(k * (B_MN ? 2048 / 16 : 32 / 16));
             const uint32_t accum = (kb > kb_begin || k > 0) ? 1u : 0u;
             if (I8) {
               if (CTA2) umma_i8_pair(d_tmem, adesc, bdesc, idesc, accum); else umma_i8(d_tmem, adesc, bdesc, idesc, accum);
@@ -636,7 +651,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // next tile's column scales and biases: loaded now, parked in registers behind this tile's work
       float nsc[4] = {0.f, 0.f, 0.f, 0.f}, nbi[4] = {0.f, 0.f, 0.f, 0.f};
       int nzw[4] = {0, 0, 0, 0};
-      if (FWD && has_next) {
+      // (a tile list with one tile column keeps the same scales from tile to tile: nothing to load)
+      const bool new_cols = has_next && (gn.n0 != g.n0 || gn.jb0 != g.jb0);
+      if (FWD && new_cols) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int64_t c = static_cast<int64_t>(gn.n0) + gn.jb0 * bc + lane + 32 * i;
@@ -841,7 +858,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           pp[1] = -xq.s * acc_c;     // Eq. 1: d(dequantised)/dZ = -s on clipped elements, 0 elsewhere
         }
       }
-      if (FWD && has_next) {
+      if (FWD && new_cols) {
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

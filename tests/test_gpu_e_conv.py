@@ -61,6 +61,8 @@ CASES = [
     _case("c3x3_shared_cin128", 2, 16, 24, 128, 136, 3, 1, seed=25),
     _case("c3x3_shared_valid_f32", 1, 16, 24, 64, 64, 3, 0, dtype=torch.float32, seed=26),
     _case("c4x4_shared_s2", 2, 32, 48, 64, 64, 4, 1, seed=27, stride=2),
+    _case("c3x3_shared_resident_2chunks", 2, 16, 24, 128, 64, 3, 1, seed=40),      # resident weights over two channel chunks
+    _case("c3x3_shared_two_tile_columns", 1, 16, 16, 64, 320, 3, 1, seed=41),      # several tile columns: weights staged per stage
     _case("resnet_56_64to64_3x3_b2", 2, 56, 56, 64, 64, 3, 1, seed=28),
     # the CIFAR-10 ResNet-20's layer shapes (16 / 32 / 64 channels on 32 x 32, 16 x 16 and 8 x 8 maps)
     _case("resnet20_stem", 2, 32, 32, 8, 16, 3, 1, seed=34),

@@ -208,7 +208,13 @@ template <typename T>
 __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab, float* sh /* [8][256] */) {
   const T* dY = static_cast<const T*>(a.dY);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t c0 = static_cast<int64_t>(cb) * 256 + lane * 8;
+  // Narrow matrices (N a power of two up to 128): a row needs only N / 8 lanes, so a warp takes
+  // 32 / (N / 8) rows per pass instead of leaving most of its lanes without a column.
+  int lpr = 32;
+  if (a.N <= 128 && (a.N & (a.N - 1)) == 0) lpr = static_cast<int>(a.N >> 3);
+  const int R = 32 / lpr;                        // rows per warp and pass
+  const int rs = lane / lpr, cl = lane - rs * lpr;
+  const int64_t c0 = static_cast<int64_t>(cb) * 256 + cl * 8;
   const int64_t rows = ceil_div(a.M, static_cast<int64_t>(a.slabs));
   const int64_t m_lo = slab * rows;
   const int64_t m_hi = (m_lo + rows < a.M) ? m_lo + rows : a.M;
@@ -216,24 +222,31 @@ __device__ __forceinline__ void job_dy_pass(const PrepArgs& a, int cb, int slab,
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
   if (c0 < a.N) {
-    for (int64_t m = m_lo + warp; m < m_hi; m += 32) {
+    for (int64_t m = m_lo + warp * R + rs; m < m_hi; m += 32 * R) {
       float v[4][8];
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        if (m + 8 * u < m_hi) ld8<T>(dY + (m + 8 * u) * a.N + c0, v[u]);
+        if (m + 8 * R * u < m_hi) ld8<T>(dY + (m + 8 * R * u) * a.N + c0, v[u]);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        if (m + 8 * u < m_hi) {
+        if (m + 8 * R * u < m_hi) {
 #pragma unroll
           for (int j = 0; j < 8; ++j) acc[j] += v[u][j];
-          if (a.dYb) st8(a.dYb + (m + 8 * u) * a.N + c0, v[u]);
+          if (a.dYb) st8(a.dYb + (m + 8 * R * u) * a.N + c0, v[u]);
         }
       }
     }
   }
-  if (a.colsum_ws) {
+  // the lanes that shared a column group add up (fixed order: reproducible)
+  for (int off = lpr; off < 32; off <<= 1) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) sh[warp * 256 + lane * 8 + j] = acc[j];
+    for (int j = 0; j < 8; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
+  }
+  if (a.colsum_ws) {
+    if (rs == 0) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) sh[warp * 256 + cl * 8 + j] = acc[j];
+    }
     __syncthreads();
     const int64_t c = static_cast<int64_t>(cb) * 256 + threadIdx.x;
     if (c < a.N) {

@@ -52,10 +52,12 @@ def _batch64_cases():
     filter column sharing one box, weights resident in shared memory) and the stride-2 3x3 that
     opens the second stage."""
     rn = {c.name: c for c in I.resnet50(64)}
-    return I.config3() + [rn["rn50_stem"], rn["rn50_s1b1_b"], rn["rn50_s2b1_b"]]
+    r20 = {c.name: c for c in I.resnet20(64)}
+    # ... and two layers of the CIFAR-10 ResNet-20 (16 channels: grad-input on strips of 4 pixels)
+    return I.config3() + [rn["rn50_stem"], rn["rn50_s1b1_b"], rn["rn50_s2b1_b"], r20["rn20_stem"], r20["rn20_s1b1_a"]]
 
 
-@pytest.mark.parametrize("li", range(11))
+@pytest.mark.parametrize("li", range(13))
 def test_config3_layer_batch64(ctx, li):
     case = _batch64_cases()[li]
     T = I.make_tensors(case)
@@ -111,7 +113,7 @@ def test_config3_layer_batch64(ctx, li):
 
     # sampled selected channels over the whole batch (dY is bf16: both operand models coincide)
     rng = np.random.default_rng(li)
-    pick = np.unique(np.concatenate([[0, k - 1], rng.choice(k, 6, replace=False)]))
+    pick = np.unique(np.concatenate([[0, k - 1], rng.choice(k, min(6, k), replace=False)]))
     d = O.conv_backward_efqat_direct(I.as_f64(T["dY"]), I.as_f64(T["X"]), W64, s_w, s_x, z_x, idx[pick],
                                      case.w_bits, case.x_bits, case.stride, case.pad, operand_model="bf16")
     U.assert_bf16_class(dW[pick], d["dW_sel"], name + " dW_sel sampled channels")

@@ -48,16 +48,6 @@ __device__ __forceinline__ uint32_t sw128_off(int r, int j) { return r * 128 + (
 template <typename T>
 __device__ __forceinline__ void load8(const T* p, float (&v)[8]);
 template <>
-__device__ __forceinline__ void load8<bf16>(const bf16* p, float (&v)[8]) {
-  const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
-  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
-}
-template <>
 __device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
   const float4 a = __ldg(reinterpret_cast<const float4*>(p));
   const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
@@ -131,7 +121,6 @@ __global__ void __launch_bounds__(SK_THREADS, 2) skinny_fwd_kernel(const __grid_
   const uint32_t tmem_base = tmem_slot;
   const uint32_t idesc = instr_desc_bf16(SK_ROWS, bn, 0, 0);
   const T* X = static_cast<const T*>(a.X);
-  T* Y = static_cast<T*>(a.Y);
   constexpr int PIECES = SK_ROWS * KB * 8 / SK_THREADS;     // 16-byte pieces of the A tile per thread: 4 or 8
 
   // raw X of a tile, one 8-element piece per (thread, i), kept as loaded (16 bytes of bf16 or 32

@@ -208,7 +208,11 @@ typedef struct {
 } efqat_net_layer;
 /* Forward of layers[0..L) in order / backward of layers[L-1..0] in reverse order, enqueued on
  * one stream with no host synchronisation in between (each launch overlaps its set-up with
- * the tail of the one before it).  Stops at, and returns, the first host-side error. */
+ * the tail of the one before it).  Stops at, and returns, the first host-side error.
+ * Layers may share one workspace; when neighbouring layers have disjoint workspaces (two buffers
+ * taken in turn are enough) the backward saves a launch per layer: a layer's last launch (the
+ * reduction of its partial sums, masks, optional SGD) then shares a launch with the first one of
+ * the layer processed next.  Results are the same bits either way. */
 int efqat_network_fwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream);
 int efqat_network_bwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream);
 /* efqat_weight_cache_update on rows idx of every layer that has a cache and k_sel > 0 (after

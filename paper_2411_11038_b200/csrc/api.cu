@@ -574,11 +574,20 @@ int fwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
 
 // Backward of one layer.  cache != NULL: the grad-input GEMM reads the dequantised weights of the
 // layer's cache instead of rebuilding them (W is still read for the clip mask of the unfrozen rows).
+// Chaining of the finalize launches over the layers of a network backward: a layer's finalize work
+// (reduction of its partial products, clip masks, dS / db, optional SGD) is independent of the next
+// layer's prepare jobs, so it may ride in that layer's prepare launch instead of a launch of its own.
+struct FinChain {
+  FinArgs pending;       // finalize work of the layer before, not launched yet
+  bool has_pending;
+  bool defer;            // this layer's finalize may be left pending for the next call
+};
+
 int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q, const void* dY, const void* X,
              const float* W, const float* s_w, const float* s_x, const float* z_x, const int32_t* idx, int64_t k_sel,
              void* dX, float* dW_sel, float* dS_w_sel, float* dS_x, float* dZ_x, float* db_or_null,
              const efqat_sgd* opt_or_null, void* ws, size_t ws_bytes, const void* cache, size_t cache_bytes,
-             efqat_stream_t stream) {
+             efqat_stream_t stream, FinChain* chain = nullptr) {
   if (!ctx || !dY || !X || !W || !s_w || !s_x || !dX || !dS_x || !dZ_x) return EFQAT_ERR_NULL;
   int rc = check_layer(layer, q);
   if (rc != EFQAT_OK) return rc;
@@ -611,6 +620,10 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   if (one_pass_bwd(layer)) {
     // short contraction: one launch reads dY and X once and leaves per-CTA partials for the finalize launch
     const int grid = skinny_bwd_grid(M, ctx->sm_count);
+    if (chain && chain->has_pending) {          // no prepare launch here to carry it
+      launch_finalize(chain->pending, st);
+      chain->has_pending = false;
+    }
     rc = run_skinny_bwd(M, N, dY, X, dX, W, cache ? wc.what : nullptr, s_w, q->w_bits, s_x, z_x, q->x_bits,
                         q->x_symmetric, gathered ? idx : nullptr, k_sel, w.P, db_or_null ? w.colsum : nullptr, w.dxpart,
                         ctx->d_status, ctx->sm_count, st);
@@ -626,7 +639,12 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
     fa.dx_partials = w.dxpart; fa.n_partials = grid * 8; fa.dS_x = dS_x; fa.dZ_x = dZ_x;
     fa.colsum_ws = w.colsum; fa.slabs = grid; fa.db = db_or_null;
     fa.status = ctx->d_status;
-    launch_finalize(fa, st);
+    if (chain && chain->defer) {
+      chain->pending = fa;
+      chain->has_pending = true;
+    } else {
+      launch_finalize(fa, st);
+    }
     return last_error();
   }
   // a2: one launch: dequantised weight operand, activation codes (only when some channel is
@@ -643,7 +661,8 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   pa.colsum_ws = db_or_null ? w.colsum : nullptr;
   pa.idx = idx; pa.k_sel = k_sel; pa.pitch = w.pitch; pa.dYsel = gathered ? w.dYsel : nullptr;
   pa.status = ctx->d_status;
-  launch_prepare(pa, 1, act_bf16, st);
+  launch_prepare(pa, 1, act_bf16, st, (chain && chain->has_pending) ? &chain->pending : nullptr);
+  if (chain) chain->has_pending = false;
   // a4 + a5: dX = (dY W^) masked, with the dS_x / dZ_x partial sums in the epilogue
   int tiles = 0, dx_grid = 0, dw_splits = w.splits;
   const bool sconv = spatial_conv(layer);
@@ -801,7 +820,12 @@ int bwd_impl(efqat_ctx* ctx, const efqat_layer_desc* layer, const efqat_qspec* q
   fa.dx_partials = w.dxpart; fa.n_partials = tiles; fa.dS_x = dS_x; fa.dZ_x = dZ_x;
   fa.colsum_ws = w.colsum; fa.slabs = prepare_slabs(M, N); fa.db = db_or_null;
   fa.status = ctx->d_status;
-  launch_finalize(fa, st);
+  if (chain && chain->defer) {
+    chain->pending = fa;
+    chain->has_pending = true;
+  } else {
+    launch_finalize(fa, st);
+  }
   return last_error();
 }
 
@@ -891,14 +915,31 @@ int efqat_network_fwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqa
 int efqat_network_bwd(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream) {
   if (!ctx || !layers) return EFQAT_ERR_NULL;
   if (L < 1) return EFQAT_ERR_SHAPE;
+  // A layer's finalize work rides in the prepare launch of the layer processed next whenever the two
+  // layers' workspaces are disjoint (the prepare jobs write theirs while the finalize blocks read the
+  // other); layers that share a workspace keep one finalize launch each.
+  FinChain ch = {};
   for (int l = L - 1; l >= 0; --l) {
     const efqat_net_layer& n = layers[l];
+    ch.defer = false;
+    if (l > 0) {
+      const efqat_net_layer& m = layers[l - 1];
+      const char* a0 = static_cast<const char*>(n.ws);
+      const char* b0 = static_cast<const char*>(m.ws);
+      ch.defer = n.ws && m.ws && (a0 + n.ws_bytes <= b0 || b0 + m.ws_bytes <= a0) && n.W != m.W;
+    }
     const int rc = bwd_impl(ctx, &n.layer, &n.q, n.dY, n.X, n.W, n.s_w, n.s_x, n.z_x, n.idx, n.k_sel, n.dX, n.dW_sel,
                             n.dS_w_sel, n.dS_x, n.dZ_x, n.db_or_null, n.opt_or_null, n.ws, n.ws_bytes,
-                            n.cache_or_null, n.cache_bytes, stream);
-    if (rc != EFQAT_OK) return rc;
+                            n.cache_or_null, n.cache_bytes, stream, &ch);
+    if (rc != EFQAT_OK || l == 0) {
+      if (ch.has_pending) {          // a layer's call failed before its prepare launch: the work still pending goes out alone
+        if (guard_device(ctx) == EFQAT_OK) launch_finalize(ch.pending, stream);
+        ch.has_pending = false;
+      }
+      if (rc != EFQAT_OK) return rc;
+    }
   }
-  return EFQAT_OK;
+  return last_error();
 }
 
 int efqat_network_cache_update(efqat_ctx* ctx, int L, const efqat_net_layer* layers, efqat_stream_t stream) {

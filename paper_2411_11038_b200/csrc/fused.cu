@@ -307,11 +307,21 @@ __device__ __forceinline__ void job_gather(const PrepArgs& a, int block, int32_t
   }
 }
 
+__device__ __forceinline__ void finalize_body(const FinArgs& a, const int b, double (*shd)[256], float4* red);
+
+// Blocks [0, nb_prep) are the prepare jobs of one layer; blocks behind them (if any) are the
+// finalize work of ANOTHER layer whose GEMMs have just completed: in a chain of layers the two
+// are independent, and as one launch they cost one launch latency instead of two.
 template <int W_MODE, typename TX>
-__global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
-  __shared__ float sh[8 * 256];
+__global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a, const FinArgs f, const int nb_prep) {
+  __shared__ __align__(16) float sh[8 * 256];
   pdl_trigger();
   pdl_wait();
+  if (static_cast<int>(blockIdx.x) >= nb_prep) {
+    finalize_body(f, static_cast<int>(blockIdx.x) - nb_prep, reinterpret_cast<double(*)[256]>(sh),
+                  reinterpret_cast<float4*>(sh + 1024));
+    return;
+  }
   const int b = blockIdx.x;
   const int per_slab = a.col_blocks * a.dy_on + a.nb_g;
   const int nb_y = per_slab * a.slabs;
@@ -332,12 +342,8 @@ __global__ void __launch_bounds__(256, 3) prepare_kernel(const PrepArgs a) {
 }
 
 // ---- finalize: dW rows (mask, dS_w, optional SGD) | dS_x, dZ_x | db ------------------------
-__global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
-  __shared__ double shd[2][256];
-  __shared__ float4 red[256];
-  pdl_trigger();
-  pdl_wait();
-  const int b = blockIdx.x;
+// Block b of the finalize work of one layer; shd / red: 4 KiB of shared memory each.
+__device__ __forceinline__ void finalize_body(const FinArgs& a, const int b, double (*shd)[256], float4* red) {
   if (b < a.k_sel) {
     const int64_t i = b;
     const int64_t n = a.idx ? static_cast<int64_t>(a.idx[i]) : i;
@@ -470,6 +476,14 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
   }
 }
 
+__global__ void __launch_bounds__(256) finalize_kernel(const FinArgs a) {
+  __shared__ double shd[2][256];
+  __shared__ float4 red[256];
+  pdl_trigger();
+  pdl_wait();
+  finalize_body(a, blockIdx.x, shd, red);
+}
+
 }  // namespace
 
 // Row slabs of the dY pass: blocks of 256 columns x one slab of rows, 64 rows (32 KiB of
@@ -491,7 +505,12 @@ static int flat_blocks(int64_t vectors, int64_t per_block) {
   return static_cast<int>(nb);
 }
 
-void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
+static int finalize_blocks(const FinArgs& a) {
+  const int nb_db = a.db ? static_cast<int>(ceil_div(a.N, 32)) : 0;
+  return static_cast<int>(a.k_sel) + 1 + nb_db;
+}
+
+void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st, const FinArgs* fin) {
   a.nb_w = flat_blocks(a.N * (a.K / 8), 256 * 4);       // 32 KiB of fp32 weights per block
   if (a.i8) a.nb_w = static_cast<int>(ceil_div(a.N, 8) < 148 * 12 ? ceil_div(a.N, 8) : 148 * 12);   // a warp per row
   if (!a.W) a.nb_w = 0;                          // weight operand supplied by the layer's cache
@@ -503,21 +522,22 @@ void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st) {
   a.slabs = prepare_slabs(a.M, a.N);
   a.dy_on = (a.dY && (a.colsum_ws || a.dYb)) ? 1 : 0;
   const int nb_y = (a.col_blocks * a.dy_on + a.nb_g) * a.slabs;
-  const int grid = a.nb_w + a.nb_x + nb_y;
+  const int nb_prep = a.nb_w + a.nb_x + nb_y;
+  const FinArgs f = fin ? *fin : FinArgs{};
+  const int grid = nb_prep + (fin ? finalize_blocks(f) : 0);
   if (grid == 0) return;                         // cached weights, nothing unfrozen, no bias gradient wanted
   count_launches(1);
   if (w_mode == 0) {
-    if (act_bf16) launch_dependent(prepare_kernel<0, bf16>, grid, 256, 0, st, 1, a);
-    else launch_dependent(prepare_kernel<0, float>, grid, 256, 0, st, 1, a);
+    if (act_bf16) launch_dependent(prepare_kernel<0, bf16>, grid, 256, 0, st, 1, a, f, nb_prep);
+    else launch_dependent(prepare_kernel<0, float>, grid, 256, 0, st, 1, a, f, nb_prep);
   } else {
-    if (act_bf16) launch_dependent(prepare_kernel<1, bf16>, grid, 256, 0, st, 1, a);
-    else launch_dependent(prepare_kernel<1, float>, grid, 256, 0, st, 1, a);
+    if (act_bf16) launch_dependent(prepare_kernel<1, bf16>, grid, 256, 0, st, 1, a, f, nb_prep);
+    else launch_dependent(prepare_kernel<1, float>, grid, 256, 0, st, 1, a, f, nb_prep);
   }
 }
 
 void launch_finalize(FinArgs a, cudaStream_t st) {
-  const int nb_db = a.db ? static_cast<int>(ceil_div(a.N, 32)) : 0;
-  const int grid = static_cast<int>(a.k_sel) + 1 + nb_db;
+  const int grid = finalize_blocks(a);
   count_launches(1);
   launch_dependent(finalize_kernel, grid, 256, 0, st, 1, a);
 }

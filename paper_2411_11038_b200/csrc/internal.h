@@ -80,7 +80,7 @@ struct PrepArgs {
   int nb_g, nb_w, nb_x, col_blocks, slabs, dy_on;   // filled by launch_prepare
 };
 int prepare_slabs(int64_t M, int64_t N);
-void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st);
+
 // One launch behind the GEMMs: dW rows (split reduction, clip mask, dS_w, optional SGD),
 // dS_x / dZ_x from the per-tile partials, db from the column-sum partials.
 struct FinArgs {
@@ -95,6 +95,8 @@ struct FinArgs {
   int* status;
 };
 void launch_finalize(FinArgs a, cudaStream_t st);
+// fin != null: the finalize work of another layer rides behind the prepare jobs in the same launch
+void launch_prepare(PrepArgs a, int w_mode, int act_bf16, cudaStream_t st, const FinArgs* fin = nullptr);
 
 // ---- optim.cu -----------------------------------------------------------------------
 void launch_qparam_adam(const efqat_adam& a, const efqat_qparam_state& st, int64_t N, const int32_t* idx,

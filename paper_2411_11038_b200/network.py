@@ -57,11 +57,12 @@ class EfqatNetwork:
     use_cache: keep a weight-operand cache per layer and refresh only the stepped rows.
     sgd = (lr, momentum, weight_decay) enables the fused update of the unfrozen rows;
     adam = dict(lr=..., log2_scale=...) enables the optimizer of the quantization parameters.
+    alternate_ws: two workspaces taken in turn (a launch less per layer in the backward) instead of one.
     """
 
     def __init__(self, ctx: B.Context, layers: Sequence[LayerState], mode: int, budget, f_samples: int,
                  batch_samples: int, use_cache: bool = True, sgd=None, adam: Optional[dict] = None,
-                 share_outputs: bool = True, want_db: bool = True):
+                 share_outputs: bool = True, want_db: bool = True, alternate_ws: bool = True):
         self.ctx, self.layers, self.mode = ctx, list(layers), mode
         self.schedule = FreezeSchedule(f_samples, batch_samples)
         self.use_cache = use_cache
@@ -98,18 +99,20 @@ class EfqatNetwork:
             spec = B.QSpec(c.w_bits, c.x_bits, 1 if c.x_symmetric else 0)
             ws_need = max(ws_need, B.workspace_bytes(d, spec, km))
             descs.append((d, spec))
-        self.ws = B.alloc_workspace(ws_need, dev)
+        # two workspaces, taken in turn: neighbouring layers then never share one, which lets the library put
+        # a layer's finalize work into the next layer's prepare launch (see efqat_network_bwd)
+        self.ws = [B.alloc_workspace(ws_need, dev) for _ in range(2 if alternate_ws else 1)]
         self.plans: List[B.LayerPlan] = []
         by_shape = {}
         self.sgds = []
         entries = []
         self.qopts = []
-        for st, km in zip(self.layers, k_max):
+        for li, (st, km) in enumerate(zip(self.layers, k_max)):
             c = st.case
             key = (c.M, c.N, c.K, c.act_dtype, c.conv, c.R, c.stride)
             plan = B.LayerPlan(ctx, c.M, c.N, c.K, c.act_dtype, c.w_bits, c.x_bits, c.x_symmetric, km, dev,
                                conv=geom(c), x_shape=tuple(st.X.shape), y_shape=tuple(st.dY.shape),
-                               with_cache=use_cache, ws=self.ws,
+                               with_cache=use_cache, ws=self.ws[li % len(self.ws)],
                                outputs=by_shape.get(key) if share_outputs else None)
             by_shape.setdefault(key, plan)
             self.plans.append(plan)

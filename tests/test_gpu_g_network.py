@@ -226,3 +226,35 @@ def test_network_calls_on_convolutions_equal_layer_calls(ctx):
     if k0:
         U.assert_bf16_class(net.plans[0].dW_sel[:k0].cpu().numpy().reshape(ex["dW_sel"].shape), ex["dW_sel"],
                             "input layer dW_sel through the network call")
+
+
+def test_shared_and_alternating_workspaces_give_the_same_bits(ctx):
+    """efqat_network_bwd puts a layer's finalize work into the next layer's prepare launch only when
+    their workspaces are disjoint: with one shared workspace every layer keeps its own finalize
+    launch.  Both ways must produce the same bits, over a stack that mixes the general backward, a
+    layer with the one-pass backward (no prepare launch to ride in) and frozen layers."""
+    shapes = [(384, 512, 512), (1024, 64, 256), (384, 512, 1024), (1024, 64, 128), (384, 1024, 512)]
+    stack = _stack(ctx, shapes, 1500)
+    total = sum(c.N for c, _ in stack)
+    outs = []
+    for alternate in (True, False):
+        states = [NW.LayerState(c, T["W"].cuda().clone(), T["X"].cuda(), T["dY"].cuda(), T["bias"].cuda())
+                  for c, T in stack]
+        net = NW.EfqatNetwork(ctx, states, B.CWPN, B.ratio_to_k(0.2, total), f_samples=1, batch_samples=1,
+                              use_cache=True, sgd=(2e-5, 0.9, 1e-4), adam=None, share_outputs=False,
+                              alternate_ws=alternate)
+        net.reselect()
+        n0 = ctx.launch_count() if hasattr(ctx, "launch_count") else None
+        net.backward()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        outs.append((states, net, n0))
+    (sa, na, _), (sb, nb, _) = outs
+    assert na.counts() == nb.counts()
+    for l, (pa, pb) in enumerate(zip(na.plans, nb.plans)):
+        k = na.counts()[l]
+        assert torch.equal(pa.dX, pb.dX), f"layer {l}: dX"
+        assert torch.equal(pa.dW_sel[:k], pb.dW_sel[:k]) and torch.equal(pa.dS_w_sel[:k], pb.dS_w_sel[:k])
+        assert torch.equal(pa.dS_x, pb.dS_x) and torch.equal(pa.dZ_x, pb.dZ_x) and torch.equal(pa.db, pb.db)
+    for x, y in zip(sa, sb):
+        assert torch.equal(x.W, y.W) and torch.equal(x.mom, y.mom)

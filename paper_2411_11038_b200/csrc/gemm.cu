@@ -468,8 +468,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // tiles differ in width (a ragged last tile column), the k-range only for split contractions
       // (both need integer divisions), and the operand descriptors of a k-block are built once and
       // advanced by adding to their address field.
-      const bool ragged_n = (p.Nc % p.BN) != 0;
-      const uint32_t idesc_full = I8 ? instr_desc_i8(TILE_M, p.BN, p.a_signed, 1) : instr_desc_bf16(TILE_M, p.BN, A_MN, B_MN);
+      // (one tile column: every tile has the same width, ragged or not)
+      const bool ragged_n = p.tiles_n > 1 && (p.Nc % p.BN) != 0;
+      const int n_first = static_cast<int>(((p.Nc < p.BN ? p.Nc : p.BN) + 15) & ~static_cast<int64_t>(15));
+      const uint32_t idesc_full = I8 ? instr_desc_i8(TILE_M, n_first, p.a_signed, 1) : instr_desc_bf16(TILE_M, n_first, A_MN, B_MN);
       const bool a_mrg = A_MN && p.merged, b_mrg = B_MN && p.merged;
       const uint32_t a_lbo = a_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
       const uint32_t b_lbo = b_mrg ? p.kps * CHUNK_BYTES : CHUNK_BYTES;
@@ -489,8 +491,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (n_eff > p.BN) n_eff = p.BN;
           n_eff = (n_eff + 15) & ~15;
           idesc = I8 ? instr_desc_i8(TILE_M, n_eff, p.a_signed, 1) : instr_desc_bf16(TILE_M, n_eff, A_MN, B_MN);
-          kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
-          kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
+          if (p.splits > 1) {
+            kb_begin = static_cast<int>(static_cast<int64_t>(split) * p.nkb / p.splits);
+            kb_end = static_cast<int>(static_cast<int64_t>(split + 1) * p.nkb / p.splits);
+          }
         }
         const int buf = acc_it & 1;
         // wait until the epilogue has drained this accumulator (two tiles ago)

@@ -279,19 +279,21 @@ struct __align__(16) WsCtl {
   int abort_flag;
 };
 
-template <int KB /* 64-wide k-blocks of the contraction: 1 or 2 */>
-__global__ void __launch_bounds__(WS_THREADS, 1)
+template <int KB /* 64-wide k-blocks of the contraction: 1 or 2 */, int NW /* worker warps: 8 or 16 */>
+__global__ void __launch_bounds__(64 + 32 * NW, 1)
 skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
                      const SkinnyFwdArgs a) {
   constexpr int TILE = KB * WS_T16K;                       // one X tile / one operand buffer
   constexpr int WS_STAGES = KB == 1 ? 3 : 2;               // X tiles in flight (compile time: the stage index is n % WS_STAGES)
-  constexpr int STG_BUFS = KB == 1 ? 2 : 1;                // staging buffers per epilogue warp
+  constexpr int STG_BUFS = (KB == 1 && NW == 8) ? 2 : 1;   // staging buffers per epilogue warp
+  constexpr int G = NW / 4;                                // worker warps per TMEM lane quarter
+  constexpr int THREADS = 64 + 32 * NW;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* b_tile = smem;                                  // [KB][BN rows][128 B] weight codes, K-major
   uint8_t* xc_t = b_tile + KB * a.BN * 128;                // [2][KB][128 rows][128 B] centred activation codes
   uint8_t* ring = xc_t + 2 * TILE;                         // [stages][KB][128 rows][128 B] raw X tiles
   uint8_t* stage = ring + WS_STAGES * TILE;                // [8 warps][stg_bufs][32 rows][128 B] output staging
-  float* sc = reinterpret_cast<float*>(stage + 8 * STG_BUFS * 4096);   // [BN] s_x * s_w[n]
+  float* sc = reinterpret_cast<float*>(stage + NW * STG_BUFS * 4096);   // [BN] s_x * s_w[n]
   float* bi = sc + a.BN;                                   // [BN] bias[n]
   WsCtl* ctl = reinterpret_cast<WsCtl*>(bi + a.BN);
 
@@ -302,13 +304,13 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   if (tid == 0) {
     for (int s = 0; s < WS_STAGES; ++s) {
       mbar_init(&ctl->full[s], 1);
-      mbar_init(&ctl->empty[s], 8);
+      mbar_init(&ctl->empty[s], NW);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&ctl->xc_full[b], 8);
+      mbar_init(&ctl->xc_full[b], NW);
       mbar_init(&ctl->xc_empty[b], 1);
       mbar_init(&ctl->acc_full[b], 1);
-      mbar_init(&ctl->acc_empty[b], 8);
+      mbar_init(&ctl->acc_empty[b], NW);
     }
     mbar_init(&ctl->drain, 1);
     ctl->abort_flag = 0;
@@ -333,7 +335,7 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     }
   }
   bool bad_scale = false;
-  for (int n = tid - 32; n >= 0 && n < a.BN; n += WS_THREADS - 32) {
+  for (int n = tid - 32; n >= 0 && n < a.BN; n += THREADS - 32) {
     if (n >= bn) {
 #pragma unroll
       for (int j = 0; j < 8 * KB; ++j)
@@ -378,7 +380,7 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   const ActQ xq = make_actq(a.s_x, a.z_x, a.x_bits, a.x_sym, &bad_x);
   if ((bad_scale || (bad_x && tid == 0)) && blockIdx.x == 0) record_status(a.status, EFQAT_DEV_BAD_SCALE);
   __syncthreads();
-  for (int n = tid; n < a.BN; n += WS_THREADS) sc[n] *= xq.s;
+  for (int n = tid; n < a.BN; n += THREADS) sc[n] *= xq.s;
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -439,7 +441,7 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     int st_it = 0;
     bool ok = true;
     // Eq. 1 on this lane's 32 * KB values (row `row`, half h of its pieces) of tile number n
-    constexpr int NP = 4 * KB;                               // 16-byte pieces per lane
+    constexpr int NP = 8 * KB / G;                           // 16-byte pieces per lane
     auto piece_off = [&](int i) { const int p = h * NP + i; return (p >> 3) * WS_T16K + sw128_off(row, p & 7); };
     auto quant_tile = [&](int n) -> bool {
       const int s = n % WS_STAGES, b = n & 1;
@@ -474,7 +476,7 @@ skinny_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     };
     if (my_tiles > 0) ok = quant_tile(0);
     const int rounds = bn / 64;                              // 128-byte rounds of output columns
-    const int rd0 = h ? (rounds + 1) / 2 : 0, rd1 = h ? rounds : (rounds + 1) / 2;
+    const int rd0 = (rounds * h + G - 1) / G, rd1 = (rounds * (h + 1) + G - 1) / G;
     for (int n = 0; n < my_tiles && ok; ++n) {
       const int t = blockIdx.x + n * gridDim.x;
       const int b = n & 1;
@@ -566,14 +568,18 @@ int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X,
     // persistent warp-specialised form: one CTA per SM and column chunk.  K = 128 doubles the weight,
     // operand and ring tiles: two X tiles in flight and one staging buffer per warp then fill the SM.
     const int kbs = a.K / 64;
+    // Worker warps: 16 where every one of them gets a 64-column round of the epilogue (256 columns;
+    // measured 2.3 -> 2.05 us per tile), else 8 (narrower tiles: 16 cost 2 us per launch; K = 128 has no
+    // shared memory for 16 staging blocks).
+    const int nw = (kbs == 1 && a.BN >= 256) ? 16 : 8;
     a.stages = kbs == 1 ? 3 : 2;
-    a.stg_bufs = kbs == 1 ? 2 : 1;
+    a.stg_bufs = (kbs == 1 && nw == 8) ? 2 : 1;
     CUtensorMap tmX, tmY;
     if (tensor_map_2d(&tmX, X, 1, M, K, K, SK_ROWS, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
     if (tensor_map_2d(&tmY, Y, 1, M, N, N, 32, 128) != EFQAT_OK) return EFQAT_ERR_CUDA;
-    const size_t smem = static_cast<size_t>(kbs) * a.BN * 128 + (2 + a.stages) * kbs * WS_T16K + 8 * a.stg_bufs * 4096 +
+    const size_t smem = static_cast<size_t>(kbs) * a.BN * 128 + (2 + a.stages) * kbs * WS_T16K + nw * a.stg_bufs * 4096 +
                         2 * a.BN * sizeof(float) + sizeof(WsCtl);
-    auto kern = kbs == 1 ? skinny_fwd_ws_kernel<1> : skinny_fwd_ws_kernel<2>;
+    auto kern = kbs == 2 ? skinny_fwd_ws_kernel<2, 8> : (nw == 16 ? skinny_fwd_ws_kernel<1, 16> : skinny_fwd_ws_kernel<1, 8>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
       return EFQAT_ERR_CUDA;
     int ctas = sm_count / chunks;
@@ -582,7 +588,7 @@ int run_skinny_fwd(int64_t M, int64_t N, int64_t K, int act_bf16, const void* X,
     count_launches(1);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(ctas), static_cast<unsigned>(chunks));
-    cfg.blockDim = dim3(WS_THREADS);
+    cfg.blockDim = dim3(64 + 32 * nw);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
